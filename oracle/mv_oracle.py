@@ -1,0 +1,202 @@
+"""CPU oracle for the majority-vote sparse DSGD step (SSGD-MV, Algorithm 1).
+
+TEST INFRASTRUCTURE ONLY.  This module is the slow, plain statement of what one
+step computes, written from the paper's definitions with numpy.  It is imported
+by the tests, by the smoke check and by the benchmark's CPU-baseline leg, and by
+nothing else; it shares no code with the CUDA library and never imports it.
+
+One step, for N workers holding d parameters each (Algorithm 1, worker side and
+parameter-server side collapsed onto one machine):
+
+  1. acc_n   = grads_n + err_n                      error feedback (Alg. 1, accumulate step)
+  2. M_n     = S_top(|acc_n|, K)                    per-worker top-K mask (Eq. 6 / S_top)
+  3. votes   = sum_n M_n                            vote count per coordinate (Eq. 9)
+  4. M       = S_top(votes, K)                      the K most voted coordinates (Eq. 9)
+  5. out_val = (1/N) sum_n (M (x) acc_n) on supp(M) shared-mask aggregate (Eq. 8, 1/N as in Eq. 7's G~)
+  6. err_n   = acc_n - M (x) acc_n                  residual (Alg. 1, error update)
+
+Readings where the paper is silent (each is also listed in the design notes):
+  * "largest absolute value" is ordered by key(x) = bits(x) & 0x7fffffff, the
+    IEEE-754 binary32 pattern with the sign cleared, which is monotone in |x|.
+  * ties in either S_top go to the lowest coordinate index, so the selected set
+    is the first K elements of the strict total order (key descending, index
+    ascending) and is therefore unique.
+  * supports are reported as ascending index lists.
+  * the aggregate is the mean (the text's 1/N), accumulated in binary64 in
+    worker order, divided by N and rounded once to binary32.
+  * the residual is "+0.0 on the mask, a bit copy elsewhere" (equal to the
+    subtraction for all finite values).
+  * acc is one binary32 round-to-nearest add, denormals kept.
+
+Every selection is written twice: `*_by_sort` is the definition executed with a
+full stable sort; the plain name reaches the same unique set with a library
+selection routine (numpy.partition) so that full-size inputs finish in seconds.
+The tests pin the two against each other, against a pure-Python brute force and
+against hand-worked examples.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+_SIGN_CLEAR = np.uint32(0x7FFFFFFF)
+
+
+# ----------------------------------------------------------------------------
+# step 1: error feedback (Algorithm 1, "Delta-bar = Delta + e")
+# ----------------------------------------------------------------------------
+def accumulate(grads: np.ndarray, err: np.ndarray) -> np.ndarray:
+    """acc[n, j] = fl32(err[n, j] + grads[n, j])."""
+    grads = np.asarray(grads, dtype=np.float32)
+    err = np.asarray(err, dtype=np.float32)
+    assert grads.shape == err.shape
+    with np.errstate(all="ignore"):
+        return np.add(err, grads, dtype=np.float32)
+
+
+def magnitude_key(x: np.ndarray) -> np.ndarray:
+    """key(x): the binary32 pattern with the sign bit cleared (monotone in |x|)."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    return x.view(np.uint32) & _SIGN_CLEAR
+
+
+# ----------------------------------------------------------------------------
+# S_top on an integer score vector: the K largest scores, ties to the lowest index
+# ----------------------------------------------------------------------------
+def _stop_by_sort(score: np.ndarray, K: int):
+    """Definition executed: stable sort by descending score, take the first K."""
+    score = np.asarray(score)
+    d = score.shape[0]
+    assert 1 <= K <= d
+    # ascending stable sort of (max - score) == descending score, index ascending
+    inv = score.max().astype(np.int64) - score.astype(np.int64)
+    order = np.argsort(inv, kind="stable")
+    chosen = order[:K]
+    thr = score[chosen[-1]]
+    cnt_gt = int(np.count_nonzero(score > thr))
+    cnt_eq = int(np.count_nonzero(score == thr))
+    return np.sort(chosen).astype(np.int32), thr, cnt_gt, cnt_eq
+
+
+def _stop(score: np.ndarray, K: int):
+    """Same set via a selection routine: threshold = K-th largest score, then
+    everything above it plus the lowest-index (K - cnt_gt) elements equal to it."""
+    score = np.asarray(score)
+    d = score.shape[0]
+    assert 1 <= K <= d
+    thr = np.partition(score, d - K)[d - K]          # K-th largest value
+    gt = score > thr
+    eq = score == thr
+    cnt_gt = int(np.count_nonzero(gt))
+    cnt_eq = int(np.count_nonzero(eq))
+    need = K - cnt_gt
+    assert 1 <= need <= cnt_eq
+    tie_rank = np.cumsum(eq, dtype=np.int64) - 1       # 0-based rank among the ties, by index
+    take = gt | (eq & (tie_rank < need))
+    return np.flatnonzero(take).astype(np.int32), thr, cnt_gt, cnt_eq
+
+
+# ----------------------------------------------------------------------------
+# step 2: per-worker top-K of |acc_n| (S_top, Eq. 6; Algorithm 1 worker side)
+# ----------------------------------------------------------------------------
+def worker_topk_by_sort(acc_row: np.ndarray, K: int):
+    """Returns (ascending int32 indices, threshold key T, cnt_gt, cnt_eq)."""
+    idx, thr, cnt_gt, cnt_eq = _stop_by_sort(magnitude_key(acc_row), K)
+    return idx, int(thr), cnt_gt, cnt_eq
+
+
+def worker_topk(acc_row: np.ndarray, K: int):
+    idx, thr, cnt_gt, cnt_eq = _stop(magnitude_key(acc_row), K)
+    return idx, int(thr), cnt_gt, cnt_eq
+
+
+def support_to_bits(idx: np.ndarray, d: int) -> np.ndarray:
+    """d-bit mask as ceil(d/32) uint32 words; bit b of word w is coordinate 32*w+b."""
+    flags = np.zeros(((d + 31) // 32) * 32, dtype=np.uint8)
+    flags[np.asarray(idx, dtype=np.int64)] = 1
+    return np.packbits(flags, bitorder="little").view(np.uint32).copy()
+
+
+# ----------------------------------------------------------------------------
+# step 3: vote count (Eq. 9, inner sum)
+# ----------------------------------------------------------------------------
+def count_votes(worker_idx, d: int) -> np.ndarray:
+    """votes[j] = number of workers whose top-K support contains j."""
+    votes = np.zeros(d, dtype=np.int64)
+    for idx in worker_idx:
+        votes[np.asarray(idx, dtype=np.int64)] += 1   # indices within one list are distinct
+    assert votes.max(initial=0) <= 255
+    return votes.astype(np.uint8)
+
+
+# ----------------------------------------------------------------------------
+# step 4: global mask = the K most voted coordinates (Eq. 9, outer S_top)
+# ----------------------------------------------------------------------------
+def select_mask_by_sort(votes: np.ndarray, K: int):
+    idx, thr, cnt_gt, cnt_eq = _stop_by_sort(np.asarray(votes), K)
+    return idx, int(thr), cnt_gt, cnt_eq
+
+
+def select_mask(votes: np.ndarray, K: int):
+    idx, thr, cnt_gt, cnt_eq = _stop(np.asarray(votes), K)
+    return idx, int(thr), cnt_gt, cnt_eq
+
+
+# ----------------------------------------------------------------------------
+# step 5: aggregate on the shared mask (Eq. 8 with the 1/N of the text)
+# ----------------------------------------------------------------------------
+def aggregate(acc: np.ndarray, idx: np.ndarray) -> np.ndarray:
+    """out_val[k] = fl32( (sum over workers, in worker order, in binary64) / N )."""
+    acc = np.asarray(acc, dtype=np.float32)
+    N = acc.shape[0]
+    cols = np.asarray(idx, dtype=np.int64)
+    total = np.zeros(cols.shape[0], dtype=np.float64)
+    with np.errstate(all="ignore"):
+        for n in range(N):
+            total = total + acc[n, cols].astype(np.float64)
+        return (total / np.float64(N)).astype(np.float32)
+
+
+# ----------------------------------------------------------------------------
+# step 6: residual (Algorithm 1, "e = Delta-bar - Delta-tilde")
+# ----------------------------------------------------------------------------
+def residual(acc: np.ndarray, idx: np.ndarray) -> np.ndarray:
+    out = np.array(acc, dtype=np.float32, copy=True)
+    out[:, np.asarray(idx, dtype=np.int64)] = np.float32(0.0)
+    return out
+
+
+# ----------------------------------------------------------------------------
+# the whole step
+# ----------------------------------------------------------------------------
+def mv_vote(grads, err, K: int, by_sort: bool = False):
+    """Steps 1-3.  Returns a dict with acc, worker_idx [N,K], worker_bits
+    [N,ceil(d/32)], votes [d] and thresh [N,3] = (T_n, cnt_gt, cnt_eq)."""
+    acc = accumulate(grads, err)
+    N, d = acc.shape
+    topk = worker_topk_by_sort if by_sort else worker_topk
+    worker_idx = np.empty((N, K), dtype=np.int32)
+    worker_bits = np.empty((N, (d + 31) // 32), dtype=np.uint32)
+    thresh = np.empty((N, 3), dtype=np.uint32)
+    for n in range(N):
+        idx, T, cnt_gt, cnt_eq = topk(acc[n], K)
+        worker_idx[n] = idx
+        worker_bits[n] = support_to_bits(idx, d)
+        thresh[n] = (T, cnt_gt, cnt_eq)
+    votes = count_votes(worker_idx, d)
+    return dict(acc=acc, worker_idx=worker_idx, worker_bits=worker_bits,
+                votes=votes, thresh=thresh)
+
+
+def mv_sparse_step(grads, err, K: int, by_sort: bool = False):
+    """One full step.  Returns a dict with everything the step defines:
+    acc, worker_idx, worker_bits, votes, thresh, out_idx [K], mask_bits,
+    vote_thresh = (v*, cnt_gt, cnt_eq), out_val [K] and the new err [N,d]."""
+    r = mv_vote(grads, err, K, by_sort=by_sort)
+    sel = select_mask_by_sort if by_sort else select_mask
+    out_idx, vstar, vgt, veq = sel(r["votes"], K)
+    r["out_idx"] = out_idx
+    r["mask_bits"] = support_to_bits(out_idx, r["acc"].shape[1])
+    r["vote_thresh"] = (vstar, vgt, veq)
+    r["out_val"] = aggregate(r["acc"], out_idx)
+    r["err"] = residual(r["acc"], out_idx)
+    return r
