@@ -1,0 +1,328 @@
+#!/usr/bin/env python
+"""Benchmark of the majority-vote sparse DSGD step.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c4|c1] [--impl ours|reference]
+
+A step is one whole pass of the hot path (error feedback, per-worker top-K, vote count, shared
+mask, aggregate, residual) over one batch of synthetic gradients; the residual is carried from
+step to step and every step gets fresh gradients from a pool that was generated before the timed
+region.  One JSON line is printed by rank 0.  With --gpus N > 1 (launched through torchrun) every
+rank runs an independent replica of the same workload: the path does not shard across devices.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+from paper_2011_06495_b200 import workloads as WL  # noqa: E402
+
+METRIC = "majority-vote sparse steps/s"
+UNIT = "steps/s"
+FALLBACK_HBM_GBS = 6650.0
+L2_BYTES = 126 * 1024 * 1024
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def kernel_source_hash():
+    src = os.path.join(ROOT, "paper_2011_06495_b200", "csrc", "mv_sparse.cu")
+    return hashlib.sha256(open(src, "rb").read()).hexdigest()[:16]
+
+
+def recorded_traffic(workload: str, n_units: int):
+    """DRAM bytes per launch of the streaming kernel from the committed ncu summary, scaled to this
+    launch by the elements processed; None if the kernel source changed since the capture."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    try:
+        rec = json.load(open(path))
+        if rec.get("source_sha256_16") != kernel_source_hash():
+            return None
+        return float(rec["dram_bytes_per_element"]) * n_units
+    except Exception:
+        return None
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.file = None
+
+    def start(self):
+        try:
+            self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=self.file, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        try:
+            self.proc.terminate()
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        try:
+            self.file.flush()
+            rows = [r.strip().split(", ") for r in open(self.file.name) if r.strip()]
+            os.unlink(self.file.name)
+        except Exception:
+            rows = []
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            if len(r) < 8:
+                continue
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, r[4:8]):
+                if val.strip().lower().startswith("active"):
+                    reasons.add(name)
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def visible_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+def host_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def oracle_steps_per_s(w: WL.Workload, steps: int, sample_workers: int, warmup: int = 0):
+    """Times the CPU oracle as it stands on a bounded sample: the first `sample_workers` rows of
+    the workload, full d and K (a majority-vote step among those workers).  Returns
+    (steps/s of the sample, seconds per step, description)."""
+    from oracle import mv_oracle as O
+    ws = WL.Workload(w.name, N=sample_workers, d=w.d, K=w.K, steps=w.steps, kind=w.kind, config_id=w.config_id,
+                     segments=w.segments, std_lo=w.std_lo, std_hi=w.std_hi, rho=w.rho, err0_std=w.err0_std,
+                     round_decimals=w.round_decimals)
+    err = WL.initial_err(ws).numpy()
+    times = []
+    for s in range(warmup + steps):
+        g = WL.gradients(ws, s).numpy()
+        t0 = time.perf_counter()
+        r = O.mv_sparse_step(g, err, ws.K)
+        dt = time.perf_counter() - t0
+        err = r["err"]
+        if s >= warmup:
+            times.append(dt)
+    per_step = float(np.mean(times))
+    # the oracle's cost is linear in the number of workers (each row is selected on its own)
+    full_step = per_step * (w.N / sample_workers)
+    desc = (f"{sample_workers} of {w.N} workers, full d={w.d} and K={w.K}, {steps} step(s); "
+            f"scaled by {w.N}/{sample_workers} to the whole step")
+    return 1.0 / full_step, full_step, desc
+
+
+def run_reference(args, w: WL.Workload):
+    """The reference arm: the CPU oracle on the host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    torch.set_num_threads(max(1, host_cores()))
+    sample_workers = min(w.N, 2 if w.d > 1_000_000 else w.N)
+    steps = max(1, min(args.steps, 3))
+    sps, sec, desc = oracle_steps_per_s(w, steps, sample_workers, warmup=min(args.warmup, 1))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": sps, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": workload_config(w),
+        "cpu_baseline": {"value": sps, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
+        "e2e": {"value": sps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(w: WL.Workload):
+    return {"workload": f"{w.name}: N={w.N} workers, d={w.d} fp32, K={w.K} ({w.note}), error feedback carried, "
+                        f"fresh gradients every step",
+            "N": w.N, "d": w.d, "K": w.K, "l2": "inputs larger than L2" if w.N * w.d * 4 > L2_BYTES else "L2-resident",
+            "parallelism": "replicas only"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2", choices=["c1", "c1_ties", "c2", "c3", "c4"])
+    ap.add_argument("--mode", default="auto", choices=["auto", "general"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    w = WL.resnet_like(args.workload)
+
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    from paper_2011_06495_b200 import binding as B
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- inputs resident in HBM before the timed region: a pool of gradient tensors, cycled
+    nbytes = w.N * w.d * 4
+    pool_n = max(2, min(args.steps + args.warmup, int(8e9 // nbytes), 8))
+    std = WL.std_vector(w, dev) if w.segments > 1 else None
+    pool = [WL.gradients(w, s, device=dev, std=std) for s in range(pool_n)]
+    err = WL.initial_err(w, device=dev)
+    out_idx = torch.empty(w.K, dtype=torch.int32, device=dev)
+    out_val = torch.empty(w.K, dtype=torch.float32, device=dev)
+    ctx = B.MvContext(w.N, w.d, w.K, device=dev, mode=B.MV_MODE_GENERAL if args.mode == "general" else B.MV_MODE_AUTO)
+
+    step_no = 0
+    for _ in range(args.warmup):
+        ctx.mv_sparse_step(pool[step_no % pool_n], err, out_idx, out_val)
+        step_no += 1
+    ctx.set_kernel_timing(True)
+    sampler = ClockSampler(visible_gpu_index(local_rank))
+    sampler.start()
+    barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(args.steps):
+        ctx.mv_sparse_step(pool[step_no % pool_n], err, out_idx, out_val)
+        step_no += 1
+    ev1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms_total = ev0.elapsed_time(ev1)
+    launches_per_step = ctx.last_launches()
+    k_ms, k_cnt = ctx.read_kernel_timing()
+    ctx.set_kernel_timing(False)
+    diag = ctx.read_diag(w.N)
+    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    value = world * args.steps / (ms_total * 1e-3)
+
+    # ---- end to end through the host entry point: gradients start in pinned host memory
+    e2e = None
+    if not args.no_e2e:
+        h_pool = [pool[i].cpu().pin_memory() for i in range(2)]
+        h_idx = torch.empty(w.K, dtype=torch.int32).pin_memory()
+        h_val = torch.empty(w.K, dtype=torch.float32).pin_memory()
+        d_grads = pool[-1]
+        e_steps = max(3, min(args.steps, 10))
+        for i in range(2):
+            ctx.mv_sparse_step_host(h_pool[i % 2], h_idx, h_val, d_grads, err, out_idx, out_val)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(e_steps):
+            ctx.mv_sparse_step_host(h_pool[i % 2], h_idx, h_val, d_grads, err, out_idx, out_val)
+        e1.record()
+        barrier()
+        te = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+        if dist is not None:
+            dist.all_reduce(te, op=dist.ReduceOp.MAX)
+        e2e = {"value": world * e_steps / (float(te.item()) * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": 8 * w.K, "steps": e_steps,
+               "note": "mv_sparse_step_host: gradients copied from pinned host memory every step, indices and "
+                       "values copied back; the residual stays on the device"}
+        del h_pool
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peak()
+    alg_bytes = 12.0 * w.N * w.d                      # read grads, read err, write acc: 12 B per element
+    k_ms_avg = k_ms / max(k_cnt, 1)
+    achieved = alg_bytes / (k_ms_avg * 1e-3) / 1e9 if k_cnt else None
+    traffic = recorded_traffic(w.name, w.N * w.d)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic", "config": workload_config(w),
+        "effective_gradient_gbs": w.N * w.d * 4 / (ms_step * 1e-3) / 1e9 * 1.0,
+        "step_roofline_frac": alg_bytes / (ms_step * 1e-3) / 1e9 / peak,
+        "roofline": {"bound": "hbm", "kernel": "k_acc_compact" if args.mode == "auto" else "k_row_hist<1,true>",
+                     "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                     "frac": (achieved / peak) if achieved else None, "traffic": traffic,
+                     "kernel_ms": k_ms_avg, "kernel_launches_timed": k_cnt, "algorithmic_bytes_per_launch": alg_bytes},
+        "clocks": clocks, "gpu_launches": launches_per_step * args.steps, "launches_per_step": launches_per_step,
+        "fallback_workers_last_step": int(diag[:, 2].sum()),
+        "candidates_over_K_last_step": float(diag[:, 0].double().mean() / w.K),
+    }
+    if e2e is not None:
+        line["e2e"] = e2e
+    if world == 1 and not args.no_cpu_baseline:
+        sample_workers = min(w.N, 2 if w.d > 1_000_000 else w.N)
+        sps, sec, desc = oracle_steps_per_s(w, 1, sample_workers)
+        line["cpu_baseline"] = {"value": sps, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc,
+                                "host_cores_available": host_cores()}
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,138 @@
+/*
+ * mv_sparse.h -- C ABI of the majority-vote sparse DSGD step for NVIDIA B200 (sm_100a).
+ *
+ * The library computes one iteration of "sparse SGD with majority voting"
+ * (Algorithm 1 of arXiv 2011.06495) for N workers held as the rows of one
+ * N x d array on a single GPU:
+ *
+ *   acc_n   = grads_n + err_n                    error feedback      (Algorithm 1, accumulate step)
+ *   M_n     = S_top(|acc_n|, K)                  per-worker top-K    (Eq. 6, definition of S_top)
+ *   votes   = sum_n M_n                          vote count          (Eq. 9, inner sum)
+ *   M       = S_top(votes, K)                    shared mask         (Eq. 9, outer S_top)
+ *   out_val = (1/N) sum_n acc_n  on supp(M)      shared-mask mean    (Eq. 8; the 1/N of the text)
+ *   err_n   = acc_n - M (x) acc_n                residual            (Algorithm 1, error update)
+ *
+ * Conventions (the paper leaves them open; they are part of this contract):
+ *   - |x| is ordered by key(x) = bits(x) & 0x7fffffff; ties in either S_top go to the
+ *     lowest coordinate index, so every result is unique.
+ *   - supports are ascending int32 index lists; bit masks are ceil(d/32) uint32 words
+ *     per row, bit b of word w standing for coordinate 32*w + b, unused tail bits zero.
+ *   - out_val is the mean: binary64 accumulation in worker order, one division by N,
+ *     one rounding to binary32.
+ *   - the residual is +0.0f on the mask and a bit copy of acc elsewhere.
+ *
+ * Memory: unless a parameter says "host", every pointer is a DEVICE pointer owned by
+ * the caller, row-major and contiguous (row pitch d), 16-byte aligned at its base.
+ * The library allocates and frees no device memory: scratch space is the caller's
+ * workspace of mv_workspace_bytes() bytes, reused by every call on the context.
+ * All work is enqueued on the stream given to mv_create; no call synchronises the
+ * host except mv_sparse_step_host and mv_read_diag.  A context is not thread-safe.
+ *
+ * Limits: 1 <= N <= 255, 1 <= d < 2^31 - 8192, 1 <= K <= d.
+ *
+ * Errors: every int-returning function returns MV_OK or a negative MV_ERR_* code;
+ * argument checks happen before anything is enqueued, so a failed call has no effect.
+ */
+#ifndef MV_SPARSE_H
+#define MV_SPARSE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  MV_OK = 0,
+  MV_ERR_INVALID_ARG = -1, /* null or misaligned pointer, N/d/K out of range, grads aliasing err */
+  MV_ERR_WORKSPACE = -2,   /* workspace smaller than mv_workspace_bytes(N, d, K) */
+  MV_ERR_CUDA = -3         /* the CUDA runtime refused a launch or a copy */
+};
+
+enum {
+  MV_MODE_AUTO = 0,    /* sampled threshold + single streaming pass, exact multi-pass select as fallback */
+  MV_MODE_GENERAL = 1  /* always the exact multi-pass radix select (no sampling) */
+};
+
+typedef struct mv_ctx mv_ctx;
+
+/* Bytes of device scratch needed for a problem of this size (host computation only).
+ * Returns 0 if N, d or K is out of range. */
+size_t mv_workspace_bytes(int N, int64_t d, int64_t K);
+
+/* Creates a context bound to `stream` (a cudaStream_t, may be NULL for the default
+ * stream) and to `workspace` (device memory, 256-byte aligned, owned by the caller,
+ * must outlive the context).  Touches no device memory. */
+int mv_create(mv_ctx** out, void* stream, void* workspace, size_t workspace_bytes);
+int mv_destroy(mv_ctx* ctx);
+
+/* Chooses how the per-worker threshold is found (MV_MODE_*).  Results are identical. */
+int mv_set_mode(mv_ctx* ctx, int mode);
+
+/* The whole step (Algorithm 1 from the accumulate line to the aggregate line).
+ *   grads   [N*d] in      the workers' model differences / gradients
+ *   err     [N*d] in/out  e_n on entry, the new residual e_n on exit
+ *   out_idx [K]   out     supp(M), ascending
+ *   out_val [K]   out     mean of acc over the workers on supp(M)
+ * Equivalent to mv_vote, mv_select, mv_aggregate in that order. */
+int mv_sparse_step(mv_ctx* ctx, const float* grads, float* err, int N, int64_t d, int64_t K,
+                   int32_t* out_idx, float* out_val);
+
+/* Voting phase, worker side and vote count (Algorithm 1 up to the vote sum; Eq. 6, Eq. 9 inner sum).
+ *   err         [N*d]           in/out  e_n on entry, acc_n on exit
+ *   worker_idx  [N*K]           out     supp(M_n) ascending, row n at n*K          (may be NULL)
+ *   worker_bits [N*ceil(d/32)]  out     M_n as bit masks                           (may be NULL)
+ *   votes       [d] uint8       out     votes per coordinate                       (may be NULL)
+ *   thresh      [N*3] uint32    out     per worker: K-th largest key T_n, number of keys above
+ *                                       it, number of keys equal to it             (may be NULL)
+ * Outputs passed as NULL are kept in the workspace. */
+int mv_vote(mv_ctx* ctx, const float* grads, float* err, int N, int64_t d, int64_t K,
+            int32_t* worker_idx, uint32_t* worker_bits, uint8_t* votes, uint32_t* thresh);
+
+/* Voting phase, server side (Eq. 9 outer S_top): the K most voted coordinates.
+ *   votes     [d] uint8        in   every value must be <= N
+ *   out_idx   [K]              out  ascending
+ *   mask_bits [ceil(d/32)]     out  the same set as a bit mask (may be NULL) */
+int mv_select(mv_ctx* ctx, const uint8_t* votes, int N, int64_t d, int64_t K,
+              int32_t* out_idx, uint32_t* mask_bits);
+
+/* Sparse communication phase (Algorithm 1 from the masked send to the aggregate; Eq. 8).
+ *   acc     [N*d] in/out  acc_n on entry, the residual on exit
+ *   idx     [K]   in      distinct coordinates in [0, d)
+ *   out_val [K]   out     mean over the workers of acc[:, idx[k]] */
+int mv_aggregate(mv_ctx* ctx, float* acc, int N, int64_t d, int64_t K, const int32_t* idx, float* out_val);
+
+/* The whole step for a caller whose gradients live in HOST memory (Algorithm 1, same lines
+ * as mv_sparse_step).  Copies h_grads (host, ideally pinned) into d_grads, runs the step on
+ * the device-resident residual d_err, copies the K indices and values back to the host
+ * buffers and waits for the stream before returning.
+ *   h_grads [N*d] host in; h_out_idx [K], h_out_val [K] host out;
+ *   d_grads [N*d], d_err [N*d], d_out_idx [K], d_out_val [K] device buffers of the caller. */
+int mv_sparse_step_host(mv_ctx* ctx, const float* h_grads, int N, int64_t d, int64_t K,
+                        int32_t* h_out_idx, float* h_out_val,
+                        float* d_grads, float* d_err, int32_t* d_out_idx, float* d_out_val);
+
+/* Diagnostics of the last mv_vote / mv_sparse_step on this context; waits for the stream.
+ *   per_worker [N*4] host uint32 out: candidates kept by the streaming pass, sampled
+ *   lower bound on the threshold key, 1 if the exact multi-pass select was used, 0 (spare). */
+int mv_read_diag(mv_ctx* ctx, int N, uint32_t* per_worker);
+
+/* Optional timing of the streaming pass (the kernel that reads grads and err and writes acc,
+ * i.e. the accumulate line of Algorithm 1 fused with the candidate filter of S_top): while
+ * enabled, every mv_vote / mv_sparse_step records a CUDA-event pair around that one kernel on
+ * the context's stream.  mv_read_kernel_timing waits for the stream, returns the summed
+ * duration in milliseconds and the number of launches it covers (at most the last 64), and
+ * restarts the count.  Enabling creates the events once; nothing is recorded while disabled. */
+int mv_set_kernel_timing(mv_ctx* ctx, int enable);
+int mv_read_kernel_timing(mv_ctx* ctx, float* total_ms, int* launches);
+
+/* Number of kernels the last call on this context enqueued. */
+int mv_last_launches(const mv_ctx* ctx);
+
+const char* mv_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MV_SPARSE_H */

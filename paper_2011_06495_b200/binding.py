@@ -1,0 +1,173 @@
+"""Thin Python binding of the C-ABI library (argument marshalling only).
+
+Every step of the method runs in the CUDA kernels of libmvsparse.so; this module only
+turns torch tensors into raw pointers, allocates the caller-owned workspace and checks
+status codes.  There is no CPU fallback: if the library has not been built, importing
+`load()` raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmvsparse.so")
+
+MV_OK = 0
+MV_ERR_INVALID_ARG = -1
+MV_ERR_WORKSPACE = -2
+MV_ERR_CUDA = -3
+MV_MODE_AUTO = 0
+MV_MODE_GENERAL = 1
+
+_lib = None
+
+
+class MvError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+def load() -> ctypes.CDLL:
+    """Loads libmvsparse.so (built in-tree by paper_2011_06495_b200.build); raises if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2011_06495_b200.build` "
+            "(there is no CPU fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    c_vp, c_i, c_i64, c_sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_size_t
+    lib.mv_workspace_bytes.restype = c_sz
+    lib.mv_workspace_bytes.argtypes = [c_i, c_i64, c_i64]
+    lib.mv_create.restype = c_i
+    lib.mv_create.argtypes = [ctypes.POINTER(c_vp), c_vp, c_vp, c_sz]
+    lib.mv_destroy.restype = c_i
+    lib.mv_destroy.argtypes = [c_vp]
+    lib.mv_set_mode.restype = c_i
+    lib.mv_set_mode.argtypes = [c_vp, c_i]
+    lib.mv_sparse_step.restype = c_i
+    lib.mv_sparse_step.argtypes = [c_vp, c_vp, c_vp, c_i, c_i64, c_i64, c_vp, c_vp]
+    lib.mv_vote.restype = c_i
+    lib.mv_vote.argtypes = [c_vp, c_vp, c_vp, c_i, c_i64, c_i64, c_vp, c_vp, c_vp, c_vp]
+    lib.mv_select.restype = c_i
+    lib.mv_select.argtypes = [c_vp, c_vp, c_i, c_i64, c_i64, c_vp, c_vp]
+    lib.mv_aggregate.restype = c_i
+    lib.mv_aggregate.argtypes = [c_vp, c_vp, c_i, c_i64, c_i64, c_vp, c_vp]
+    lib.mv_sparse_step_host.restype = c_i
+    lib.mv_sparse_step_host.argtypes = [c_vp, c_vp, c_i, c_i64, c_i64, c_vp, c_vp, c_vp, c_vp, c_vp, c_vp]
+    lib.mv_read_diag.restype = c_i
+    lib.mv_read_diag.argtypes = [c_vp, c_i, c_vp]
+    lib.mv_set_kernel_timing.restype = c_i
+    lib.mv_set_kernel_timing.argtypes = [c_vp, c_i]
+    lib.mv_read_kernel_timing.restype = c_i
+    lib.mv_read_kernel_timing.argtypes = [c_vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(c_i)]
+    lib.mv_last_launches.restype = c_i
+    lib.mv_last_launches.argtypes = [c_vp]
+    lib.mv_status_string.restype = ctypes.c_char_p
+    lib.mv_status_string.argtypes = [c_i]
+    _lib = lib
+    return lib
+
+
+def status_string(status: int) -> str:
+    return load().mv_status_string(int(status)).decode()
+
+
+def workspace_bytes(N: int, d: int, K: int) -> int:
+    return int(load().mv_workspace_bytes(int(N), int(d), int(K)))
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _check(status: int, where: str):
+    if status != MV_OK:
+        raise MvError(status, where)
+
+
+class MvContext:
+    """A context bound to the current CUDA stream and to a workspace tensor it keeps alive."""
+
+    def __init__(self, N: int, d: int, K: int, device="cuda", stream: Optional[torch.cuda.Stream] = None,
+                 mode: int = MV_MODE_AUTO):
+        self.lib = load()
+        self.N, self.d, self.K = int(N), int(d), int(K)
+        nbytes = workspace_bytes(N, d, K)
+        if nbytes == 0:
+            raise MvError(MV_ERR_INVALID_ARG, "mv_workspace_bytes")
+        self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=device)
+        self.stream = stream if stream is not None else torch.cuda.current_stream(self.workspace.device)
+        handle = ctypes.c_void_p()
+        _check(self.lib.mv_create(ctypes.byref(handle), ctypes.c_void_p(self.stream.cuda_stream),
+                                  _ptr(self.workspace), nbytes), "mv_create")
+        self.handle = handle
+        self.set_mode(mode)
+
+    def close(self):
+        if getattr(self, "handle", None):
+            self.lib.mv_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def set_mode(self, mode: int):
+        _check(self.lib.mv_set_mode(self.handle, int(mode)), "mv_set_mode")
+
+    # the calls below mirror include/mv_sparse.h one to one
+    def mv_sparse_step(self, grads, err, out_idx, out_val, K: Optional[int] = None):
+        N, d = grads.shape
+        _check(self.lib.mv_sparse_step(self.handle, _ptr(grads), _ptr(err), N, d, K or self.K,
+                                       _ptr(out_idx), _ptr(out_val)), "mv_sparse_step")
+
+    def mv_vote(self, grads, err, worker_idx=None, worker_bits=None, votes=None, thresh=None, K: Optional[int] = None):
+        N, d = grads.shape
+        _check(self.lib.mv_vote(self.handle, _ptr(grads), _ptr(err), N, d, K or self.K, _ptr(worker_idx),
+                                _ptr(worker_bits), _ptr(votes), _ptr(thresh)), "mv_vote")
+
+    def mv_select(self, votes, N: int, out_idx, mask_bits=None, K: Optional[int] = None):
+        _check(self.lib.mv_select(self.handle, _ptr(votes), N, votes.numel(), K or self.K, _ptr(out_idx),
+                                  _ptr(mask_bits)), "mv_select")
+
+    def mv_aggregate(self, acc, idx, out_val):
+        N, d = acc.shape
+        _check(self.lib.mv_aggregate(self.handle, _ptr(acc), N, d, idx.numel(), _ptr(idx), _ptr(out_val)),
+               "mv_aggregate")
+
+    def mv_sparse_step_host(self, h_grads, h_out_idx, h_out_val, d_grads, d_err, d_out_idx, d_out_val,
+                            K: Optional[int] = None):
+        N, d = h_grads.shape
+        _check(self.lib.mv_sparse_step_host(self.handle, _ptr(h_grads), N, d, K or self.K, _ptr(h_out_idx),
+                                            _ptr(h_out_val), _ptr(d_grads), _ptr(d_err), _ptr(d_out_idx),
+                                            _ptr(d_out_val)), "mv_sparse_step_host")
+
+    def read_diag(self, N: Optional[int] = None) -> torch.Tensor:
+        N = N or self.N
+        out = torch.zeros((N, 4), dtype=torch.int64)
+        buf = (ctypes.c_uint32 * (4 * N))()
+        _check(self.lib.mv_read_diag(self.handle, N, buf), "mv_read_diag")
+        out.copy_(torch.tensor(list(buf), dtype=torch.int64).view(N, 4))
+        return out
+
+    def set_kernel_timing(self, enable: bool):
+        _check(self.lib.mv_set_kernel_timing(self.handle, int(bool(enable))), "mv_set_kernel_timing")
+
+    def read_kernel_timing(self):
+        """(total milliseconds, launches covered) of the streaming pass since the last read."""
+        ms, cnt = ctypes.c_float(), ctypes.c_int()
+        _check(self.lib.mv_read_kernel_timing(self.handle, ctypes.byref(ms), ctypes.byref(cnt)),
+               "mv_read_kernel_timing")
+        return float(ms.value), int(cnt.value)
+
+    def last_launches(self) -> int:
+        return int(self.lib.mv_last_launches(self.handle))

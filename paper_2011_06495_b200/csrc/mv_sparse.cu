@@ -1,0 +1,1549 @@
+// Majority-vote sparse DSGD step (Algorithm 1 of arXiv 2011.06495) for sm_100a.
+//
+// N workers are the rows of one N x d array.  A step is a short sequence of kernels on
+// one stream, with no host synchronisation and no device allocation:
+//
+//   sample     k_sample_hist, k_sample_pick   a strided sample of |grads+err| per worker gives a
+//                                             lower bound tau_n on the K-th largest magnitude key
+//   stream     k_acc_compact                  the one pass over N x d: acc = err + grads written in
+//                                             place, elements with key >= tau_n compacted per chunk
+//   select     k_cand_hist<1..3>, k_cand_count  exact K-th key T_n by radix select on the candidates
+//   fallback   k_row_hist<1..3>, k_row_count, k_row_exact   exact radix select over the full rows for
+//                                             workers whose candidate count missed [K, cap]
+//   order      k_chunk_scan                   lowest-index tie quota and list offsets per chunk
+//   vote       k_build_votes                  per-worker bit masks and index lists, bit-sliced vote count
+//   mask       k_vote_hist, k_vote_scan, k_vote_write   counting select over vote values 0..N
+//   aggregate  k_gather                       mean on the shared mask, residual zeroed in place
+//
+// The magnitude order is the order of key(x) = bits(x) & 0x7fffffff; ties go to the lowest index.
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <math.h>
+#include <new>
+
+#include "../../include/mv_sparse.h"
+
+namespace {
+
+constexpr int CH = 4096;             // coordinates per chunk (row-relative, so chunks are mask-word aligned)
+constexpr int WPC = CH / 32;         // mask words per chunk
+constexpr int TPB = 256;             // threads per CTA of the chunk kernels
+constexpr int SB_BINS = 8192;        // sample histogram: top 13 bits of the 31-bit key
+constexpr int SB_SHIFT = 18;
+constexpr int H1_BINS = 2048;        // radix digits of the 31-bit key: 11 + 10 + 10 bits
+constexpr int H2_BINS = 1024;
+constexpr int H3_BINS = 1024;
+constexpr unsigned FULL = 0xffffffffu;
+
+struct P {
+  int N;
+  int nchunks;
+  uint32_t cap;           // candidate slots per worker
+  int force_general;
+  int64_t d;
+  int64_t K;
+  int64_t W;              // mask words per row = ceil(d/32)
+  uint32_t* samp_hist;    // [N][SB_BINS]
+  uint32_t* hist1;        // [N][H1_BINS]
+  uint32_t* hist2;        // [N][H2_BINS]
+  uint32_t* hist3;        // [N][H3_BINS]
+  uint32_t* cand_cnt;     // [N]
+  uint32_t* vote_hist;    // [256]
+  uint32_t* tau;          // [N]
+  uint32_t* wstate;       // [N][8]: b1, rem1, b2, rem2, T, cnt_gt, cnt_eq, need
+  uint32_t* thresh;       // [N][3]
+  uint32_t* vstate;       // [4]: v*, cnt_gt, cnt_eq, quota
+  uint2* cand;            // [N][cap] (key, index)
+  uint32_t* chunk_base;   // [N][nchunks]
+  uint32_t* chunk_cnt;
+  uint32_t* chunk_gt;
+  uint32_t* chunk_eq;
+  uint32_t* tie_base;
+  uint32_t* sel_base;
+  uint32_t* worker_bits;  // [N][W]
+  int32_t* worker_idx;    // [N][K]
+  uint8_t* votes;         // [d]
+  uint16_t* chunk_vh;     // [nchunks][N+1]
+  uint32_t* out_base;     // [nchunks]
+  uint32_t* tie_take;     // [nchunks]
+};
+
+__device__ __forceinline__ uint32_t fkey(float x) { return __float_as_uint(x) & 0x7fffffffu; }
+
+__device__ __forceinline__ uint32_t lanemask_lt() {
+  uint32_t m;
+  asm("mov.u32 %0, %%lanemask_lt;" : "=r"(m));
+  return m;
+}
+
+__device__ __forceinline__ bool worker_fast(const P& p, int n) {
+  if (p.force_general) return false;
+  const uint32_t c = p.cand_cnt[n];
+  return c >= (uint32_t)p.K && c <= p.cap;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Chunk geometry.  Chunk c of row n covers coordinates [c*CH, min(d, (c+1)*CH)).  Rows start at flat
+// element n*d, which need not be a multiple of 4, so the chunk is read as the 16-byte aligned
+// float4 "slots" that overlap it: slot s starts at flat element fa + 4*s, i.e. at coordinate
+// j0 - h + 4*s.  Slots fully inside the chunk use vector accesses, the (at most two) partial ones
+// scalar accesses restricted to the chunk's own elements.  A full chunk has 1024 slots when h == 0
+// and 1025 otherwise; slot 1024 is handled by thread 255 after all others ("extra").
+// ---------------------------------------------------------------------------------------------
+struct Geom {
+  size_t fa;
+  int j0, jend, h, nslots;
+};
+
+__device__ __forceinline__ Geom chunk_geom(int n, int c, int64_t d) {
+  Geom g;
+  const size_t r0 = (size_t)n * (size_t)d;
+  g.j0 = c * CH;
+  const int64_t je = (int64_t)g.j0 + CH;
+  g.jend = (int)(je < d ? je : d);
+  const size_t f0 = r0 + (size_t)g.j0;
+  g.fa = f0 & ~(size_t)3;
+  g.h = (int)(f0 - g.fa);
+  g.nslots = (g.h + (g.jend - g.j0) + 3) >> 2;
+  return g;
+}
+
+// Thread (warp w, lane l) owns slots w*128 + i*32 + l, i = 0..3: a warp covers 512 consecutive
+// coordinates, in index order (i, l, element).  ACC: acc = err + grads is computed and stored to err.
+template <bool ACC>
+__device__ __forceinline__ void load_keys(const Geom& g, const float* __restrict__ grads, float* __restrict__ err,
+                                          uint32_t (&key)[4][4], uint32_t (&vm)[4]) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float4 ev[4], gv[4];
+  int kind[4];
+#pragma unroll
+  for (int i = 0; i < 4; i++) {
+    const int s = warp * 128 + i * 32 + lane;
+    const int jf = g.j0 - g.h + 4 * s;
+    kind[i] = 0;
+    if (s < g.nslots) kind[i] = (jf >= g.j0 && jf + 3 < g.jend) ? 2 : 1;
+    if (kind[i] == 2) {
+      const size_t f = g.fa + 4 * (size_t)s;
+      ev[i] = __ldcs(reinterpret_cast<const float4*>(err + f));
+      if (ACC) gv[i] = __ldcs(reinterpret_cast<const float4*>(grads + f));
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 4; i++) {
+    const int s = warp * 128 + i * 32 + lane;
+    const int jf = g.j0 - g.h + 4 * s;
+    const size_t f = g.fa + 4 * (size_t)s;
+    vm[i] = 0;
+    key[i][0] = key[i][1] = key[i][2] = key[i][3] = 0;
+    if (kind[i] == 2) {
+      float4 a = ev[i];
+      if (ACC) {
+        a.x = __fadd_rn(ev[i].x, gv[i].x);
+        a.y = __fadd_rn(ev[i].y, gv[i].y);
+        a.z = __fadd_rn(ev[i].z, gv[i].z);
+        a.w = __fadd_rn(ev[i].w, gv[i].w);
+        __stcs(reinterpret_cast<float4*>(err + f), a);
+      }
+      key[i][0] = fkey(a.x);
+      key[i][1] = fkey(a.y);
+      key[i][2] = fkey(a.z);
+      key[i][3] = fkey(a.w);
+      vm[i] = 0xF;
+    } else if (kind[i] == 1) {
+#pragma unroll
+      for (int e = 0; e < 4; e++) {
+        const int j = jf + e;
+        if (j >= g.j0 && j < g.jend) {
+          float a = err[f + e];
+          if (ACC) {
+            a = __fadd_rn(a, grads[f + e]);
+            err[f + e] = a;
+          }
+          key[i][e] = fkey(a);
+          vm[i] |= 1u << e;
+        }
+      }
+    }
+  }
+}
+
+// Slot 1024 (exists only when the chunk is full and h != 0); call from one thread.
+template <bool ACC>
+__device__ __forceinline__ void load_extra(const Geom& g, const float* __restrict__ grads, float* __restrict__ err,
+                                           uint32_t (&key)[4], uint32_t& vm) {
+  vm = 0;
+  key[0] = key[1] = key[2] = key[3] = 0;
+  if (g.nslots > 1024) {
+    const int jf = g.j0 - g.h + 4096;
+    const size_t f = g.fa + 4096;
+#pragma unroll
+    for (int e = 0; e < 4; e++) {
+      const int j = jf + e;
+      if (j >= g.j0 && j < g.jend) {
+        float a = err[f + e];
+        if (ACC) {
+          a = __fadd_rn(a, grads[f + e]);
+          err[f + e] = a;
+        }
+        key[e] = fkey(a);
+        vm |= 1u << e;
+      }
+    }
+  }
+}
+
+// Ordered rank helper: m is this lane's 4-bit element mask for one iteration.  rank0 = number of
+// set bits in lower lanes (all four elements), total = set bits in the whole warp.
+__device__ __forceinline__ void iter_ranks(uint32_t m, uint32_t lt, uint32_t& rank0, uint32_t& total) {
+  const uint32_t b0 = __ballot_sync(FULL, m & 1u);
+  const uint32_t b1 = __ballot_sync(FULL, m & 2u);
+  const uint32_t b2 = __ballot_sync(FULL, m & 4u);
+  const uint32_t b3 = __ballot_sync(FULL, m & 8u);
+  rank0 = __popc(b0 & lt) + __popc(b1 & lt) + __popc(b2 & lt) + __popc(b3 & lt);
+  total = __popc(b0) + __popc(b1) + __popc(b2) + __popc(b3);
+}
+
+__device__ __forceinline__ uint32_t ge_mask(const uint32_t (&k)[4], uint32_t t) {
+  return (k[0] >= t ? 1u : 0u) | (k[1] >= t ? 2u : 0u) | (k[2] >= t ? 4u : 0u) | (k[3] >= t ? 8u : 0u);
+}
+__device__ __forceinline__ uint32_t gt_mask(const uint32_t (&k)[4], uint32_t t) {
+  return (k[0] > t ? 1u : 0u) | (k[1] > t ? 2u : 0u) | (k[2] > t ? 4u : 0u) | (k[3] > t ? 8u : 0u);
+}
+__device__ __forceinline__ uint32_t eq_mask(const uint32_t (&k)[4], uint32_t t) {
+  return (k[0] == t ? 1u : 0u) | (k[1] == t ? 2u : 0u) | (k[2] == t ? 4u : 0u) | (k[3] == t ? 8u : 0u);
+}
+
+// Finds the bin holding the rank-th largest element of a histogram (rank counted from the top,
+// 1-based): the largest bin b with sum(hist[b..]) >= rank, and rem = rank - sum(hist[b+1..]).
+// All TPB threads call it; if the histogram holds fewer than rank elements, bin = rem = 0.
+template <int NB>
+__device__ void block_pick(const uint32_t* __restrict__ hist, uint32_t rank, uint32_t& bin, uint32_t& rem) {
+  constexpr int PER = NB / TPB;
+  __shared__ uint32_t s_wsum[TPB / 32];
+  __shared__ uint32_t s_res[2];
+  const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+  uint32_t loc[PER];
+  uint32_t sum = 0;
+#pragma unroll
+  for (int k = 0; k < PER; k++) {
+    loc[k] = hist[t * PER + k];
+    sum += loc[k];
+  }
+  if (t == 0) {
+    s_res[0] = 0;
+    s_res[1] = 0;
+  }
+  uint32_t x = sum;  // inclusive suffix sum within the warp
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const uint32_t y = __shfl_down_sync(FULL, x, off);
+    if (lane + off < 32) x += y;
+  }
+  if (lane == 0) s_wsum[warp] = x;
+  __syncthreads();
+  uint32_t above = x - sum;
+  for (int w = warp + 1; w < TPB / 32; w++) above += s_wsum[w];
+  if (above < rank && rank <= above + sum) {
+    bool done = false;
+#pragma unroll
+    for (int k = PER - 1; k >= 0; k--) {
+      if (!done) {
+        if (above + loc[k] >= rank) {
+          s_res[0] = (uint32_t)(t * PER + k);
+          s_res[1] = rank - above;
+          done = true;
+        } else {
+          above += loc[k];
+        }
+      }
+    }
+  }
+  __syncthreads();
+  bin = s_res[0];
+  rem = s_res[1];
+  __syncthreads();
+}
+
+// Exclusive prefix sum over the threads of a CTA (NT = 256 or 1024); `total` gets the CTA sum.
+template <int NT>
+__device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* s_w /*NT/32 + 1*/, uint32_t& total) {
+  const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+  uint32_t x = v;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const uint32_t y = __shfl_up_sync(FULL, x, off);
+    if (lane >= off) x += y;
+  }
+  __syncthreads();  // protects s_w against a previous use
+  if (lane == 31) s_w[warp] = x;
+  __syncthreads();
+  uint32_t base = 0;
+  uint32_t tot = 0;
+  for (int w = 0; w < NT / 32; w++) {
+    const uint32_t sw = s_w[w];
+    if (w < warp) base += sw;
+    tot += sw;
+  }
+  total = tot;
+  return base + x - v;
+}
+
+// ---------------------------------------------------------------------------------------------
+// sample: histogram of the top 13 key bits over evenly spaced 32-element lines of each row
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(512) k_sample_hist(P p, const float* __restrict__ grads,
+                                                     const float* __restrict__ err, uint32_t U, uint32_t L, int all) {
+  __shared__ uint32_t sh[SB_BINS];
+  const int n = blockIdx.y;
+  for (int b = threadIdx.x; b < SB_BINS; b += 512) sh[b] = 0;
+  __syncthreads();
+  const size_t r0 = (size_t)n * (size_t)p.d;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (uint32_t u0 = (blockIdx.x * 16u + warp) * 4u; u0 < U; u0 += gridDim.x * 64u) {
+    float a[4];
+    bool ok[4];
+#pragma unroll
+    for (int q = 0; q < 4; q++) {
+      const uint32_t u = u0 + q;
+      ok[q] = false;
+      a[q] = 0.f;
+      if (u < U) {
+        const uint32_t line = all ? u : (uint32_t)(((uint64_t)u * L) / U);
+        const int64_t j = (int64_t)line * 32 + lane;
+        if (j < p.d) {
+          ok[q] = true;
+          a[q] = __fadd_rn(err[r0 + j], grads[r0 + j]);
+        }
+      }
+    }
+#pragma unroll
+    for (int q = 0; q < 4; q++)
+      if (ok[q]) atomicAdd(&sh[fkey(a[q]) >> SB_SHIFT], 1u);
+  }
+  __syncthreads();
+  uint32_t* gh = p.samp_hist + (size_t)n * SB_BINS;
+  for (int b = threadIdx.x; b < SB_BINS; b += 512) {
+    const uint32_t v = sh[b];
+    if (v) atomicAdd(&gh[b], v);
+  }
+}
+
+// tau_n = lower edge of the sample-histogram bin that holds the rank-th largest sampled key
+__global__ void __launch_bounds__(TPB) k_sample_pick(P p, uint32_t rank) {
+  const int n = blockIdx.x;
+  uint32_t bin, rem;
+  block_pick<SB_BINS>(p.samp_hist + (size_t)n * SB_BINS, rank, bin, rem);
+  if (threadIdx.x == 0) p.tau[n] = bin << SB_SHIFT;
+}
+
+// ---------------------------------------------------------------------------------------------
+// stream: acc = err + grads in place; elements with key >= tau_n appended, in index order, to the
+// chunk's own run of the worker's candidate buffer (one global atomic per chunk that has any)
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(TPB) k_acc_compact(P p, const float* __restrict__ grads, float* __restrict__ err) {
+  __shared__ uint32_t s_w[9];
+  __shared__ uint32_t s_base, s_total;
+  const int n = blockIdx.y, c = blockIdx.x;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const Geom g = chunk_geom(n, c, p.d);
+  const uint32_t tau = p.tau[n];
+  uint32_t key[4][4], vm[4], cm[4];
+  load_keys<true>(g, grads, err, key, vm);
+  uint32_t xkey[4], xcm = 0;
+  if (threadIdx.x == TPB - 1) {
+    uint32_t xvm;
+    load_extra<true>(g, grads, err, xkey, xvm);
+    xcm = xvm & ge_mask(xkey, tau);
+  }
+  uint32_t wsum = 0;
+#pragma unroll
+  for (int i = 0; i < 4; i++) {
+    cm[i] = vm[i] & ge_mask(key[i], tau);
+    wsum += __popc(cm[i]);
+  }
+  wsum = __reduce_add_sync(FULL, wsum);
+  if (lane == 0) s_w[warp] = wsum;
+  if (threadIdx.x == TPB - 1) s_w[8] = __popc(xcm);
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    uint32_t total = 0;
+    for (int w = 0; w < 9; w++) total += s_w[w];
+    uint32_t base = 0;
+    if (total) base = atomicAdd(&p.cand_cnt[n], total);
+    p.chunk_base[(size_t)n * p.nchunks + c] = base;
+    p.chunk_cnt[(size_t)n * p.nchunks + c] = total;
+    s_base = base;
+    s_total = total;
+  }
+  __syncthreads();
+  if (s_total == 0) return;
+  uint32_t off = s_base;
+  for (int w = 0; w < warp; w++) off += s_w[w];
+  uint2* out = p.cand + (size_t)n * p.cap;
+  const uint32_t lt = lanemask_lt();
+#pragma unroll
+  for (int i = 0; i < 4; i++) {
+    uint32_t rank0, tot;
+    iter_ranks(cm[i], lt, rank0, tot);
+    if (cm[i]) {
+      const int jf = g.j0 - g.h + 4 * (warp * 128 + i * 32 + lane);
+#pragma unroll
+      for (int e = 0; e < 4; e++) {
+        if (cm[i] & (1u << e)) {
+          const uint32_t pos = off + rank0 + __popc(cm[i] & ((1u << e) - 1u));
+          if (pos < p.cap) out[pos] = make_uint2(key[i][e], (uint32_t)(jf + e));
+        }
+      }
+    }
+    off += tot;
+  }
+  if (threadIdx.x == TPB - 1 && xcm) {
+    uint32_t xoff = s_base;
+    for (int w = 0; w < 8; w++) xoff += s_w[w];
+    const int jf = g.j0 - g.h + 4096;
+#pragma unroll
+    for (int e = 0; e < 4; e++) {
+      if (xcm & (1u << e)) {
+        const uint32_t pos = xoff + __popc(xcm & ((1u << e) - 1u));
+        if (pos < p.cap) out[pos] = make_uint2(xkey[e], (uint32_t)(jf + e));
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// exact K-th key by radix select (11 + 10 + 10 bits).  Pass q first resolves digit q-1 from the
+// previous pass's histogram (every CTA repeats that small scan; CTA 0 records it), then counts
+// digit q among the elements whose higher digits match.
+// ---------------------------------------------------------------------------------------------
+template <int PASS>
+__device__ __forceinline__ uint32_t resolve_prefix(const P& p, int n) {
+  uint32_t* ws = p.wstate + (size_t)n * 8;
+  if (PASS == 2) {
+    uint32_t b1, rem1;
+    block_pick<H1_BINS>(p.hist1 + (size_t)n * H1_BINS, (uint32_t)p.K, b1, rem1);
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+      ws[0] = b1;
+      ws[1] = rem1;
+    }
+    return b1;
+  }
+  if (PASS == 3) {
+    const uint32_t b1 = ws[0], rem1 = ws[1];
+    uint32_t b2, rem2;
+    block_pick<H2_BINS>(p.hist2 + (size_t)n * H2_BINS, rem1, b2, rem2);
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+      ws[2] = b2;
+      ws[3] = rem2;
+    }
+    return (b1 << 10) | b2;
+  }
+  return 0;
+}
+
+// Last digit: T_n, cnt_gt, cnt_eq and the tie quota (need) -- returns T.
+__device__ __forceinline__ uint32_t resolve_threshold(const P& p, int n) {
+  uint32_t* ws = p.wstate + (size_t)n * 8;
+  const uint32_t b1 = ws[0], b2 = ws[2], rem2 = ws[3];
+  uint32_t b3, rem3;
+  block_pick<H3_BINS>(p.hist3 + (size_t)n * H3_BINS, rem2, b3, rem3);
+  const uint32_t T = (b1 << 20) | (b2 << 10) | b3;
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    const uint32_t cnt_eq = p.hist3[(size_t)n * H3_BINS + b3];
+    const uint32_t cnt_gt = (uint32_t)p.K - rem3;
+    ws[4] = T;
+    ws[5] = cnt_gt;
+    ws[6] = cnt_eq;
+    ws[7] = rem3;
+    p.thresh[n * 3 + 0] = T;
+    p.thresh[n * 3 + 1] = cnt_gt;
+    p.thresh[n * 3 + 2] = cnt_eq;
+  }
+  return T;
+}
+
+template <int PASS>
+__device__ __forceinline__ void hist_add(uint32_t* sh, uint32_t key, uint32_t prefix) {
+  if (PASS == 1) {
+    atomicAdd(&sh[key >> 20], 1u);
+  } else if (PASS == 2) {
+    if ((key >> 20) == prefix) atomicAdd(&sh[(key >> 10) & 1023u], 1u);
+  } else {
+    if ((key >> 10) == prefix) atomicAdd(&sh[key & 1023u], 1u);
+  }
+}
+
+template <int PASS>
+__device__ __forceinline__ uint32_t* hist_of(const P& p, int n) {
+  if (PASS == 1) return p.hist1 + (size_t)n * H1_BINS;
+  if (PASS == 2) return p.hist2 + (size_t)n * H2_BINS;
+  return p.hist3 + (size_t)n * H3_BINS;
+}
+
+template <int PASS>
+__global__ void __launch_bounds__(TPB) k_cand_hist(P p) {
+  constexpr int NB = PASS == 1 ? H1_BINS : H2_BINS;
+  __shared__ uint32_t sh[NB];
+  const int n = blockIdx.y;
+  if (!worker_fast(p, n)) return;
+  const uint32_t prefix = resolve_prefix<PASS>(p, n);
+  for (int b = threadIdx.x; b < NB; b += TPB) sh[b] = 0;
+  __syncthreads();
+  const uint32_t cnt = p.cand_cnt[n];
+  const uint2* cd = p.cand + (size_t)n * p.cap;
+  for (uint32_t i = blockIdx.x * TPB + threadIdx.x; i < cnt; i += gridDim.x * TPB) hist_add<PASS>(sh, cd[i].x, prefix);
+  __syncthreads();
+  uint32_t* gh = hist_of<PASS>(p, n);
+  for (int b = threadIdx.x; b < NB; b += TPB) {
+    const uint32_t v = sh[b];
+    if (v) atomicAdd(&gh[b], v);
+  }
+}
+
+// per chunk: how many candidates lie above / at the threshold
+__global__ void __launch_bounds__(TPB) k_cand_count(P p) {
+  const int n = blockIdx.y;
+  if (!worker_fast(p, n)) return;
+  const uint32_t T = resolve_threshold(p, n);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint2* cd = p.cand + (size_t)n * p.cap;
+  for (int c = blockIdx.x * (TPB / 32) + warp; c < p.nchunks; c += gridDim.x * (TPB / 32)) {
+    const size_t ci = (size_t)n * p.nchunks + c;
+    const uint32_t cnt = p.chunk_cnt[ci], base = p.chunk_base[ci];
+    uint32_t gt = 0, eq = 0;
+    for (uint32_t i = lane; i < cnt; i += 32) {
+      const uint32_t k = cd[base + i].x;
+      gt += k > T;
+      eq += k == T;
+    }
+    gt = __reduce_add_sync(FULL, gt);
+    eq = __reduce_add_sync(FULL, eq);
+    if (lane == 0) {
+      p.chunk_gt[ci] = gt;
+      p.chunk_eq[ci] = eq;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// fallback / general path: the same radix select over the full rows of the workers that are not
+// "fast".  PASS 1 with ACC fuses the error-feedback add (used when sampling is switched off).
+// ---------------------------------------------------------------------------------------------
+template <int PASS, bool ACC>
+__global__ void __launch_bounds__(TPB) k_row_hist(P p, const float* __restrict__ grads, float* __restrict__ err) {
+  constexpr int NB = PASS == 1 ? H1_BINS : H2_BINS;
+  __shared__ uint32_t sh[NB];
+  const int n = blockIdx.y;
+  if (worker_fast(p, n)) return;
+  const uint32_t prefix = resolve_prefix<PASS>(p, n);
+  for (int b = threadIdx.x; b < NB; b += TPB) sh[b] = 0;
+  __syncthreads();
+  for (int c = blockIdx.x; c < p.nchunks; c += gridDim.x) {
+    const Geom g = chunk_geom(n, c, p.d);
+    uint32_t key[4][4], vm[4];
+    load_keys<ACC>(g, grads, err, key, vm);
+#pragma unroll
+    for (int i = 0; i < 4; i++)
+#pragma unroll
+      for (int e = 0; e < 4; e++)
+        if (vm[i] & (1u << e)) hist_add<PASS>(sh, key[i][e], prefix);
+    if (threadIdx.x == TPB - 1) {
+      uint32_t xkey[4], xvm;
+      load_extra<ACC>(g, grads, err, xkey, xvm);
+#pragma unroll
+      for (int e = 0; e < 4; e++)
+        if (xvm & (1u << e)) hist_add<PASS>(sh, xkey[e], prefix);
+    }
+  }
+  __syncthreads();
+  uint32_t* gh = hist_of<PASS>(p, n);
+  for (int b = threadIdx.x; b < NB; b += TPB) {
+    const uint32_t v = sh[b];
+    if (v) atomicAdd(&gh[b], v);
+  }
+}
+
+__global__ void __launch_bounds__(TPB) k_row_count(P p, float* __restrict__ err) {
+  __shared__ uint32_t s_g[TPB / 32], s_e[TPB / 32];
+  const int n = blockIdx.y;
+  if (worker_fast(p, n)) return;
+  const uint32_t T = resolve_threshold(p, n);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int c = blockIdx.x; c < p.nchunks; c += gridDim.x) {
+    const Geom g = chunk_geom(n, c, p.d);
+    uint32_t key[4][4], vm[4];
+    load_keys<false>(g, nullptr, err, key, vm);
+    uint32_t gt = 0, eq = 0;
+#pragma unroll
+    for (int i = 0; i < 4; i++) {
+      gt += __popc(vm[i] & gt_mask(key[i], T));
+      eq += __popc(vm[i] & eq_mask(key[i], T));
+    }
+    if (threadIdx.x == TPB - 1) {
+      uint32_t xkey[4], xvm;
+      load_extra<false>(g, nullptr, err, xkey, xvm);
+      gt += __popc(xvm & gt_mask(xkey, T));
+      eq += __popc(xvm & eq_mask(xkey, T));
+    }
+    gt = __reduce_add_sync(FULL, gt);
+    eq = __reduce_add_sync(FULL, eq);
+    __syncthreads();
+    if (lane == 0) {
+      s_g[warp] = gt;
+      s_e[warp] = eq;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      uint32_t tg = 0, te = 0;
+      for (int w = 0; w < TPB / 32; w++) {
+        tg += s_g[w];
+        te += s_e[w];
+      }
+      p.chunk_gt[(size_t)n * p.nchunks + c] = tg;
+      p.chunk_eq[(size_t)n * p.nchunks + c] = te;
+    }
+  }
+}
+
+// exact compaction: writes precisely the selected elements of each chunk, in index order, at the
+// chunk's list offset (so the candidate buffer of such a worker holds its K picks, sorted)
+__global__ void __launch_bounds__(TPB) k_row_exact(P p, float* __restrict__ err) {
+  __shared__ uint32_t s_we[9], s_ws[9];
+  const int n = blockIdx.y;
+  if (worker_fast(p, n)) return;
+  const uint32_t* ws = p.wstate + (size_t)n * 8;
+  const uint32_t T = ws[4], need = ws[7];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t lt = lanemask_lt();
+  uint2* out = p.cand + (size_t)n * p.cap;
+  for (int c = blockIdx.x; c < p.nchunks; c += gridDim.x) {
+    const size_t ci = (size_t)n * p.nchunks + c;
+    const Geom g = chunk_geom(n, c, p.d);
+    uint32_t key[4][4], vm[4], em[4], sm[4];
+    load_keys<false>(g, nullptr, err, key, vm);
+    uint32_t xkey[4], xvm = 0, xem = 0, xsm = 0;
+    if (threadIdx.x == TPB - 1) {
+      load_extra<false>(g, nullptr, err, xkey, xvm);
+      xem = xvm & eq_mask(xkey, T);
+    }
+    uint32_t weq = 0;
+#pragma unroll
+    for (int i = 0; i < 4; i++) {
+      em[i] = vm[i] & eq_mask(key[i], T);
+      weq += __popc(em[i]);
+    }
+    weq = __reduce_add_sync(FULL, weq);
+    __syncthreads();  // previous chunk's readers of s_we / s_ws are done
+    if (lane == 0) s_we[warp] = weq;
+    if (threadIdx.x == TPB - 1) s_we[8] = __popc(xem);
+    __syncthreads();
+    const uint32_t tb = p.tie_base[ci];
+    uint32_t eoff = tb;
+    for (int w = 0; w < warp; w++) eoff += s_we[w];
+    uint32_t wsel = 0;
+#pragma unroll
+    for (int i = 0; i < 4; i++) {
+      uint32_t rank0, tot;
+      iter_ranks(em[i], lt, rank0, tot);
+      uint32_t take = 0;
+#pragma unroll
+      for (int e = 0; e < 4; e++) {
+        if (em[i] & (1u << e)) {
+          const uint32_t r = eoff + rank0 + __popc(em[i] & ((1u << e) - 1u));
+          if (r < need) take |= 1u << e;
+        }
+      }
+      sm[i] = (vm[i] & gt_mask(key[i], T)) | take;
+      wsel += __popc(sm[i]);
+      eoff += tot;
+    }
+    if (threadIdx.x == TPB - 1) {
+      uint32_t xoff = tb;
+      for (int w = 0; w < 8; w++) xoff += s_we[w];
+      uint32_t take = 0;
+#pragma unroll
+      for (int e = 0; e < 4; e++) {
+        if (xem & (1u << e)) {
+          const uint32_t r = xoff + __popc(xem & ((1u << e) - 1u));
+          if (r < need) take |= 1u << e;
+        }
+      }
+      xsm = (xvm & gt_mask(xkey, T)) | take;
+    }
+    wsel = __reduce_add_sync(FULL, wsel);
+    if (lane == 0) s_ws[warp] = wsel;
+    if (threadIdx.x == TPB - 1) s_ws[8] = __popc(xsm);
+    __syncthreads();
+    const uint32_t sb = p.sel_base[ci];
+    uint32_t soff = sb;
+    for (int w = 0; w < warp; w++) soff += s_ws[w];
+#pragma unroll
+    for (int i = 0; i < 4; i++) {
+      uint32_t rank0, tot;
+      iter_ranks(sm[i], lt, rank0, tot);
+      if (sm[i]) {
+        const int jf = g.j0 - g.h + 4 * (warp * 128 + i * 32 + lane);
+#pragma unroll
+        for (int e = 0; e < 4; e++) {
+          if (sm[i] & (1u << e)) {
+            const uint32_t pos = soff + rank0 + __popc(sm[i] & ((1u << e) - 1u));
+            if (pos < p.cap) out[pos] = make_uint2(key[i][e], (uint32_t)(jf + e));
+          }
+        }
+      }
+      soff += tot;
+    }
+    if (threadIdx.x == TPB - 1 && xsm) {
+      uint32_t xoff = sb;
+      for (int w = 0; w < 8; w++) xoff += s_ws[w];
+      const int jf = g.j0 - g.h + 4096;
+#pragma unroll
+      for (int e = 0; e < 4; e++) {
+        if (xsm & (1u << e)) {
+          const uint32_t pos = xoff + __popc(xsm & ((1u << e) - 1u));
+          if (pos < p.cap) out[pos] = make_uint2(xkey[e], (uint32_t)(jf + e));
+        }
+      }
+    }
+    if (threadIdx.x == 0) {
+      uint32_t tot = 0;
+      for (int w = 0; w < 9; w++) tot += s_ws[w];
+      p.chunk_base[ci] = sb;
+      p.chunk_cnt[ci] = tot;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// order: per worker, running count of threshold ties before each chunk (tie_base) and of selected
+// elements before each chunk (sel_base), given the quota `need` of ties to keep, lowest index first
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024) k_chunk_scan(P p) {
+  __shared__ uint32_t s_w[33];
+  const int n = blockIdx.x;
+  const uint32_t need = p.wstate[(size_t)n * 8 + 7];
+  const int per = (p.nchunks + 1023) / 1024;
+  const int c0 = min(p.nchunks, (int)threadIdx.x * per), c1 = min(p.nchunks, c0 + per);
+  const size_t rb = (size_t)n * p.nchunks;
+  uint32_t esum = 0;
+  for (int c = c0; c < c1; c++) esum += p.chunk_eq[rb + c];
+  uint32_t tot;
+  const uint32_t epre = block_excl_scan<1024>(esum, s_w, tot);
+  uint32_t run = epre, ssum = 0;
+  for (int c = c0; c < c1; c++) {
+    const uint32_t eq = p.chunk_eq[rb + c];
+    const uint32_t take = run >= need ? 0u : min(eq, need - run);
+    p.tie_base[rb + c] = run;
+    run += eq;
+    ssum += p.chunk_gt[rb + c] + take;
+  }
+  const uint32_t spre = block_excl_scan<1024>(ssum, s_w, tot);
+  run = epre;
+  uint32_t srun = spre;
+  for (int c = c0; c < c1; c++) {
+    const uint32_t eq = p.chunk_eq[rb + c];
+    const uint32_t take = run >= need ? 0u : min(eq, need - run);
+    p.sel_base[rb + c] = srun;
+    run += eq;
+    srun += p.chunk_gt[rb + c] + take;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// vote: one CTA per chunk, all workers.  The selected candidates set bits in shared-memory masks
+// (32 workers at a time); the masks are written out, turned into ascending index lists, and added
+// up bit-sliced (8 counter planes per 32-coordinate word) into the vote count.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(TPB) k_build_votes(P p) {
+  __shared__ uint32_t masks[32][WPC];
+  __shared__ uint32_t s_cnt[32], s_base[32], s_T[32], s_need[32], s_tb[32], s_sb[32], s_partial[32], s_pref[33];
+  __shared__ uint32_t s_vh[256];
+  const int c = blockIdx.x;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t lt = lanemask_lt();
+  uint32_t planes[8];
+#pragma unroll
+  for (int q = 0; q < 8; q++) planes[q] = 0;
+  s_vh[tid] = 0;
+  for (int g0 = 0; g0 < p.N; g0 += 32) {
+    const int G = min(32, p.N - g0);
+    __syncthreads();  // previous group's readers are done
+    for (int i = tid; i < G * WPC; i += TPB) masks[i / WPC][i % WPC] = 0;
+    if (tid < G) {
+      const int n = g0 + tid;
+      const size_t ci = (size_t)n * p.nchunks + c;
+      const uint32_t* ws = p.wstate + (size_t)n * 8;
+      s_cnt[tid] = p.chunk_cnt[ci];
+      s_base[tid] = p.chunk_base[ci];
+      s_T[tid] = ws[4];
+      s_need[tid] = ws[7];
+      s_partial[tid] = ws[7] < ws[6] ? 1u : 0u;  // not every threshold tie is kept
+      s_tb[tid] = p.tie_base[ci];
+      s_sb[tid] = p.sel_base[ci];
+    }
+    __syncthreads();
+    if (tid == 0) {
+      uint32_t a = 0;
+      for (int g = 0; g < G; g++) {
+        s_pref[g] = a;
+        a += s_cnt[g];
+      }
+      s_pref[G] = a;
+    }
+    __syncthreads();
+    const uint32_t total = s_pref[G];
+    // everything above the threshold, plus the ties of workers that keep all of them
+    for (uint32_t i = tid; i < total; i += TPB) {
+      int lo = 0, hi = G - 1;  // last g with s_pref[g] <= i
+      while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (s_pref[mid] <= i) lo = mid; else hi = mid - 1;
+      }
+      const int gi = lo;
+      const uint2 kv = p.cand[(size_t)(g0 + gi) * p.cap + s_base[gi] + (i - s_pref[gi])];
+      const uint32_t T = s_T[gi];
+      if (kv.x > T || (kv.x == T && !s_partial[gi])) {
+        const uint32_t rel = kv.y - (uint32_t)(c * CH);
+        if (rel < (uint32_t)CH) atomicOr(&masks[gi][rel >> 5], 1u << (rel & 31u));
+      }
+    }
+    // workers that keep only part of their ties: ordered walk, lowest index first
+    for (int gi = warp; gi < G; gi += TPB / 32) {
+      if (!s_partial[gi] || s_cnt[gi] == 0) continue;
+      const uint2* cd = p.cand + (size_t)(g0 + gi) * p.cap + s_base[gi];
+      const uint32_t T = s_T[gi], need = s_need[gi], cnt = s_cnt[gi];
+      uint32_t run = s_tb[gi];
+      for (uint32_t i0 = 0; i0 < cnt && run < need; i0 += 32) {
+        const uint32_t i = i0 + lane;
+        uint2 kv = make_uint2(0, 0);
+        bool eq = false;
+        if (i < cnt) {
+          kv = cd[i];
+          eq = kv.x == T;
+        }
+        const uint32_t eb = __ballot_sync(FULL, eq);
+        if (eq && run + __popc(eb & lt) < need) {
+          const uint32_t rel = kv.y - (uint32_t)(c * CH);
+          if (rel < (uint32_t)CH) atomicOr(&masks[gi][rel >> 5], 1u << (rel & 31u));
+        }
+        run += __popc(eb);
+      }
+    }
+    __syncthreads();
+    // masks out (coalesced)
+    for (int i = tid; i < G * WPC; i += TPB) {
+      const int gi = i / WPC, w = i % WPC;
+      const int64_t wi = (int64_t)c * WPC + w;
+      if (wi < p.W) p.worker_bits[(size_t)(g0 + gi) * p.W + wi] = masks[gi][w];
+    }
+    // ascending index lists: a warp per worker, four mask words per lane
+    for (int gi = warp; gi < G; gi += TPB / 32) {
+      uint32_t m[4];
+      uint32_t pc = 0;
+#pragma unroll
+      for (int q = 0; q < 4; q++) {
+        m[q] = masks[gi][lane * 4 + q];
+        pc += __popc(m[q]);
+      }
+      uint32_t x = pc;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t y = __shfl_up_sync(FULL, x, off);
+        if (lane >= off) x += y;
+      }
+      uint32_t pos = s_sb[gi] + x - pc;
+      int32_t* lst = p.worker_idx + (size_t)(g0 + gi) * p.K;
+#pragma unroll
+      for (int q = 0; q < 4; q++) {
+        uint32_t mm = m[q];
+        while (mm) {
+          const int b = __ffs(mm) - 1;
+          mm &= mm - 1;
+          if (pos < (uint32_t)p.K) lst[pos] = c * CH + (lane * 4 + q) * 32 + b;
+          pos++;
+        }
+      }
+    }
+    // vote planes: thread w adds word w of every worker into its bit-sliced counters
+    if (tid < WPC) {
+      for (int gi = 0; gi < G; gi++) {
+        uint32_t carry = masks[gi][tid];
+#pragma unroll
+        for (int q = 0; q < 8; q++) {
+          const uint32_t t2 = planes[q] & carry;
+          planes[q] ^= carry;
+          carry = t2;
+        }
+      }
+    }
+  }
+  // expand the planes into 32 vote bytes per thread
+  const int64_t jb = (int64_t)c * CH + (int64_t)tid * 32;
+  if (tid < WPC && jb < p.d) {
+    uint32_t wv[8];
+#pragma unroll
+    for (int q = 0; q < 8; q++) wv[q] = 0;
+#pragma unroll
+    for (int b = 0; b < 32; b++) {
+      uint32_t v = 0;
+#pragma unroll
+      for (int q = 0; q < 8; q++) v |= ((planes[q] >> b) & 1u) << q;
+      wv[b >> 2] |= v << (8 * (b & 3));
+      if (v && jb + b < p.d) atomicAdd(&s_vh[v], 1u);
+    }
+    if (jb + 32 <= p.d) {
+      uint4* dst = reinterpret_cast<uint4*>(p.votes + jb);
+      dst[0] = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+      dst[1] = make_uint4(wv[4], wv[5], wv[6], wv[7]);
+    } else {
+      for (int b = 0; b < 32 && jb + b < p.d; b++) p.votes[jb + b] = (uint8_t)((wv[b >> 2] >> (8 * (b & 3))) & 0xffu);
+    }
+  }
+  __syncthreads();
+  if (tid == 0) {
+    const int64_t rem = p.d - (int64_t)c * CH;
+    uint32_t valid = (uint32_t)(rem < CH ? rem : CH), nz = 0;
+    for (int v = 1; v < 256; v++) nz += s_vh[v];
+    s_vh[0] = valid - nz;
+  }
+  __syncthreads();
+  if (tid <= p.N) {
+    const uint32_t v = s_vh[tid];
+    p.chunk_vh[(size_t)c * (p.N + 1) + tid] = (uint16_t)v;
+    if (v) atomicAdd(&p.vote_hist[tid], v);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// mask: counting select over the vote values 0..N
+// ---------------------------------------------------------------------------------------------
+// per-chunk and global histogram of vote values, from a vote vector (stand-alone mv_select)
+__global__ void __launch_bounds__(TPB) k_vote_hist(P p, const uint8_t* __restrict__ votes) {
+  __shared__ uint32_t s_vh[256];
+  const int c = blockIdx.x, tid = threadIdx.x;
+  s_vh[tid] = 0;
+  __syncthreads();
+  const int64_t jb = (int64_t)c * CH + (int64_t)tid * 16;
+  if (jb < p.d) {
+    if (jb + 16 <= p.d) {
+      const uint4 q = *reinterpret_cast<const uint4*>(votes + jb);
+      const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+      for (int b = 0; b < 16; b++) {
+        const uint32_t v = (w[b >> 2] >> (8 * (b & 3))) & 0xffu;
+        if (v) atomicAdd(&s_vh[v], 1u);
+      }
+    } else {
+      for (int b = 0; b < 16 && jb + b < p.d; b++) {
+        const uint32_t v = votes[jb + b];
+        if (v) atomicAdd(&s_vh[v], 1u);
+      }
+    }
+  }
+  __syncthreads();
+  if (tid == 0) {
+    const int64_t rem = p.d - (int64_t)c * CH;
+    uint32_t valid = (uint32_t)(rem < CH ? rem : CH), nz = 0;
+    for (int v = 1; v < 256; v++) nz += s_vh[v];
+    s_vh[0] = valid - nz;
+  }
+  __syncthreads();
+  if (tid <= p.N) {
+    const uint32_t v = s_vh[tid];
+    p.chunk_vh[(size_t)c * (p.N + 1) + tid] = (uint16_t)v;
+    if (v) atomicAdd(&p.vote_hist[tid], v);
+  }
+}
+
+// v* = the vote value of the K-th most voted coordinate; then per chunk the output offset and the
+// number of v*-ties it may keep (lowest index first)
+__global__ void __launch_bounds__(1024) k_vote_scan(P p) {
+  __shared__ uint32_t s_w[33];
+  __shared__ uint32_t s_v[4];
+  if (threadIdx.x == 0) {
+    uint32_t acc = 0, vstar = 0, cgt = 0, ceq = 0;
+    for (int v = p.N; v >= 0; v--) {
+      const uint32_t h = p.vote_hist[v];
+      if (acc + h >= (uint32_t)p.K) {
+        vstar = (uint32_t)v;
+        cgt = acc;
+        ceq = h;
+        break;
+      }
+      acc += h;
+    }
+    s_v[0] = vstar;
+    s_v[1] = cgt;
+    s_v[2] = ceq;
+    s_v[3] = (uint32_t)p.K - cgt;
+    p.vstate[0] = vstar;
+    p.vstate[1] = cgt;
+    p.vstate[2] = ceq;
+    p.vstate[3] = (uint32_t)p.K - cgt;
+  }
+  __syncthreads();
+  const uint32_t vstar = s_v[0], quota = s_v[3];
+  const int stride = p.N + 1;
+  const int per = (p.nchunks + 1023) / 1024;
+  const int c0 = min(p.nchunks, (int)threadIdx.x * per), c1 = min(p.nchunks, c0 + per);
+  uint32_t esum = 0;
+  for (int c = c0; c < c1; c++) esum += p.chunk_vh[(size_t)c * stride + vstar];
+  uint32_t tot;
+  const uint32_t epre = block_excl_scan<1024>(esum, s_w, tot);
+  uint32_t run = epre, ssum = 0;
+  for (int c = c0; c < c1; c++) {
+    const uint16_t* h = p.chunk_vh + (size_t)c * stride;
+    const uint32_t eq = h[vstar];
+    const uint32_t take = run >= quota ? 0u : min(eq, quota - run);
+    uint32_t gt = 0;
+    for (int v = (int)vstar + 1; v <= p.N; v++) gt += h[v];
+    p.tie_take[c] = take;
+    run += eq;
+    ssum += gt + take;
+  }
+  const uint32_t spre = block_excl_scan<1024>(ssum, s_w, tot);
+  run = epre;
+  uint32_t srun = spre;
+  for (int c = c0; c < c1; c++) {
+    const uint16_t* h = p.chunk_vh + (size_t)c * stride;
+    const uint32_t eq = h[vstar];
+    const uint32_t take = run >= quota ? 0u : min(eq, quota - run);
+    uint32_t gt = 0;
+    for (int v = (int)vstar + 1; v <= p.N; v++) gt += h[v];
+    p.out_base[c] = srun;
+    run += eq;
+    srun += gt + take;
+  }
+}
+
+// writes supp(M) (ascending) and optionally M as a bit mask
+__global__ void __launch_bounds__(TPB) k_vote_write(P p, const uint8_t* __restrict__ votes, int32_t* __restrict__ out_idx,
+                                                    uint32_t* __restrict__ mask_bits) {
+  __shared__ uint32_t s_w[TPB / 32 + 1];
+  const int c = blockIdx.x, tid = threadIdx.x;
+  const uint32_t vstar = p.vstate[0];
+  const uint32_t take = p.tie_take[c];
+  const uint32_t ob = p.out_base[c];
+  const int64_t jb = (int64_t)c * CH + (int64_t)tid * 16;
+  uint32_t gm = 0, em = 0;
+  if (jb < p.d) {
+    if (jb + 16 <= p.d) {
+      const uint4 q = *reinterpret_cast<const uint4*>(votes + jb);
+      const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+      for (int b = 0; b < 16; b++) {
+        const uint32_t v = (w[b >> 2] >> (8 * (b & 3))) & 0xffu;
+        gm |= (v > vstar ? 1u : 0u) << b;
+        em |= (v == vstar ? 1u : 0u) << b;
+      }
+    } else {
+      for (int b = 0; b < 16 && jb + b < p.d; b++) {
+        const uint32_t v = votes[jb + b];
+        gm |= (v > vstar ? 1u : 0u) << b;
+        em |= (v == vstar ? 1u : 0u) << b;
+      }
+    }
+  }
+  uint32_t sm = gm;
+  if (take > 0) {  // uniform over the CTA
+    uint32_t tot;
+    const uint32_t epre = block_excl_scan<TPB>(__popc(em), s_w, tot);
+    if (epre < take) {
+      const uint32_t room = take - epre;  // keep this thread's first `room` ties
+      uint32_t e2 = em, kept = 0, cntk = 0;
+      while (e2 && cntk < room) {
+        const uint32_t low = e2 & (0u - e2);
+        kept |= low;
+        e2 ^= low;
+        cntk++;
+      }
+      sm |= kept;
+    }
+  }
+  uint32_t tot;
+  uint32_t pos = ob + block_excl_scan<TPB>(__popc(sm), s_w, tot);
+  uint32_t s2 = sm;
+  while (s2) {
+    const int b = __ffs(s2) - 1;
+    s2 &= s2 - 1;
+    if (pos < (uint32_t)p.K) out_idx[pos] = (int32_t)(jb + b);
+    pos++;
+  }
+  if (mask_bits != nullptr) {
+    const uint32_t other = __shfl_xor_sync(FULL, sm, 1);
+    if ((tid & 1) == 0) {
+      const int64_t wi = (int64_t)c * WPC + (tid >> 1);
+      if (wi < p.W) mask_bits[wi] = sm | (other << 16);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// aggregate: out_val[k] = fl32( (sum_n (double)acc[n][idx[k]]) / N ), then acc[n][idx[k]] = +0
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(TPB) k_gather(float* __restrict__ acc, int N, int64_t d, int64_t K,
+                                                const int32_t* __restrict__ idx, float* __restrict__ out_val) {
+  const int64_t k = (int64_t)blockIdx.x * TPB + threadIdx.x;
+  if (k >= K) return;
+  const int64_t j = idx[k];
+  if (j < 0 || j >= d) {
+    out_val[k] = 0.f;
+    return;
+  }
+  float* col = acc + j;
+  double s = 0.0;
+  int n = 0;
+  for (; n + 8 <= N; n += 8) {
+    float v[8];
+#pragma unroll
+    for (int q = 0; q < 8; q++) v[q] = col[(size_t)(n + q) * (size_t)d];
+#pragma unroll
+    for (int q = 0; q < 8; q++) {
+      s += (double)v[q];
+      col[(size_t)(n + q) * (size_t)d] = 0.0f;
+    }
+  }
+  for (; n < N; n++) {
+    s += (double)col[(size_t)n * (size_t)d];
+    col[(size_t)n * (size_t)d] = 0.0f;
+  }
+  out_val[k] = (float)(s / (double)N);
+}
+
+// ---------------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------------
+struct Layout {
+  int nchunks;
+  int64_t W;
+  uint32_t cap;
+  size_t zero_bytes;  // the leading region cleared at the start of every vote
+  size_t samp_hist, hist1, hist2, hist3, cand_cnt, vote_hist;
+  size_t tau, wstate, thresh, vstate, cand, chunk_base, chunk_cnt, chunk_gt, chunk_eq, tie_base, sel_base;
+  size_t worker_bits, worker_idx, votes, chunk_vh, out_base, tie_take;
+  size_t total;
+};
+
+bool sizes_ok(int N, int64_t d, int64_t K) {
+  return N >= 1 && N <= 255 && d >= 1 && d < ((int64_t)1 << 31) - 8192 && K >= 1 && K <= d;
+}
+
+size_t take(size_t& off, size_t bytes) {
+  const size_t at = off;
+  off += (bytes + 255) & ~(size_t)255;
+  return at;
+}
+
+Layout make_layout(int N, int64_t d, int64_t K) {
+  Layout L;
+  L.nchunks = (int)((d + CH - 1) / CH);
+  L.W = (d + 31) / 32;
+  const int64_t cap = 4 * K + 4096;
+  L.cap = (uint32_t)(cap < d ? cap : d);
+  size_t off = 0;
+  const size_t n = (size_t)N, nc = (size_t)L.nchunks;
+  L.samp_hist = take(off, n * SB_BINS * 4);
+  L.hist1 = take(off, n * H1_BINS * 4);
+  L.hist2 = take(off, n * H2_BINS * 4);
+  L.hist3 = take(off, n * H3_BINS * 4);
+  L.cand_cnt = take(off, n * 4);
+  L.vote_hist = take(off, 256 * 4);
+  L.zero_bytes = off;
+  L.tau = take(off, n * 4);
+  L.wstate = take(off, n * 8 * 4);
+  L.thresh = take(off, n * 3 * 4);
+  L.vstate = take(off, 4 * 4);
+  L.cand = take(off, n * (size_t)L.cap * 8);
+  L.chunk_base = take(off, n * nc * 4);
+  L.chunk_cnt = take(off, n * nc * 4);
+  L.chunk_gt = take(off, n * nc * 4);
+  L.chunk_eq = take(off, n * nc * 4);
+  L.tie_base = take(off, n * nc * 4);
+  L.sel_base = take(off, n * nc * 4);
+  L.worker_bits = take(off, n * (size_t)L.W * 4);
+  L.worker_idx = take(off, n * (size_t)K * 4);
+  L.votes = take(off, nc * CH);
+  L.chunk_vh = take(off, nc * (n + 1) * 2);
+  L.out_base = take(off, nc * 4);
+  L.tie_take = take(off, nc * 4);
+  L.total = off;
+  return L;
+}
+
+bool aligned16(const void* q) { return ((uintptr_t)q & 15u) == 0; }
+
+}  // namespace
+
+struct mv_ctx {
+  cudaStream_t stream;
+  char* ws;
+  size_t ws_bytes;
+  int mode;
+  int launches;
+  // optional CUDA-event timing of the streaming pass (ring of event pairs)
+  int timing;
+  int timed;                 // pairs recorded since the last read
+  cudaEvent_t ev[2 * 64];
+  bool ev_made;
+  // remembered for mv_read_diag
+  int last_N;
+  int64_t last_d, last_K;
+};
+
+namespace {
+
+P make_params(const mv_ctx* ctx, const Layout& L, int N, int64_t d, int64_t K) {
+  P p;
+  char* b = ctx->ws;
+  p.N = N;
+  p.nchunks = L.nchunks;
+  p.cap = L.cap;
+  p.force_general = ctx->mode == MV_MODE_GENERAL ? 1 : 0;
+  p.d = d;
+  p.K = K;
+  p.W = L.W;
+  p.samp_hist = (uint32_t*)(b + L.samp_hist);
+  p.hist1 = (uint32_t*)(b + L.hist1);
+  p.hist2 = (uint32_t*)(b + L.hist2);
+  p.hist3 = (uint32_t*)(b + L.hist3);
+  p.cand_cnt = (uint32_t*)(b + L.cand_cnt);
+  p.vote_hist = (uint32_t*)(b + L.vote_hist);
+  p.tau = (uint32_t*)(b + L.tau);
+  p.wstate = (uint32_t*)(b + L.wstate);
+  p.thresh = (uint32_t*)(b + L.thresh);
+  p.vstate = (uint32_t*)(b + L.vstate);
+  p.cand = (uint2*)(b + L.cand);
+  p.chunk_base = (uint32_t*)(b + L.chunk_base);
+  p.chunk_cnt = (uint32_t*)(b + L.chunk_cnt);
+  p.chunk_gt = (uint32_t*)(b + L.chunk_gt);
+  p.chunk_eq = (uint32_t*)(b + L.chunk_eq);
+  p.tie_base = (uint32_t*)(b + L.tie_base);
+  p.sel_base = (uint32_t*)(b + L.sel_base);
+  p.worker_bits = (uint32_t*)(b + L.worker_bits);
+  p.worker_idx = (int32_t*)(b + L.worker_idx);
+  p.votes = (uint8_t*)(b + L.votes);
+  p.chunk_vh = (uint16_t*)(b + L.chunk_vh);
+  p.out_base = (uint32_t*)(b + L.out_base);
+  p.tie_take = (uint32_t*)(b + L.tie_take);
+  return p;
+}
+
+int per_row_ctas(int N, int want, int budget) {
+  int lim = budget / N;
+  if (lim < 1) lim = 1;
+  if (want < 1) want = 1;
+  return want < lim ? want : lim;
+}
+
+#define MV_LAUNCH_CHECK()                          \
+  do {                                             \
+    ctx->launches++;                               \
+    if (cudaGetLastError() != cudaSuccess) return MV_ERR_CUDA; \
+  } while (0)
+
+// sample size and rank for the threshold estimate
+void sample_plan(int64_t d, int64_t K, uint32_t& U, uint32_t& L, int& all, uint32_t& rank) {
+  int64_t S = d / 64;
+  if (S < 131072) S = 131072;
+  if (S > (1 << 20)) S = 1 << 20;
+  if (d <= 2 * S) {
+    all = 1;
+    U = (uint32_t)((d + 31) / 32);
+    L = U;
+    rank = (uint32_t)K;
+    return;
+  }
+  all = 0;
+  U = (uint32_t)(S / 32);
+  L = (uint32_t)(d / 32);
+  const double Sn = (double)U * 32.0;
+  const double m = Sn * (double)K / (double)d;
+  double r = ceil(m + 6.0 * sqrt(m) + 8.0);
+  if (r > Sn) r = Sn;
+  rank = (uint32_t)r;
+}
+
+// steps a1-a3: accumulate, per-worker top-K, votes
+int vote_impl(mv_ctx* ctx, P p, const Layout& L, const float* grads, float* err) {
+  cudaStream_t st = ctx->stream;
+  const int N = p.N;
+  if (cudaMemsetAsync(ctx->ws, 0, L.zero_bytes, st) != cudaSuccess) return MV_ERR_CUDA;
+  const int gg = per_row_ctas(N, p.nchunks, 148 * 8);
+  if (!p.force_general) {
+    uint32_t U, Ls, rank;
+    int all;
+    sample_plan(p.d, p.K, U, Ls, all, rank);
+    const int gs = per_row_ctas(N, (int)((U + 63) / 64), 148 * 2);
+    k_sample_hist<<<dim3(gs, N), 512, 0, st>>>(p, grads, err, U, Ls, all);
+    MV_LAUNCH_CHECK();
+    k_sample_pick<<<N, TPB, 0, st>>>(p, rank);
+    MV_LAUNCH_CHECK();
+    if (ctx->timing) cudaEventRecord(ctx->ev[2 * (ctx->timed % 64)], st);
+    k_acc_compact<<<dim3(p.nchunks, N), TPB, 0, st>>>(p, grads, err);
+    MV_LAUNCH_CHECK();
+    if (ctx->timing) cudaEventRecord(ctx->ev[2 * (ctx->timed++ % 64) + 1], st);
+    const int gc = per_row_ctas(N, (int)((p.cap + TPB * 16 - 1) / (TPB * 16)), 148 * 4);
+    k_cand_hist<1><<<dim3(gc, N), TPB, 0, st>>>(p);
+    MV_LAUNCH_CHECK();
+    k_cand_hist<2><<<dim3(gc, N), TPB, 0, st>>>(p);
+    MV_LAUNCH_CHECK();
+    k_cand_hist<3><<<dim3(gc, N), TPB, 0, st>>>(p);
+    MV_LAUNCH_CHECK();
+    const int g4 = per_row_ctas(N, (p.nchunks + 31) / 32, 148 * 4);
+    k_cand_count<<<dim3(g4, N), TPB, 0, st>>>(p);
+    MV_LAUNCH_CHECK();
+    k_row_hist<1, false><<<dim3(gg, N), TPB, 0, st>>>(p, nullptr, err);
+    MV_LAUNCH_CHECK();
+  } else {
+    if (ctx->timing) cudaEventRecord(ctx->ev[2 * (ctx->timed % 64)], st);
+    k_row_hist<1, true><<<dim3(gg, N), TPB, 0, st>>>(p, grads, err);
+    MV_LAUNCH_CHECK();
+    if (ctx->timing) cudaEventRecord(ctx->ev[2 * (ctx->timed++ % 64) + 1], st);
+  }
+  k_row_hist<2, false><<<dim3(gg, N), TPB, 0, st>>>(p, nullptr, err);
+  MV_LAUNCH_CHECK();
+  k_row_hist<3, false><<<dim3(gg, N), TPB, 0, st>>>(p, nullptr, err);
+  MV_LAUNCH_CHECK();
+  k_row_count<<<dim3(gg, N), TPB, 0, st>>>(p, err);
+  MV_LAUNCH_CHECK();
+  k_chunk_scan<<<N, 1024, 0, st>>>(p);
+  MV_LAUNCH_CHECK();
+  k_row_exact<<<dim3(gg, N), TPB, 0, st>>>(p, err);
+  MV_LAUNCH_CHECK();
+  k_build_votes<<<p.nchunks, TPB, 0, st>>>(p);
+  MV_LAUNCH_CHECK();
+  return MV_OK;
+}
+
+// step a4; `have_hist`: chunk_vh / vote_hist were already filled by k_build_votes
+int select_impl(mv_ctx* ctx, P p, const Layout& L, const uint8_t* votes, bool have_hist, int32_t* out_idx,
+                uint32_t* mask_bits) {
+  cudaStream_t st = ctx->stream;
+  if (!have_hist) {
+    if (cudaMemsetAsync(ctx->ws + L.vote_hist, 0, 256 * 4, st) != cudaSuccess) return MV_ERR_CUDA;
+    k_vote_hist<<<p.nchunks, TPB, 0, st>>>(p, votes);
+    MV_LAUNCH_CHECK();
+  }
+  k_vote_scan<<<1, 1024, 0, st>>>(p);
+  MV_LAUNCH_CHECK();
+  k_vote_write<<<p.nchunks, TPB, 0, st>>>(p, votes, out_idx, mask_bits);
+  MV_LAUNCH_CHECK();
+  return MV_OK;
+}
+
+// steps a5-a6
+int aggregate_impl(mv_ctx* ctx, float* acc, int N, int64_t d, int64_t K, const int32_t* idx, float* out_val) {
+  k_gather<<<(unsigned)((K + TPB - 1) / TPB), TPB, 0, ctx->stream>>>(acc, N, d, K, idx, out_val);
+  MV_LAUNCH_CHECK();
+  return MV_OK;
+}
+
+bool overlap(const void* a, size_t na, const void* b, size_t nb) {
+  const uintptr_t x = (uintptr_t)a, y = (uintptr_t)b;
+  return x < y + nb && y < x + na;
+}
+
+int check_common(const mv_ctx* ctx, int N, int64_t d, int64_t K, Layout& L) {
+  if (ctx == nullptr) return MV_ERR_INVALID_ARG;
+  if (!sizes_ok(N, d, K)) return MV_ERR_INVALID_ARG;
+  L = make_layout(N, d, K);
+  if (ctx->ws_bytes < L.total) return MV_ERR_WORKSPACE;
+  return MV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t mv_workspace_bytes(int N, int64_t d, int64_t K) {
+  if (!sizes_ok(N, d, K)) return 0;
+  return make_layout(N, d, K).total;
+}
+
+int mv_create(mv_ctx** out, void* stream, void* workspace, size_t workspace_bytes) {
+  if (out == nullptr) return MV_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (workspace == nullptr || ((uintptr_t)workspace & 255u) != 0) return MV_ERR_INVALID_ARG;
+  mv_ctx* c = new (std::nothrow) mv_ctx;
+  if (c == nullptr) return MV_ERR_INVALID_ARG;
+  c->stream = (cudaStream_t)stream;
+  c->ws = (char*)workspace;
+  c->ws_bytes = workspace_bytes;
+  c->mode = MV_MODE_AUTO;
+  c->launches = 0;
+  c->timing = 0;
+  c->timed = 0;
+  c->ev_made = false;
+  c->last_N = 0;
+  c->last_d = 0;
+  c->last_K = 0;
+  *out = c;
+  return MV_OK;
+}
+
+int mv_destroy(mv_ctx* ctx) {
+  if (ctx == nullptr) return MV_ERR_INVALID_ARG;
+  if (ctx->ev_made)
+    for (int i = 0; i < 2 * 64; i++) cudaEventDestroy(ctx->ev[i]);
+  delete ctx;
+  return MV_OK;
+}
+
+int mv_set_kernel_timing(mv_ctx* ctx, int enable) {
+  if (ctx == nullptr) return MV_ERR_INVALID_ARG;
+  if (enable && !ctx->ev_made) {
+    for (int i = 0; i < 2 * 64; i++)
+      if (cudaEventCreate(&ctx->ev[i]) != cudaSuccess) return MV_ERR_CUDA;
+    ctx->ev_made = true;
+  }
+  ctx->timing = enable ? 1 : 0;
+  ctx->timed = 0;
+  return MV_OK;
+}
+
+int mv_read_kernel_timing(mv_ctx* ctx, float* total_ms, int* launches) {
+  if (ctx == nullptr || total_ms == nullptr || launches == nullptr || !ctx->ev_made) return MV_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return MV_ERR_CUDA;
+  const int cnt = ctx->timed < 64 ? ctx->timed : 64;
+  float sum = 0.f;
+  for (int i = 0; i < cnt; i++) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, ctx->ev[2 * i], ctx->ev[2 * i + 1]) != cudaSuccess) return MV_ERR_CUDA;
+    sum += ms;
+  }
+  *total_ms = sum;
+  *launches = cnt;
+  ctx->timed = 0;
+  return MV_OK;
+}
+
+int mv_set_mode(mv_ctx* ctx, int mode) {
+  if (ctx == nullptr || (mode != MV_MODE_AUTO && mode != MV_MODE_GENERAL)) return MV_ERR_INVALID_ARG;
+  ctx->mode = mode;
+  return MV_OK;
+}
+
+int mv_vote(mv_ctx* ctx, const float* grads, float* err, int N, int64_t d, int64_t K, int32_t* worker_idx,
+            uint32_t* worker_bits, uint8_t* votes, uint32_t* thresh) {
+  Layout L;
+  const int rc = check_common(ctx, N, d, K, L);
+  if (rc != MV_OK) return rc;
+  if (grads == nullptr || err == nullptr || !aligned16(grads) || !aligned16(err)) return MV_ERR_INVALID_ARG;
+  const size_t nb = (size_t)N * (size_t)d * 4;
+  if (overlap(grads, nb, err, nb)) return MV_ERR_INVALID_ARG;
+  if ((worker_idx && !aligned16(worker_idx)) || (worker_bits && !aligned16(worker_bits)) ||
+      (votes && !aligned16(votes)) || (thresh && !aligned16(thresh)))
+    return MV_ERR_INVALID_ARG;
+  ctx->launches = 0;
+  P p = make_params(ctx, L, N, d, K);
+  if (worker_idx) p.worker_idx = worker_idx;
+  if (worker_bits) p.worker_bits = worker_bits;
+  if (votes) p.votes = votes;
+  if (thresh) p.thresh = thresh;
+  ctx->last_N = N;
+  ctx->last_d = d;
+  ctx->last_K = K;
+  return vote_impl(ctx, p, L, grads, err);
+}
+
+int mv_select(mv_ctx* ctx, const uint8_t* votes, int N, int64_t d, int64_t K, int32_t* out_idx, uint32_t* mask_bits) {
+  Layout L;
+  const int rc = check_common(ctx, N, d, K, L);
+  if (rc != MV_OK) return rc;
+  if (votes == nullptr || out_idx == nullptr || !aligned16(votes) || !aligned16(out_idx)) return MV_ERR_INVALID_ARG;
+  if (mask_bits && !aligned16(mask_bits)) return MV_ERR_INVALID_ARG;
+  ctx->launches = 0;
+  P p = make_params(ctx, L, N, d, K);
+  return select_impl(ctx, p, L, votes, false, out_idx, mask_bits);
+}
+
+int mv_aggregate(mv_ctx* ctx, float* acc, int N, int64_t d, int64_t K, const int32_t* idx, float* out_val) {
+  Layout L;
+  const int rc = check_common(ctx, N, d, K, L);
+  if (rc != MV_OK) return rc;
+  if (acc == nullptr || idx == nullptr || out_val == nullptr || !aligned16(acc) || !aligned16(idx) || !aligned16(out_val))
+    return MV_ERR_INVALID_ARG;
+  ctx->launches = 0;
+  return aggregate_impl(ctx, acc, N, d, K, idx, out_val);
+}
+
+int mv_sparse_step(mv_ctx* ctx, const float* grads, float* err, int N, int64_t d, int64_t K, int32_t* out_idx,
+                   float* out_val) {
+  Layout L;
+  int rc = check_common(ctx, N, d, K, L);
+  if (rc != MV_OK) return rc;
+  if (grads == nullptr || err == nullptr || out_idx == nullptr || out_val == nullptr) return MV_ERR_INVALID_ARG;
+  if (!aligned16(grads) || !aligned16(err) || !aligned16(out_idx) || !aligned16(out_val)) return MV_ERR_INVALID_ARG;
+  const size_t nb = (size_t)N * (size_t)d * 4;
+  if (overlap(grads, nb, err, nb)) return MV_ERR_INVALID_ARG;
+  ctx->launches = 0;
+  P p = make_params(ctx, L, N, d, K);
+  ctx->last_N = N;
+  ctx->last_d = d;
+  ctx->last_K = K;
+  rc = vote_impl(ctx, p, L, grads, err);
+  if (rc != MV_OK) return rc;
+  rc = select_impl(ctx, p, L, p.votes, true, out_idx, nullptr);
+  if (rc != MV_OK) return rc;
+  return aggregate_impl(ctx, err, N, d, K, out_idx, out_val);
+}
+
+int mv_sparse_step_host(mv_ctx* ctx, const float* h_grads, int N, int64_t d, int64_t K, int32_t* h_out_idx,
+                        float* h_out_val, float* d_grads, float* d_err, int32_t* d_out_idx, float* d_out_val) {
+  Layout L;
+  int rc = check_common(ctx, N, d, K, L);
+  if (rc != MV_OK) return rc;
+  if (h_grads == nullptr || h_out_idx == nullptr || h_out_val == nullptr) return MV_ERR_INVALID_ARG;
+  if (d_grads == nullptr || d_err == nullptr || d_out_idx == nullptr || d_out_val == nullptr) return MV_ERR_INVALID_ARG;
+  if (!aligned16(d_grads) || !aligned16(d_err) || !aligned16(d_out_idx) || !aligned16(d_out_val)) return MV_ERR_INVALID_ARG;
+  const size_t nb = (size_t)N * (size_t)d * 4;
+  if (overlap(d_grads, nb, d_err, nb)) return MV_ERR_INVALID_ARG;
+  if (cudaMemcpyAsync(d_grads, h_grads, nb, cudaMemcpyHostToDevice, ctx->stream) != cudaSuccess) return MV_ERR_CUDA;
+  rc = mv_sparse_step(ctx, d_grads, d_err, N, d, K, d_out_idx, d_out_val);
+  if (rc != MV_OK) return rc;
+  if (cudaMemcpyAsync(h_out_idx, d_out_idx, (size_t)K * 4, cudaMemcpyDeviceToHost, ctx->stream) != cudaSuccess)
+    return MV_ERR_CUDA;
+  if (cudaMemcpyAsync(h_out_val, d_out_val, (size_t)K * 4, cudaMemcpyDeviceToHost, ctx->stream) != cudaSuccess)
+    return MV_ERR_CUDA;
+  if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return MV_ERR_CUDA;
+  return MV_OK;
+}
+
+int mv_read_diag(mv_ctx* ctx, int N, uint32_t* per_worker) {
+  if (ctx == nullptr || per_worker == nullptr || N < 1 || N != ctx->last_N) return MV_ERR_INVALID_ARG;
+  const Layout L = make_layout(ctx->last_N, ctx->last_d, ctx->last_K);
+  uint32_t* cnt = (uint32_t*)malloc((size_t)N * 8);
+  if (cnt == nullptr) return MV_ERR_INVALID_ARG;
+  uint32_t* tau = cnt + N;
+  cudaError_t e = cudaMemcpyAsync(cnt, ctx->ws + L.cand_cnt, (size_t)N * 4, cudaMemcpyDeviceToHost, ctx->stream);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(tau, ctx->ws + L.tau, (size_t)N * 4, cudaMemcpyDeviceToHost, ctx->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
+  if (e != cudaSuccess) {
+    free(cnt);
+    return MV_ERR_CUDA;
+  }
+  for (int n = 0; n < N; n++) {
+    const bool general = ctx->mode == MV_MODE_GENERAL || cnt[n] < (uint32_t)ctx->last_K || cnt[n] > L.cap;
+    per_worker[n * 4 + 0] = cnt[n];
+    per_worker[n * 4 + 1] = ctx->mode == MV_MODE_GENERAL ? 0u : tau[n];
+    per_worker[n * 4 + 2] = general ? 1u : 0u;
+    per_worker[n * 4 + 3] = 0u;
+  }
+  free(cnt);
+  return MV_OK;
+}
+
+int mv_last_launches(const mv_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+const char* mv_status_string(int status) {
+  switch (status) {
+    case MV_OK: return "ok";
+    case MV_ERR_INVALID_ARG: return "invalid argument (null or misaligned pointer, size out of range, or grads overlapping err)";
+    case MV_ERR_WORKSPACE: return "workspace smaller than mv_workspace_bytes(N, d, K)";
+    case MV_ERR_CUDA: return "the CUDA runtime reported an error";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

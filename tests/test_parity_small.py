@@ -1,0 +1,213 @@
+"""GPU parity, small and mid sizes: every entry point against the CPU oracle, element by element,
+in both threshold modes, over shapes that cover several chunks, ragged tails, misaligned rows,
+ties, degenerate inputs and the fallback from the sampled pass to the exact select."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mv_oracle as O
+from paper_2011_06495_b200 import binding as B
+from paper_2011_06495_b200 import workloads as WL
+from tests import parity as PT
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+MODES = [B.MV_MODE_AUTO, B.MV_MODE_GENERAL]
+
+
+def make(N, d, kind, seed):
+    g = torch.Generator().manual_seed(seed)
+    grads = torch.randn(N, d, generator=g)
+    err = 0.3 * torch.randn(N, d, generator=g)
+    if kind == "gauss":
+        pass
+    elif kind == "ties":
+        grads = (grads * 4).round() / 4
+        err = (err * 4).round() / 4
+    elif kind == "equal":
+        grads = torch.full((N, d), 0.5)
+        grads[::2] *= -1
+        err = torch.full((N, d), 0.25)
+        err[::2] *= -1
+    elif kind == "zeros":
+        grads = torch.zeros(N, d)
+        err = torch.zeros(N, d)
+    elif kind == "sparse":          # mostly zero, a few large values: threshold lands on the zero ties
+        keep = torch.rand(N, d, generator=g) < 0.01
+        grads = grads * keep
+        err = torch.zeros(N, d)
+    elif kind == "layers":          # scale changes by decades along the row
+        scale = 10.0 ** (-3 * torch.arange(d) / max(d - 1, 1))
+        grads = grads * scale
+        err = err * scale
+    else:
+        raise ValueError(kind)
+    return grads.float().contiguous(), err.float().contiguous()
+
+
+SHAPES = [
+    # N, d, K
+    (1, 1, 1), (1, 5, 5), (3, 31, 4), (2, 33, 33), (4, 4096, 10), (4, 4097, 7), (3, 8191, 100),
+    (5, 10001, 1000), (7, 12289, 1), (9, 65538, 655), (10, 100003, 1000), (33, 5000, 50), (64, 20000, 200),
+    (2, 12288, 12288), (3, 9001, 9000),
+]
+
+
+@pytest.mark.parametrize("mode", MODES, ids=["auto", "general"])
+@pytest.mark.parametrize("kind", ["gauss", "ties", "layers"])
+@pytest.mark.parametrize("N,d,K", SHAPES)
+def test_shapes(N, d, K, kind, mode):
+    grads, err = make(N, d, kind, seed=N * 1000 + d + K)
+    ctx = B.MvContext(N, d, K, device=DEV, mode=mode)
+    PT.compare_all(ctx, grads.to(DEV), err.to(DEV), K, by_sort=(d <= 20000), label=f"[{N}x{d} K={K} {kind}] ")
+
+
+@pytest.mark.parametrize("mode", MODES, ids=["auto", "general"])
+@pytest.mark.parametrize("kind", ["equal", "zeros", "sparse"])
+@pytest.mark.parametrize("N,d,K", [(3, 5000, 17), (4, 20011, 300), (2, 300007, 10)])
+def test_degenerate(N, d, K, kind, mode):
+    grads, err = make(N, d, kind, seed=d + K)
+    ctx = B.MvContext(N, d, K, device=DEV, mode=mode)
+    PT.compare_all(ctx, grads.to(DEV), err.to(DEV), K, label=f"[{N}x{d} K={K} {kind}] ")
+
+
+def test_max_workers():
+    N, d, K = 255, 3001, 30
+    grads, err = make(N, d, "ties", seed=255)
+    ctx = B.MvContext(N, d, K, device=DEV)
+    PT.compare_all(ctx, grads.to(DEV), err.to(DEV), K, label="[N=255] ")
+
+
+@pytest.mark.parametrize("name", ["c1", "c1_ties"])
+@pytest.mark.parametrize("mode", MODES, ids=["auto", "general"])
+def test_config_c1(name, mode):
+    w = WL.resnet_like(name)
+    grads = WL.gradients(w, 0)
+    err = WL.initial_err(w)
+    if name == "c1":
+        key = O.magnitude_key(grads.numpy())
+        assert all(np.unique(key[n]).size == w.d for n in range(w.N)), "c1 is meant to be tie-free"
+    ctx = B.MvContext(w.N, w.d, w.K, device=DEV, mode=mode)
+    ref, ph, fu = PT.compare_all(ctx, grads.to(DEV), err.to(DEV), w.K, by_sort=True, label=f"[{name}] ")
+    if name == "c1_ties":
+        assert (ref["thresh"][:, 2] > 1).all(), "forced ties should straddle every worker's threshold"
+
+
+def test_special_values():
+    """Signed zeros, denormals and infinities follow the bit-pattern order; residual bytes are exact."""
+    N, d, K = 3, 4500, 40
+    grads, err = make(N, d, "gauss", seed=4500)
+    grads[0, 7] = float("inf")
+    grads[1, 4099] = float("-inf")
+    grads[2, 10:60] = 1e-41          # denormals
+    err[2, 10:60] = 0.0
+    grads[0, 100:200] = -0.0
+    err[0, 100:200] = -0.0
+    for mode in MODES:
+        ctx = B.MvContext(N, d, K, device=DEV, mode=mode)
+        PT.compare_all(ctx, grads.to(DEV), err.to(DEV), K, by_sort=True, label="[special] ")
+
+
+@pytest.mark.parametrize("N,d,K", [(4, 300007, 3000), (3, 1000003, 250), (16, 1 << 20, 1048)])
+def test_sampled_threshold_path(N, d, K):
+    """d large enough that the threshold bound comes from a strided sample; the streaming pass must
+    succeed for every worker (no fallback) on smooth data, and all results stay exact."""
+    grads, err = make(N, d, "gauss", seed=d)
+    ctx = B.MvContext(N, d, K, device=DEV)
+    ref, ph, fu = PT.compare_all(ctx, grads.to(DEV), err.to(DEV), K, label=f"[sampled {N}x{d}] ")
+    diag = ph["diag"]
+    assert (diag[:, 2] == 0).all(), f"fallback used: {diag.tolist()}"
+    assert (diag[:, 0] >= K).all() and (diag[:, 0] <= 4 * K + 4096).all()
+
+
+def test_fallback_per_worker():
+    """One smooth worker next to one whose values are all equal (its candidate count overflows):
+    the second takes the exact multi-pass select, the first does not, results are exact."""
+    N, d, K = 3, 300007, 100
+    grads, err = make(N, d, "gauss", seed=99)
+    grads[1] = 0.125
+    err[1] = 0.0
+    ctx = B.MvContext(N, d, K, device=DEV)
+    ref, ph, fu = PT.compare_all(ctx, grads.to(DEV), err.to(DEV), K, label="[fallback] ")
+    assert ph["diag"][:, 2].tolist() == [0, 1, 0]
+    assert ref["worker_idx"][1].tolist() == list(range(K))
+
+
+def test_error_feedback_over_steps():
+    """Residuals carried over several steps stay bit-identical to the oracle's."""
+    w = WL.scaled(WL.resnet_like("c2"), d=200003, N=6, steps=5)
+    ctx = B.MvContext(w.N, w.d, w.K, device=DEV)
+    err_gpu = WL.initial_err(w).to(DEV)
+    err_ref = WL.initial_err(w).numpy()
+    out_idx = torch.empty(w.K, dtype=torch.int32, device=DEV)
+    out_val = torch.empty(w.K, dtype=torch.float32, device=DEV)
+    for step in range(w.steps):
+        grads = WL.gradients(w, step)
+        ref = O.mv_sparse_step(grads.numpy(), err_ref, w.K)
+        ctx.mv_sparse_step(grads.to(DEV), err_gpu, out_idx, out_val)
+        torch.cuda.synchronize()
+        PT.first_diff(PT.npy(out_idx), ref["out_idx"], f"step {step} out_idx")
+        PT.check_out_val(PT.npy(out_val), ref, ref["acc"], ref["out_idx"].astype(np.int64), f"step {step} out_val")
+        PT.first_diff(PT.bits(PT.npy(err_gpu)), PT.bits(ref["err"]), f"step {step} err")
+        err_ref = ref["err"]
+
+
+def test_checkpoint_resume():
+    """The residual is the only state: saving and restoring it mid-run changes nothing."""
+    w = WL.scaled(WL.resnet_like("c3"), d=50021, N=5, steps=6)
+    outs = []
+    for split in (None, 3):
+        ctx = B.MvContext(w.N, w.d, w.K, device=DEV)
+        err = WL.initial_err(w).to(DEV)
+        out_idx = torch.empty(w.K, dtype=torch.int32, device=DEV)
+        out_val = torch.empty(w.K, dtype=torch.float32, device=DEV)
+        for step in range(w.steps):
+            if split is not None and step == split:
+                saved = err.cpu().clone()
+                ctx = B.MvContext(w.N, w.d, w.K, device=DEV)
+                err = saved.to(DEV)
+            ctx.mv_sparse_step(WL.gradients(w, step).to(DEV), err, out_idx, out_val)
+        torch.cuda.synchronize()
+        outs.append((err.cpu(), out_idx.cpu(), out_val.cpu()))
+    for a, b in zip(*outs):
+        assert torch.equal(a.view(torch.int32), b.view(torch.int32))
+
+
+def test_host_entry_point():
+    """mv_sparse_step_host: gradients in pinned host memory, results back in host memory."""
+    N, d, K = 4, 70001, 700
+    grads, err = make(N, d, "gauss", seed=5)
+    ref = O.mv_sparse_step(grads.numpy(), err.numpy(), K)
+    ctx = B.MvContext(N, d, K, device=DEV)
+    h_grads = grads.pin_memory()
+    h_idx = torch.empty(K, dtype=torch.int32).pin_memory()
+    h_val = torch.empty(K, dtype=torch.float32).pin_memory()
+    d_grads = torch.empty(N, d, device=DEV)
+    d_err = err.to(DEV)
+    d_idx = torch.empty(K, dtype=torch.int32, device=DEV)
+    d_val = torch.empty(K, dtype=torch.float32, device=DEV)
+    ctx.mv_sparse_step_host(h_grads, h_idx, h_val, d_grads, d_err, d_idx, d_val)
+    PT.first_diff(h_idx.numpy(), ref["out_idx"], "host out_idx")
+    PT.check_out_val(h_val.numpy(), ref, ref["acc"], ref["out_idx"].astype(np.int64), "host out_val")
+    PT.first_diff(PT.bits(PT.npy(d_err)), PT.bits(ref["err"]), "host err")
+
+
+def test_argument_errors_on_device_pointers():
+    N, d, K = 2, 1000, 10
+    ctx = B.MvContext(N, d, K, device=DEV)
+    g = torch.zeros(N, d, device=DEV)
+    e = torch.zeros(N, d, device=DEV)
+    oi = torch.zeros(K, dtype=torch.int32, device=DEV)
+    ov = torch.zeros(K, device=DEV)
+    with pytest.raises(B.MvError) as ei:
+        ctx.mv_sparse_step(g, g, oi, ov)                    # grads aliases err
+    assert ei.value.status == B.MV_ERR_INVALID_ARG
+    with pytest.raises(B.MvError) as ei:
+        ctx.mv_sparse_step(g, e, oi, ov, K=d + 1)           # K > d
+    assert ei.value.status == B.MV_ERR_INVALID_ARG
+    big = torch.zeros(N, 100 * d, device=DEV)
+    with pytest.raises(B.MvError) as ei:
+        ctx.mv_sparse_step(big, big.clone(), oi, ov)        # workspace sized for a smaller problem
+    assert ei.value.status == B.MV_ERR_WORKSPACE
+    ctx.mv_sparse_step(g, e, oi, ov)                        # the context is still usable
+    torch.cuda.synchronize()
