@@ -77,12 +77,24 @@ class ClockSampler:
         try:
             self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "20",
                  "-i", str(self.index)], stdout=self.file, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
-    def stop(self):
+    def rows_so_far(self) -> int:
+        try:
+            return sum(1 for r in open(self.file.name) if r.strip())
+        except Exception:
+            return 0
+
+    def wait_for_first_sample(self, limit_s: float = 3.0):
+        t0 = time.time()
+        while self.proc is not None and self.rows_so_far() == 0 and time.time() - t0 < limit_s:
+            time.sleep(0.02)
+
+    def stop(self, first_row: int = 0):
+        """Median SM clock and the throttle reasons seen in the rows from `first_row` on."""
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is None:
             return out
@@ -94,6 +106,7 @@ class ClockSampler:
         try:
             self.file.flush()
             rows = [r.strip().split(", ") for r in open(self.file.name) if r.strip()]
+            rows = rows[max(0, min(first_row, len(rows) - 1)):]
             os.unlink(self.file.name)
         except Exception:
             rows = []
@@ -188,7 +201,7 @@ def workload_config(w: WL.Workload):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=400)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2", choices=["c1", "c1_ties", "c2", "c3", "c4"])
@@ -234,14 +247,16 @@ def main():
     out_val = torch.empty(w.K, dtype=torch.float32, device=dev)
     ctx = B.MvContext(w.N, w.d, w.K, device=dev, mode=B.MV_MODE_GENERAL if args.mode == "general" else B.MV_MODE_AUTO)
 
+    sampler = ClockSampler(visible_gpu_index(local_rank))
+    sampler.start()
     step_no = 0
     for _ in range(args.warmup):
         ctx.mv_sparse_step(pool[step_no % pool_n], err, out_idx, out_val)
         step_no += 1
     ctx.set_kernel_timing(True)
-    sampler = ClockSampler(visible_gpu_index(local_rank))
-    sampler.start()
+    sampler.wait_for_first_sample()
     barrier()
+    first_row = sampler.rows_so_far()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record()
     for _ in range(args.steps):
@@ -249,7 +264,8 @@ def main():
         step_no += 1
     ev1.record()
     barrier()
-    clocks = sampler.stop()
+    time.sleep(0.03)
+    clocks = sampler.stop(first_row)
     ms_total = ev0.elapsed_time(ev1)
     launches_per_step = ctx.last_launches()
     k_ms, k_cnt = ctx.read_kernel_timing()

@@ -3,15 +3,16 @@
 // N workers are the rows of one N x d array.  A step is a short sequence of kernels on
 // one stream, with no host synchronisation and no device allocation:
 //
-//   sample     k_sample_hist, k_sample_pick   a strided sample of |grads+err| per worker gives a
+//   sample     k_sample_hist                  a strided sample of |grads+err| per worker gives a
 //                                             lower bound tau_n on the K-th largest magnitude key
 //   stream     k_acc_compact                  the one pass over N x d: acc = err + grads written in
 //                                             place, elements with key >= tau_n compacted per chunk
-//   select     k_cand_hist<1..3>, k_cand_count  exact K-th key T_n by radix select on the candidates
-//   fallback   k_row_hist<1..3>, k_row_count, k_row_exact   exact radix select over the full rows for
-//                                             workers whose candidate count missed [K, cap]
-//   order      k_chunk_scan                   lowest-index tie quota and list offsets per chunk
-//   vote       k_build_votes                  per-worker bit masks and index lists, bit-sliced vote count
+//   select     k_hist<1..3>, k_count          exact K-th key T_n by radix select: on the candidates, or over
+//                                             the full row for a worker whose candidate count missed [K, cap]
+//   order      k_chunk_scan, k_row_exact      lowest-index tie quota per chunk; exact compaction for the
+//                                             full-row workers
+//   vote       k_set_bits, k_tie_bits, k_votes  per-worker bit masks, bit-sliced vote count
+//   lists      k_scan_sel, k_lists            ascending per-worker index lists from the masks
 //   mask       k_vote_hist, k_vote_scan, k_vote_write   counting select over vote values 0..N
 //   aggregate  k_gather                       mean on the shared mask, residual zeroed in place
 //
@@ -49,6 +50,7 @@ struct P {
   uint32_t* hist2;        // [N][H2_BINS]
   uint32_t* hist3;        // [N][H3_BINS]
   uint32_t* cand_cnt;     // [N]
+  uint32_t* sample_done;  // [N] ticket counters
   uint32_t* vote_hist;    // [256]
   uint32_t* tau;          // [N]
   uint32_t* wstate;       // [N][8]: b1, rem1, b2, rem2, T, cnt_gt, cnt_eq, need
@@ -61,6 +63,7 @@ struct P {
   uint32_t* chunk_eq;
   uint32_t* tie_base;
   uint32_t* sel_base;
+  uint32_t* chunk_sel;    // [N][nchunks] selected elements per chunk
   uint32_t* worker_bits;  // [N][W]
   int32_t* worker_idx;    // [N][K]
   uint8_t* votes;         // [d]
@@ -216,18 +219,18 @@ __device__ __forceinline__ uint32_t eq_mask(const uint32_t (&k)[4], uint32_t t) 
 
 // Finds the bin holding the rank-th largest element of a histogram (rank counted from the top,
 // 1-based): the largest bin b with sum(hist[b..]) >= rank, and rem = rank - sum(hist[b+1..]).
-// All TPB threads call it; if the histogram holds fewer than rank elements, bin = rem = 0.
-template <int NB>
+// All NT threads of the CTA call it; if the histogram holds fewer than rank elements, bin = rem = 0.
+template <int NB, int NT>
 __device__ void block_pick(const uint32_t* __restrict__ hist, uint32_t rank, uint32_t& bin, uint32_t& rem) {
-  constexpr int PER = NB / TPB;
-  __shared__ uint32_t s_wsum[TPB / 32];
+  constexpr int PER = NB / NT;
+  __shared__ uint32_t s_wsum[NT / 32];
   __shared__ uint32_t s_res[2];
   const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
   uint32_t loc[PER];
   uint32_t sum = 0;
 #pragma unroll
   for (int k = 0; k < PER; k++) {
-    loc[k] = hist[t * PER + k];
+    loc[k] = __ldcg(hist + t * PER + k);
     sum += loc[k];
   }
   if (t == 0) {
@@ -243,7 +246,7 @@ __device__ void block_pick(const uint32_t* __restrict__ hist, uint32_t rank, uin
   if (lane == 0) s_wsum[warp] = x;
   __syncthreads();
   uint32_t above = x - sum;
-  for (int w = warp + 1; w < TPB / 32; w++) above += s_wsum[w];
+  for (int w = warp + 1; w < NT / 32; w++) above += s_wsum[w];
   if (above < rank && rank <= above + sum) {
     bool done = false;
 #pragma unroll
@@ -290,11 +293,15 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* s_w /*
 }
 
 // ---------------------------------------------------------------------------------------------
-// sample: histogram of the top 13 key bits over evenly spaced 32-element lines of each row
+// sample: histogram of the top 13 key bits over evenly spaced 32-element lines of each row; the
+// last CTA of a worker to finish turns it into tau_n = lower edge of the bin that holds the
+// rank-th largest sampled key (a ticket counter, no waiting)
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(512) k_sample_hist(P p, const float* __restrict__ grads,
-                                                     const float* __restrict__ err, uint32_t U, uint32_t L, int all) {
+                                                     const float* __restrict__ err, uint32_t U, uint32_t L, int all,
+                                                     uint32_t rank) {
   __shared__ uint32_t sh[SB_BINS];
+  __shared__ uint32_t s_last;
   const int n = blockIdx.y;
   for (int b = threadIdx.x; b < SB_BINS; b += 512) sh[b] = 0;
   __syncthreads();
@@ -309,7 +316,7 @@ __global__ void __launch_bounds__(512) k_sample_hist(P p, const float* __restric
       ok[q] = false;
       a[q] = 0.f;
       if (u < U) {
-        const uint32_t line = all ? u : (uint32_t)(((uint64_t)u * L) / U);
+        const uint32_t line = all ? u : u * L;  // L = line stride
         const int64_t j = (int64_t)line * 32 + lane;
         if (j < p.d) {
           ok[q] = true;
@@ -327,13 +334,14 @@ __global__ void __launch_bounds__(512) k_sample_hist(P p, const float* __restric
     const uint32_t v = sh[b];
     if (v) atomicAdd(&gh[b], v);
   }
-}
-
-// tau_n = lower edge of the sample-histogram bin that holds the rank-th largest sampled key
-__global__ void __launch_bounds__(TPB) k_sample_pick(P p, uint32_t rank) {
-  const int n = blockIdx.x;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) s_last = (atomicAdd(&p.sample_done[n], 1u) == gridDim.x - 1) ? 1u : 0u;
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
   uint32_t bin, rem;
-  block_pick<SB_BINS>(p.samp_hist + (size_t)n * SB_BINS, rank, bin, rem);
+  block_pick<SB_BINS, 512>(gh, rank, bin, rem);
   if (threadIdx.x == 0) p.tau[n] = bin << SB_SHIFT;
 }
 
@@ -350,6 +358,10 @@ __global__ void __launch_bounds__(TPB) k_acc_compact(P p, const float* __restric
   const uint32_t tau = p.tau[n];
   uint32_t key[4][4], vm[4], cm[4];
   load_keys<true>(g, grads, err, key, vm);
+  if (threadIdx.x < WPC) {  // the worker's mask starts out empty
+    const int64_t wi = (int64_t)c * WPC + threadIdx.x;
+    if (wi < p.W) p.worker_bits[(size_t)n * p.W + wi] = 0u;
+  }
   uint32_t xkey[4], xcm = 0;
   if (threadIdx.x == TPB - 1) {
     uint32_t xvm;
@@ -422,7 +434,7 @@ __device__ __forceinline__ uint32_t resolve_prefix(const P& p, int n) {
   uint32_t* ws = p.wstate + (size_t)n * 8;
   if (PASS == 2) {
     uint32_t b1, rem1;
-    block_pick<H1_BINS>(p.hist1 + (size_t)n * H1_BINS, (uint32_t)p.K, b1, rem1);
+    block_pick<H1_BINS, TPB>(p.hist1 + (size_t)n * H1_BINS, (uint32_t)p.K, b1, rem1);
     if (blockIdx.x == 0 && threadIdx.x == 0) {
       ws[0] = b1;
       ws[1] = rem1;
@@ -432,7 +444,7 @@ __device__ __forceinline__ uint32_t resolve_prefix(const P& p, int n) {
   if (PASS == 3) {
     const uint32_t b1 = ws[0], rem1 = ws[1];
     uint32_t b2, rem2;
-    block_pick<H2_BINS>(p.hist2 + (size_t)n * H2_BINS, rem1, b2, rem2);
+    block_pick<H2_BINS, TPB>(p.hist2 + (size_t)n * H2_BINS, rem1, b2, rem2);
     if (blockIdx.x == 0 && threadIdx.x == 0) {
       ws[2] = b2;
       ws[3] = rem2;
@@ -442,15 +454,17 @@ __device__ __forceinline__ uint32_t resolve_prefix(const P& p, int n) {
   return 0;
 }
 
-// Last digit: T_n, cnt_gt, cnt_eq and the tie quota (need) -- returns T.
-__device__ __forceinline__ uint32_t resolve_threshold(const P& p, int n) {
+// Last digit: T_n, cnt_gt, cnt_eq and the tie quota `need` (how many elements equal to T_n are
+// kept); every thread gets T, need and cnt_eq, CTA 0 records them.
+__device__ __forceinline__ uint32_t resolve_threshold(const P& p, int n, uint32_t& need, uint32_t& cnt_eq) {
   uint32_t* ws = p.wstate + (size_t)n * 8;
   const uint32_t b1 = ws[0], b2 = ws[2], rem2 = ws[3];
   uint32_t b3, rem3;
-  block_pick<H3_BINS>(p.hist3 + (size_t)n * H3_BINS, rem2, b3, rem3);
+  block_pick<H3_BINS, TPB>(p.hist3 + (size_t)n * H3_BINS, rem2, b3, rem3);
   const uint32_t T = (b1 << 20) | (b2 << 10) | b3;
+  cnt_eq = __ldcg(p.hist3 + (size_t)n * H3_BINS + b3);
+  need = rem3;
   if (blockIdx.x == 0 && threadIdx.x == 0) {
-    const uint32_t cnt_eq = p.hist3[(size_t)n * H3_BINS + b3];
     const uint32_t cnt_gt = (uint32_t)p.K - rem3;
     ws[4] = T;
     ws[5] = cnt_gt;
@@ -481,79 +495,58 @@ __device__ __forceinline__ uint32_t* hist_of(const P& p, int n) {
   return p.hist3 + (size_t)n * H3_BINS;
 }
 
-template <int PASS>
-__global__ void __launch_bounds__(TPB) k_cand_hist(P p) {
+// Histogram pass PASS for worker blockIdx.y.  A worker whose candidate count landed in [K, cap]
+// ("fast") is counted over its candidate buffer; any other worker over its full row (read back
+// from err, which holds acc by now).  FUSED (PASS 1 only) instead reads grads and err, writes acc
+// and counts every element: the first pass when sampling is switched off.
+template <int PASS, bool FUSED>
+__global__ void __launch_bounds__(TPB) k_hist(P p, const float* __restrict__ grads, float* __restrict__ err) {
   constexpr int NB = PASS == 1 ? H1_BINS : H2_BINS;
   __shared__ uint32_t sh[NB];
   const int n = blockIdx.y;
-  if (!worker_fast(p, n)) return;
+  const bool fast = !FUSED && worker_fast(p, n);
   const uint32_t prefix = resolve_prefix<PASS>(p, n);
   for (int b = threadIdx.x; b < NB; b += TPB) sh[b] = 0;
   __syncthreads();
-  const uint32_t cnt = p.cand_cnt[n];
-  const uint2* cd = p.cand + (size_t)n * p.cap;
-  for (uint32_t i = blockIdx.x * TPB + threadIdx.x; i < cnt; i += gridDim.x * TPB) hist_add<PASS>(sh, cd[i].x, prefix);
-  __syncthreads();
-  uint32_t* gh = hist_of<PASS>(p, n);
-  for (int b = threadIdx.x; b < NB; b += TPB) {
-    const uint32_t v = sh[b];
-    if (v) atomicAdd(&gh[b], v);
-  }
-}
-
-// per chunk: how many candidates lie above / at the threshold
-__global__ void __launch_bounds__(TPB) k_cand_count(P p) {
-  const int n = blockIdx.y;
-  if (!worker_fast(p, n)) return;
-  const uint32_t T = resolve_threshold(p, n);
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint2* cd = p.cand + (size_t)n * p.cap;
-  for (int c = blockIdx.x * (TPB / 32) + warp; c < p.nchunks; c += gridDim.x * (TPB / 32)) {
-    const size_t ci = (size_t)n * p.nchunks + c;
-    const uint32_t cnt = p.chunk_cnt[ci], base = p.chunk_base[ci];
-    uint32_t gt = 0, eq = 0;
-    for (uint32_t i = lane; i < cnt; i += 32) {
-      const uint32_t k = cd[base + i].x;
-      gt += k > T;
-      eq += k == T;
+  if (fast) {
+    const uint32_t cnt = p.cand_cnt[n];
+    const uint2* cd = p.cand + (size_t)n * p.cap;
+    const uint32_t stride = gridDim.x * TPB;
+    const uint32_t lane = threadIdx.x & 31;
+    for (uint32_t b0 = blockIdx.x * TPB + (threadIdx.x & ~31u); b0 < cnt; b0 += 4 * stride) {  // warp-uniform
+      uint32_t k[4];
+#pragma unroll
+      for (int q = 0; q < 4; q++) {
+        const uint32_t i = b0 + q * stride + lane;
+        k[q] = i < cnt ? __ldcg(&cd[i].x) : 0u;
+      }
+#pragma unroll
+      for (int q = 0; q < 4; q++) {
+        if (b0 + q * stride >= cnt) break;  // warp-uniform
+        if (b0 + q * stride + lane < cnt) hist_add<PASS>(sh, k[q], prefix);
+      }
     }
-    gt = __reduce_add_sync(FULL, gt);
-    eq = __reduce_add_sync(FULL, eq);
-    if (lane == 0) {
-      p.chunk_gt[ci] = gt;
-      p.chunk_eq[ci] = eq;
-    }
-  }
-}
-
-// ---------------------------------------------------------------------------------------------
-// fallback / general path: the same radix select over the full rows of the workers that are not
-// "fast".  PASS 1 with ACC fuses the error-feedback add (used when sampling is switched off).
-// ---------------------------------------------------------------------------------------------
-template <int PASS, bool ACC>
-__global__ void __launch_bounds__(TPB) k_row_hist(P p, const float* __restrict__ grads, float* __restrict__ err) {
-  constexpr int NB = PASS == 1 ? H1_BINS : H2_BINS;
-  __shared__ uint32_t sh[NB];
-  const int n = blockIdx.y;
-  if (worker_fast(p, n)) return;
-  const uint32_t prefix = resolve_prefix<PASS>(p, n);
-  for (int b = threadIdx.x; b < NB; b += TPB) sh[b] = 0;
-  __syncthreads();
-  for (int c = blockIdx.x; c < p.nchunks; c += gridDim.x) {
-    const Geom g = chunk_geom(n, c, p.d);
-    uint32_t key[4][4], vm[4];
-    load_keys<ACC>(g, grads, err, key, vm);
+  } else {
+    for (int c = blockIdx.x; c < p.nchunks; c += gridDim.x) {
+      const Geom g = chunk_geom(n, c, p.d);
+      uint32_t key[4][4], vm[4];
+      load_keys<FUSED>(g, grads, err, key, vm);
+      if (FUSED && threadIdx.x < WPC) {  // the worker's mask starts out empty
+        const int64_t wi = (int64_t)c * WPC + threadIdx.x;
+        if (wi < p.W) p.worker_bits[(size_t)n * p.W + wi] = 0u;
+      }
 #pragma unroll
-    for (int i = 0; i < 4; i++)
+      for (int i = 0; i < 4; i++)
 #pragma unroll
-      for (int e = 0; e < 4; e++)
-        if (vm[i] & (1u << e)) hist_add<PASS>(sh, key[i][e], prefix);
-    if (threadIdx.x == TPB - 1) {
-      uint32_t xkey[4], xvm;
-      load_extra<ACC>(g, grads, err, xkey, xvm);
+        for (int e = 0; e < 4; e++)
+          if (vm[i] & (1u << e)) hist_add<PASS>(sh, key[i][e], prefix);
+      if (threadIdx.x == TPB - 1) {
+        uint32_t xkey[4], xvm;
+        load_extra<FUSED>(g, grads, err, xkey, xvm);
 #pragma unroll
-      for (int e = 0; e < 4; e++)
-        if (xvm & (1u << e)) hist_add<PASS>(sh, xkey[e], prefix);
+        for (int e = 0; e < 4; e++)
+          if (xvm & (1u << e)) hist_add<PASS>(sh, xkey[e], prefix);
+      }
     }
   }
   __syncthreads();
@@ -564,12 +557,29 @@ __global__ void __launch_bounds__(TPB) k_row_hist(P p, const float* __restrict__
   }
 }
 
-__global__ void __launch_bounds__(TPB) k_row_count(P p, float* __restrict__ err) {
+// Resolves T_n for every worker, then counts per chunk what the ordering needs:
+//   - a fast worker that keeps all of its threshold ties needs nothing here;
+//   - a fast worker that keeps only some of them needs the ties per chunk (from its candidates);
+//   - any other worker needs, from its full row, the elements above and at the threshold per chunk.
+__global__ void __launch_bounds__(TPB) k_count(P p, float* __restrict__ err) {
   __shared__ uint32_t s_g[TPB / 32], s_e[TPB / 32];
   const int n = blockIdx.y;
-  if (worker_fast(p, n)) return;
-  const uint32_t T = resolve_threshold(p, n);
+  uint32_t need, cnt_eq;
+  const uint32_t T = resolve_threshold(p, n, need, cnt_eq);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (worker_fast(p, n)) {
+    if (need >= cnt_eq) return;  // every tie is kept: no order needed
+    const uint2* cd = p.cand + (size_t)n * p.cap;
+    for (int c = blockIdx.x * (TPB / 32) + warp; c < p.nchunks; c += gridDim.x * (TPB / 32)) {
+      const size_t ci = (size_t)n * p.nchunks + c;
+      const uint32_t cnt = p.chunk_cnt[ci], base = p.chunk_base[ci];
+      uint32_t eq = 0;
+      for (uint32_t i = lane; i < cnt; i += 32) eq += __ldcg(&cd[base + i].x) == T;
+      eq = __reduce_add_sync(FULL, eq);
+      if (lane == 0) p.chunk_eq[ci] = eq;
+    }
+    return;
+  }
   for (int c = blockIdx.x; c < p.nchunks; c += gridDim.x) {
     const Geom g = chunk_geom(n, c, p.d);
     uint32_t key[4][4], vm[4];
@@ -723,6 +733,8 @@ __global__ void __launch_bounds__(1024) k_chunk_scan(P p) {
   __shared__ uint32_t s_w[33];
   const int n = blockIdx.x;
   const uint32_t need = p.wstate[(size_t)n * 8 + 7];
+  const bool fast = worker_fast(p, n);
+  if (fast && need >= p.wstate[(size_t)n * 8 + 6]) return;  // keeps every tie: nothing to order
   const int per = (p.nchunks + 1023) / 1024;
   const int c0 = min(p.nchunks, (int)threadIdx.x * per), c1 = min(p.nchunks, c0 + per);
   const size_t rb = (size_t)n * p.nchunks;
@@ -736,8 +748,9 @@ __global__ void __launch_bounds__(1024) k_chunk_scan(P p) {
     const uint32_t take = run >= need ? 0u : min(eq, need - run);
     p.tie_base[rb + c] = run;
     run += eq;
-    ssum += p.chunk_gt[rb + c] + take;
+    if (!fast) ssum += p.chunk_gt[rb + c] + take;
   }
+  if (fast) return;  // a fast worker only needs tie_base (uniform over the CTA)
   const uint32_t spre = block_excl_scan<1024>(ssum, s_w, tot);
   run = epre;
   uint32_t srun = spre;
@@ -750,147 +763,153 @@ __global__ void __launch_bounds__(1024) k_chunk_scan(P p) {
   }
 }
 
+// s_vh[v] (v >= 1) holds how many coordinates of chunk c got exactly v votes.  Stores, per chunk,
+// the cumulative counts cum[v] = #{votes >= v} (v = 0..N) and adds the exact counts to the global
+// histogram.  All TPB threads call it.
+__device__ __forceinline__ void store_vote_hist_impl(const P& p, int c, uint32_t* s_vh) {
+  const int tid = threadIdx.x;
+  if (tid <= p.N) {
+    const int64_t rem = p.d - (int64_t)c * CH;
+    const uint32_t valid = (uint32_t)(rem < CH ? rem : CH);
+    uint32_t ge = 0;  // coordinates with votes >= max(tid, 1)
+    for (int v = max(tid, 1); v <= p.N; v++) ge += s_vh[v];
+    uint32_t exact;
+    if (tid == 0) {
+      exact = valid - ge;
+      ge = valid;
+    } else {
+      exact = s_vh[tid];
+    }
+    p.chunk_vh[(size_t)c * (p.N + 1) + tid] = (uint16_t)ge;
+    if (exact) atomicAdd(&p.vote_hist[tid], exact);
+  }
+}
+
 // ---------------------------------------------------------------------------------------------
-// vote: one CTA per chunk, all workers.  The selected candidates set bits in shared-memory masks
-// (32 workers at a time); the masks are written out, turned into ascending index lists, and added
-// up bit-sliced (8 counter planes per 32-coordinate word) into the vote count.
+// vote.  (1) k_set_bits: every worker's candidate buffer is walked flat (balanced however the
+// candidates cluster); a thread takes 8 consecutive candidates, which are index-sorted within a
+// chunk's run and so mostly share a mask word, merges their bits and ORs each word into the
+// worker's global bit mask (zeroed by the streaming pass).  (2) k_tie_bits: workers that keep only
+// part of their threshold ties add those, lowest index first.  (3) k_votes: one CTA per chunk adds
+// the N masks bit-sliced (8 counter planes per 32-coordinate word) into the vote count.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(TPB) k_build_votes(P p) {
-  __shared__ uint32_t masks[32][WPC];
-  __shared__ uint32_t s_cnt[32], s_base[32], s_T[32], s_need[32], s_tb[32], s_sb[32], s_partial[32], s_pref[33];
-  __shared__ uint32_t s_vh[256];
-  const int c = blockIdx.x;
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+__global__ void __launch_bounds__(TPB) k_set_bits(P p) {
+  const int n = blockIdx.y;
+  const bool fast = worker_fast(p, n);
+  const uint32_t* ws = p.wstate + (size_t)n * 8;
+  const uint32_t T = ws[4];
+  const bool all_ties = ws[7] >= ws[6];
+  const uint32_t cnt = fast ? p.cand_cnt[n] : (uint32_t)p.K;  // a full-row worker's buffer holds exactly its picks
+  const uint2* cd = p.cand + (size_t)n * p.cap;               // cap is a multiple of 8: rows are 64-byte aligned
+  uint32_t* bits_row = p.worker_bits + (size_t)n * p.W;
+  for (uint32_t i0 = (blockIdx.x * TPB + threadIdx.x) * 8u; i0 < cnt; i0 += gridDim.x * TPB * 8u) {
+    uint4 v[4];
+#pragma unroll
+    for (int q = 0; q < 4; q++) v[q] = __ldcg(reinterpret_cast<const uint4*>(cd + i0) + q);
+    uint32_t curw = 0xffffffffu, acc = 0;
+#pragma unroll
+    for (int q = 0; q < 8; q++) {
+      const uint32_t key = (q & 1) ? v[q >> 1].z : v[q >> 1].x;
+      const uint32_t j = (q & 1) ? v[q >> 1].w : v[q >> 1].y;
+      const bool sel = i0 + q < cnt && (!fast || key > T || (key == T && all_ties));
+      if (sel && (int64_t)j < p.d) {
+        const uint32_t w = j >> 5;
+        if (w != curw) {
+          if (acc) atomicOr(bits_row + curw, acc);
+          curw = w;
+          acc = 0;
+        }
+        acc |= 1u << (j & 31u);
+      }
+    }
+    if (acc) atomicOr(bits_row + curw, acc);
+  }
+}
+
+__global__ void __launch_bounds__(TPB) k_tie_bits(P p) {
+  const int n = blockIdx.y;
+  const uint32_t* ws = p.wstate + (size_t)n * 8;
+  const uint32_t T = ws[4], need = ws[7];
+  if (!worker_fast(p, n) || need >= ws[6]) return;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t lt = lanemask_lt();
+  uint32_t* bits_row = p.worker_bits + (size_t)n * p.W;
+  for (int c = blockIdx.x * (TPB / 32) + warp; c < p.nchunks; c += gridDim.x * (TPB / 32)) {
+    const size_t ci = (size_t)n * p.nchunks + c;
+    const uint32_t cnt = p.chunk_cnt[ci];
+    uint32_t run = p.tie_base[ci];
+    if (cnt == 0 || run >= need) continue;
+    const uint2* cd = p.cand + (size_t)n * p.cap + p.chunk_base[ci];
+    for (uint32_t i0 = 0; i0 < cnt && run < need; i0 += 32) {
+      const uint32_t i = i0 + lane;
+      uint2 kv = make_uint2(0, 0);
+      bool eq = false;
+      if (i < cnt) {
+        kv = __ldcg(cd + i);
+        eq = kv.x == T;
+      }
+      const uint32_t eb = __ballot_sync(FULL, eq);
+      if (eq && run + __popc(eb & lt) < need && (int64_t)kv.y < p.d) atomicOr(bits_row + (kv.y >> 5), 1u << (kv.y & 31u));
+      run += __popc(eb);
+    }
+  }
+}
+
+__global__ void __launch_bounds__(TPB) k_votes(P p) {
+  __shared__ uint32_t s_vh[256];
+  __shared__ uint32_t s_sel[256];
+  __shared__ uint32_t s_any;
+  const int c = blockIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31;
+  s_vh[tid] = 0;
+  s_sel[tid] = 0;
+  if (tid == 0) s_any = 0;
+  __syncthreads();
+  // a chunk in which no worker kept a candidate has all-zero masks: skip reading them
+  if (tid < p.N && p.chunk_cnt[(size_t)tid * p.nchunks + c] != 0) s_any = 1;
+  __syncthreads();
+  const int64_t jb = (int64_t)c * CH + (int64_t)tid * 32;
+  const int64_t wi = (int64_t)c * WPC + tid;
   uint32_t planes[8];
 #pragma unroll
   for (int q = 0; q < 8; q++) planes[q] = 0;
-  s_vh[tid] = 0;
-  for (int g0 = 0; g0 < p.N; g0 += 32) {
-    const int G = min(32, p.N - g0);
-    __syncthreads();  // previous group's readers are done
-    for (int i = tid; i < G * WPC; i += TPB) masks[i / WPC][i % WPC] = 0;
-    if (tid < G) {
-      const int n = g0 + tid;
-      const size_t ci = (size_t)n * p.nchunks + c;
-      const uint32_t* ws = p.wstate + (size_t)n * 8;
-      s_cnt[tid] = p.chunk_cnt[ci];
-      s_base[tid] = p.chunk_base[ci];
-      s_T[tid] = ws[4];
-      s_need[tid] = ws[7];
-      s_partial[tid] = ws[7] < ws[6] ? 1u : 0u;  // not every threshold tie is kept
-      s_tb[tid] = p.tie_base[ci];
-      s_sb[tid] = p.sel_base[ci];
-    }
-    __syncthreads();
-    if (tid == 0) {
-      uint32_t a = 0;
-      for (int g = 0; g < G; g++) {
-        s_pref[g] = a;
-        a += s_cnt[g];
-      }
-      s_pref[G] = a;
-    }
-    __syncthreads();
-    const uint32_t total = s_pref[G];
-    // everything above the threshold, plus the ties of workers that keep all of them
-    for (uint32_t i = tid; i < total; i += TPB) {
-      int lo = 0, hi = G - 1;  // last g with s_pref[g] <= i
-      while (lo < hi) {
-        const int mid = (lo + hi + 1) >> 1;
-        if (s_pref[mid] <= i) lo = mid; else hi = mid - 1;
-      }
-      const int gi = lo;
-      const uint2 kv = p.cand[(size_t)(g0 + gi) * p.cap + s_base[gi] + (i - s_pref[gi])];
-      const uint32_t T = s_T[gi];
-      if (kv.x > T || (kv.x == T && !s_partial[gi])) {
-        const uint32_t rel = kv.y - (uint32_t)(c * CH);
-        if (rel < (uint32_t)CH) atomicOr(&masks[gi][rel >> 5], 1u << (rel & 31u));
-      }
-    }
-    // workers that keep only part of their ties: ordered walk, lowest index first
-    for (int gi = warp; gi < G; gi += TPB / 32) {
-      if (!s_partial[gi] || s_cnt[gi] == 0) continue;
-      const uint2* cd = p.cand + (size_t)(g0 + gi) * p.cap + s_base[gi];
-      const uint32_t T = s_T[gi], need = s_need[gi], cnt = s_cnt[gi];
-      uint32_t run = s_tb[gi];
-      for (uint32_t i0 = 0; i0 < cnt && run < need; i0 += 32) {
-        const uint32_t i = i0 + lane;
-        uint2 kv = make_uint2(0, 0);
-        bool eq = false;
-        if (i < cnt) {
-          kv = cd[i];
-          eq = kv.x == T;
+  if (s_any && tid < WPC) {  // warps 0..3, all lanes
+    const bool inb = wi < p.W;
+    const uint32_t* col = p.worker_bits + (inb ? wi : 0);
+    for (int n0 = 0; n0 < p.N; n0 += 8) {
+      uint32_t w[8];
+#pragma unroll
+      for (int q = 0; q < 8; q++) w[q] = (inb && n0 + q < p.N) ? __ldcg(col + (size_t)(n0 + q) * p.W) : 0u;
+#pragma unroll
+      for (int q = 0; q < 8; q++) {
+        uint32_t carry = w[q];
+        if (n0 + q < p.N) {  // uniform
+          const uint32_t pc = __reduce_add_sync(FULL, (uint32_t)__popc(carry));
+          if (lane == 0 && pc) atomicAdd(&s_sel[n0 + q], pc);
         }
-        const uint32_t eb = __ballot_sync(FULL, eq);
-        if (eq && run + __popc(eb & lt) < need) {
-          const uint32_t rel = kv.y - (uint32_t)(c * CH);
-          if (rel < (uint32_t)CH) atomicOr(&masks[gi][rel >> 5], 1u << (rel & 31u));
-        }
-        run += __popc(eb);
-      }
-    }
-    __syncthreads();
-    // masks out (coalesced)
-    for (int i = tid; i < G * WPC; i += TPB) {
-      const int gi = i / WPC, w = i % WPC;
-      const int64_t wi = (int64_t)c * WPC + w;
-      if (wi < p.W) p.worker_bits[(size_t)(g0 + gi) * p.W + wi] = masks[gi][w];
-    }
-    // ascending index lists: a warp per worker, four mask words per lane
-    for (int gi = warp; gi < G; gi += TPB / 32) {
-      uint32_t m[4];
-      uint32_t pc = 0;
 #pragma unroll
-      for (int q = 0; q < 4; q++) {
-        m[q] = masks[gi][lane * 4 + q];
-        pc += __popc(m[q]);
-      }
-      uint32_t x = pc;
-#pragma unroll
-      for (int off = 1; off < 32; off <<= 1) {
-        const uint32_t y = __shfl_up_sync(FULL, x, off);
-        if (lane >= off) x += y;
-      }
-      uint32_t pos = s_sb[gi] + x - pc;
-      int32_t* lst = p.worker_idx + (size_t)(g0 + gi) * p.K;
-#pragma unroll
-      for (int q = 0; q < 4; q++) {
-        uint32_t mm = m[q];
-        while (mm) {
-          const int b = __ffs(mm) - 1;
-          mm &= mm - 1;
-          if (pos < (uint32_t)p.K) lst[pos] = c * CH + (lane * 4 + q) * 32 + b;
-          pos++;
-        }
-      }
-    }
-    // vote planes: thread w adds word w of every worker into its bit-sliced counters
-    if (tid < WPC) {
-      for (int gi = 0; gi < G; gi++) {
-        uint32_t carry = masks[gi][tid];
-#pragma unroll
-        for (int q = 0; q < 8; q++) {
-          const uint32_t t2 = planes[q] & carry;
-          planes[q] ^= carry;
+        for (int r = 0; r < 8; r++) {
+          const uint32_t t2 = planes[r] & carry;
+          planes[r] ^= carry;
           carry = t2;
         }
       }
     }
   }
   // expand the planes into 32 vote bytes per thread
-  const int64_t jb = (int64_t)c * CH + (int64_t)tid * 32;
   if (tid < WPC && jb < p.d) {
     uint32_t wv[8];
 #pragma unroll
     for (int q = 0; q < 8; q++) wv[q] = 0;
+    if (planes[0] | planes[1] | planes[2] | planes[3] | planes[4] | planes[5] | planes[6] | planes[7]) {
 #pragma unroll
-    for (int b = 0; b < 32; b++) {
-      uint32_t v = 0;
+      for (int b = 0; b < 32; b++) {
+        uint32_t v = 0;
 #pragma unroll
-      for (int q = 0; q < 8; q++) v |= ((planes[q] >> b) & 1u) << q;
-      wv[b >> 2] |= v << (8 * (b & 3));
-      if (v && jb + b < p.d) atomicAdd(&s_vh[v], 1u);
+        for (int q = 0; q < 8; q++) v |= ((planes[q] >> b) & 1u) << q;
+        wv[b >> 2] |= v << (8 * (b & 3));
+        if (v && jb + b < p.d) atomicAdd(&s_vh[v], 1u);
+      }
     }
     if (jb + 32 <= p.d) {
       uint4* dst = reinterpret_cast<uint4*>(p.votes + jb);
@@ -901,17 +920,69 @@ __global__ void __launch_bounds__(TPB) k_build_votes(P p) {
     }
   }
   __syncthreads();
-  if (tid == 0) {
-    const int64_t rem = p.d - (int64_t)c * CH;
-    uint32_t valid = (uint32_t)(rem < CH ? rem : CH), nz = 0;
-    for (int v = 1; v < 256; v++) nz += s_vh[v];
-    s_vh[0] = valid - nz;
+  if (tid < p.N) p.chunk_sel[(size_t)tid * p.nchunks + c] = s_sel[tid];
+  store_vote_hist_impl(p, c, s_vh);
+}
+
+// per worker: list offset of every chunk = exclusive prefix of the selected counts
+__global__ void __launch_bounds__(1024) k_scan_sel(P p) {
+  __shared__ uint32_t s_w[33];
+  const int n = blockIdx.x;
+  const int per = (p.nchunks + 1023) / 1024;
+  const int c0 = min(p.nchunks, (int)threadIdx.x * per), c1 = min(p.nchunks, c0 + per);
+  const size_t rb = (size_t)n * p.nchunks;
+  uint32_t sum = 0;
+  for (int c = c0; c < c1; c++) sum += p.chunk_sel[rb + c];
+  uint32_t tot;
+  uint32_t run = block_excl_scan<1024>(sum, s_w, tot);
+  for (int c = c0; c < c1; c++) {
+    const uint32_t v = p.chunk_sel[rb + c];
+    p.chunk_sel[rb + c] = run;  // in place: count -> offset
+    run += v;
   }
-  __syncthreads();
-  if (tid <= p.N) {
-    const uint32_t v = s_vh[tid];
-    p.chunk_vh[(size_t)c * (p.N + 1) + tid] = (uint16_t)v;
-    if (v) atomicAdd(&p.vote_hist[tid], v);
+}
+
+// ascending index lists from the bit masks: a warp per (worker, chunk).  In round q lane l owns mask
+// word 32*q + l; its set bits are staged in shared memory in order and copied out coalesced.
+__global__ void __launch_bounds__(TPB) k_lists(P p) {
+  __shared__ uint16_t s_buf[TPB / 32][1024];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n = blockIdx.y;
+  const int c = blockIdx.x * (TPB / 32) + warp;
+  if (c >= p.nchunks) return;
+  const uint32_t next = c + 1 < p.nchunks ? p.chunk_sel[(size_t)n * p.nchunks + c + 1] : (uint32_t)p.K;
+  uint32_t pos = p.chunk_sel[(size_t)n * p.nchunks + c];
+  if (next == pos) return;  // nothing selected in this chunk (warp-uniform)
+  uint32_t m[4];
+#pragma unroll
+  for (int q = 0; q < 4; q++) {
+    const int64_t wi = (int64_t)c * WPC + q * 32 + lane;
+    m[q] = wi < p.W ? __ldcg(p.worker_bits + (size_t)n * p.W + wi) : 0u;
+  }
+  int32_t* lst = p.worker_idx + (size_t)n * p.K;
+  uint16_t* buf = s_buf[warp];
+#pragma unroll
+  for (int q = 0; q < 4; q++) {
+    const uint32_t pc = __popc(m[q]);
+    uint32_t x = pc;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const uint32_t y = __shfl_up_sync(FULL, x, off);
+      if (lane >= off) x += y;
+    }
+    const uint32_t tot = __shfl_sync(FULL, x, 31);
+    uint32_t o = x - pc;
+    uint32_t mm = m[q];
+    while (mm) {
+      const int b = __ffs(mm) - 1;
+      mm &= mm - 1;
+      buf[o++] = (uint16_t)((q * 32 + lane) * 32 + b);
+    }
+    __syncwarp();
+    for (uint32_t t = lane; t < tot; t += 32)
+      if (pos + t < (uint32_t)p.K) lst[pos + t] = c * CH + (int)buf[t];
+    __syncwarp();
+    pos += tot;
   }
 }
 
@@ -942,18 +1013,7 @@ __global__ void __launch_bounds__(TPB) k_vote_hist(P p, const uint8_t* __restric
     }
   }
   __syncthreads();
-  if (tid == 0) {
-    const int64_t rem = p.d - (int64_t)c * CH;
-    uint32_t valid = (uint32_t)(rem < CH ? rem : CH), nz = 0;
-    for (int v = 1; v < 256; v++) nz += s_vh[v];
-    s_vh[0] = valid - nz;
-  }
-  __syncthreads();
-  if (tid <= p.N) {
-    const uint32_t v = s_vh[tid];
-    p.chunk_vh[(size_t)c * (p.N + 1) + tid] = (uint16_t)v;
-    if (v) atomicAdd(&p.vote_hist[tid], v);
-  }
+  store_vote_hist_impl(p, c, s_vh);
 }
 
 // v* = the vote value of the K-th most voted coordinate; then per chunk the output offset and the
@@ -961,10 +1021,13 @@ __global__ void __launch_bounds__(TPB) k_vote_hist(P p, const uint8_t* __restric
 __global__ void __launch_bounds__(1024) k_vote_scan(P p) {
   __shared__ uint32_t s_w[33];
   __shared__ uint32_t s_v[4];
+  __shared__ uint32_t s_h[256];
+  if ((int)threadIdx.x <= p.N) s_h[threadIdx.x] = __ldcg(p.vote_hist + threadIdx.x);
+  __syncthreads();
   if (threadIdx.x == 0) {
     uint32_t acc = 0, vstar = 0, cgt = 0, ceq = 0;
     for (int v = p.N; v >= 0; v--) {
-      const uint32_t h = p.vote_hist[v];
+      const uint32_t h = s_h[v];
       if (acc + h >= (uint32_t)p.K) {
         vstar = (uint32_t)v;
         cgt = acc;
@@ -987,34 +1050,34 @@ __global__ void __launch_bounds__(1024) k_vote_scan(P p) {
   const int stride = p.N + 1;
   const int per = (p.nchunks + 1023) / 1024;
   const int c0 = min(p.nchunks, (int)threadIdx.x * per), c1 = min(p.nchunks, c0 + per);
+  // chunk_vh[c][v] = #{coordinates of chunk c with votes >= v}
   uint32_t esum = 0;
-  for (int c = c0; c < c1; c++) esum += p.chunk_vh[(size_t)c * stride + vstar];
+  for (int c = c0; c < c1; c++) {
+    const uint16_t* h = p.chunk_vh + (size_t)c * stride;
+    const uint32_t gt = (int)vstar < p.N ? h[vstar + 1] : 0u;
+    esum += h[vstar] - gt;
+  }
   uint32_t tot;
   const uint32_t epre = block_excl_scan<1024>(esum, s_w, tot);
   uint32_t run = epre, ssum = 0;
   for (int c = c0; c < c1; c++) {
     const uint16_t* h = p.chunk_vh + (size_t)c * stride;
-    const uint32_t eq = h[vstar];
+    const uint32_t gt = (int)vstar < p.N ? h[vstar + 1] : 0u;
+    const uint32_t eq = h[vstar] - gt;
     const uint32_t take = run >= quota ? 0u : min(eq, quota - run);
-    uint32_t gt = 0;
-    for (int v = (int)vstar + 1; v <= p.N; v++) gt += h[v];
     p.tie_take[c] = take;
     run += eq;
     ssum += gt + take;
   }
   const uint32_t spre = block_excl_scan<1024>(ssum, s_w, tot);
-  run = epre;
   uint32_t srun = spre;
   for (int c = c0; c < c1; c++) {
     const uint16_t* h = p.chunk_vh + (size_t)c * stride;
-    const uint32_t eq = h[vstar];
-    const uint32_t take = run >= quota ? 0u : min(eq, quota - run);
-    uint32_t gt = 0;
-    for (int v = (int)vstar + 1; v <= p.N; v++) gt += h[v];
+    const uint32_t gt = (int)vstar < p.N ? h[vstar + 1] : 0u;
     p.out_base[c] = srun;
-    run += eq;
-    srun += gt + take;
+    srun += gt + p.tie_take[c];
   }
+  if (threadIdx.x == 0) p.out_base[p.nchunks] = (uint32_t)p.K;  // sentinel: end of the last chunk
 }
 
 // writes supp(M) (ascending) and optionally M as a bit mask
@@ -1026,6 +1089,13 @@ __global__ void __launch_bounds__(TPB) k_vote_write(P p, const uint8_t* __restri
   const uint32_t take = p.tie_take[c];
   const uint32_t ob = p.out_base[c];
   const int64_t jb = (int64_t)c * CH + (int64_t)tid * 16;
+  if (p.out_base[c + 1] == ob) {  // no coordinate of this chunk is in the mask (uniform over the CTA)
+    if (mask_bits != nullptr && (tid & 1) == 0) {
+      const int64_t wi = (int64_t)c * WPC + (tid >> 1);
+      if (wi < p.W) mask_bits[wi] = 0u;
+    }
+    return;
+  }
   uint32_t gm = 0, em = 0;
   if (jb < p.d) {
     if (jb + 16 <= p.d) {
@@ -1119,8 +1189,8 @@ struct Layout {
   int64_t W;
   uint32_t cap;
   size_t zero_bytes;  // the leading region cleared at the start of every vote
-  size_t samp_hist, hist1, hist2, hist3, cand_cnt, vote_hist;
-  size_t tau, wstate, thresh, vstate, cand, chunk_base, chunk_cnt, chunk_gt, chunk_eq, tie_base, sel_base;
+  size_t samp_hist, hist1, hist2, hist3, cand_cnt, sample_done, vote_hist;
+  size_t tau, wstate, thresh, vstate, cand, chunk_base, chunk_cnt, chunk_gt, chunk_eq, tie_base, sel_base, chunk_sel;
   size_t worker_bits, worker_idx, votes, chunk_vh, out_base, tie_take;
   size_t total;
 };
@@ -1139,8 +1209,9 @@ Layout make_layout(int N, int64_t d, int64_t K) {
   Layout L;
   L.nchunks = (int)((d + CH - 1) / CH);
   L.W = (d + 31) / 32;
-  const int64_t cap = 4 * K + 4096;
-  L.cap = (uint32_t)(cap < d ? cap : d);
+  int64_t cap = 4 * K + 4096;
+  if (cap > d) cap = d;
+  L.cap = (uint32_t)((cap + 7) & ~(int64_t)7);  // multiple of 8: every worker's buffer is 64-byte aligned
   size_t off = 0;
   const size_t n = (size_t)N, nc = (size_t)L.nchunks;
   L.samp_hist = take(off, n * SB_BINS * 4);
@@ -1148,6 +1219,7 @@ Layout make_layout(int N, int64_t d, int64_t K) {
   L.hist2 = take(off, n * H2_BINS * 4);
   L.hist3 = take(off, n * H3_BINS * 4);
   L.cand_cnt = take(off, n * 4);
+  L.sample_done = take(off, n * 4);
   L.vote_hist = take(off, 256 * 4);
   L.zero_bytes = off;
   L.tau = take(off, n * 4);
@@ -1161,11 +1233,12 @@ Layout make_layout(int N, int64_t d, int64_t K) {
   L.chunk_eq = take(off, n * nc * 4);
   L.tie_base = take(off, n * nc * 4);
   L.sel_base = take(off, n * nc * 4);
+  L.chunk_sel = take(off, n * nc * 4);
   L.worker_bits = take(off, n * (size_t)L.W * 4);
   L.worker_idx = take(off, n * (size_t)K * 4);
   L.votes = take(off, nc * CH);
   L.chunk_vh = take(off, nc * (n + 1) * 2);
-  L.out_base = take(off, nc * 4);
+  L.out_base = take(off, (nc + 1) * 4);
   L.tie_take = take(off, nc * 4);
   L.total = off;
   return L;
@@ -1208,6 +1281,7 @@ P make_params(const mv_ctx* ctx, const Layout& L, int N, int64_t d, int64_t K) {
   p.hist2 = (uint32_t*)(b + L.hist2);
   p.hist3 = (uint32_t*)(b + L.hist3);
   p.cand_cnt = (uint32_t*)(b + L.cand_cnt);
+  p.sample_done = (uint32_t*)(b + L.sample_done);
   p.vote_hist = (uint32_t*)(b + L.vote_hist);
   p.tau = (uint32_t*)(b + L.tau);
   p.wstate = (uint32_t*)(b + L.wstate);
@@ -1220,6 +1294,7 @@ P make_params(const mv_ctx* ctx, const Layout& L, int N, int64_t d, int64_t K) {
   p.chunk_eq = (uint32_t*)(b + L.chunk_eq);
   p.tie_base = (uint32_t*)(b + L.tie_base);
   p.sel_base = (uint32_t*)(b + L.sel_base);
+  p.chunk_sel = (uint32_t*)(b + L.chunk_sel);
   p.worker_bits = (uint32_t*)(b + L.worker_bits);
   p.worker_idx = (int32_t*)(b + L.worker_idx);
   p.votes = (uint8_t*)(b + L.votes);
@@ -1256,7 +1331,7 @@ void sample_plan(int64_t d, int64_t K, uint32_t& U, uint32_t& L, int& all, uint3
   }
   all = 0;
   U = (uint32_t)(S / 32);
-  L = (uint32_t)(d / 32);
+  L = (uint32_t)((d / 32) / U);  // line stride (>= 2): lines 0, L, 2L, ... are sampled
   const double Sn = (double)U * 32.0;
   const double m = Sn * (double)K / (double)d;
   double r = ceil(m + 6.0 * sqrt(m) + 8.0);
@@ -1269,49 +1344,47 @@ int vote_impl(mv_ctx* ctx, P p, const Layout& L, const float* grads, float* err)
   cudaStream_t st = ctx->stream;
   const int N = p.N;
   if (cudaMemsetAsync(ctx->ws, 0, L.zero_bytes, st) != cudaSuccess) return MV_ERR_CUDA;
-  const int gg = per_row_ctas(N, p.nchunks, 148 * 8);
+  // CTAs per worker of the select kernels: enough for a full-row pass, not more than the candidates need
+  const int gh = per_row_ctas(N, p.force_general ? p.nchunks : (int)((p.cap + TPB * 4 - 1) / (TPB * 4)), 148 * 8);
   if (!p.force_general) {
     uint32_t U, Ls, rank;
     int all;
     sample_plan(p.d, p.K, U, Ls, all, rank);
-    const int gs = per_row_ctas(N, (int)((U + 63) / 64), 148 * 2);
-    k_sample_hist<<<dim3(gs, N), 512, 0, st>>>(p, grads, err, U, Ls, all);
-    MV_LAUNCH_CHECK();
-    k_sample_pick<<<N, TPB, 0, st>>>(p, rank);
+    const int gs = per_row_ctas(N, (int)((U + 63) / 64), 148 * 4);
+    k_sample_hist<<<dim3(gs, N), 512, 0, st>>>(p, grads, err, U, Ls, all, rank);
     MV_LAUNCH_CHECK();
     if (ctx->timing) cudaEventRecord(ctx->ev[2 * (ctx->timed % 64)], st);
     k_acc_compact<<<dim3(p.nchunks, N), TPB, 0, st>>>(p, grads, err);
     MV_LAUNCH_CHECK();
     if (ctx->timing) cudaEventRecord(ctx->ev[2 * (ctx->timed++ % 64) + 1], st);
-    const int gc = per_row_ctas(N, (int)((p.cap + TPB * 16 - 1) / (TPB * 16)), 148 * 4);
-    k_cand_hist<1><<<dim3(gc, N), TPB, 0, st>>>(p);
-    MV_LAUNCH_CHECK();
-    k_cand_hist<2><<<dim3(gc, N), TPB, 0, st>>>(p);
-    MV_LAUNCH_CHECK();
-    k_cand_hist<3><<<dim3(gc, N), TPB, 0, st>>>(p);
-    MV_LAUNCH_CHECK();
-    const int g4 = per_row_ctas(N, (p.nchunks + 31) / 32, 148 * 4);
-    k_cand_count<<<dim3(g4, N), TPB, 0, st>>>(p);
-    MV_LAUNCH_CHECK();
-    k_row_hist<1, false><<<dim3(gg, N), TPB, 0, st>>>(p, nullptr, err);
+    k_hist<1, false><<<dim3(gh, N), TPB, 0, st>>>(p, nullptr, err);
     MV_LAUNCH_CHECK();
   } else {
     if (ctx->timing) cudaEventRecord(ctx->ev[2 * (ctx->timed % 64)], st);
-    k_row_hist<1, true><<<dim3(gg, N), TPB, 0, st>>>(p, grads, err);
+    k_hist<1, true><<<dim3(gh, N), TPB, 0, st>>>(p, grads, err);
     MV_LAUNCH_CHECK();
     if (ctx->timing) cudaEventRecord(ctx->ev[2 * (ctx->timed++ % 64) + 1], st);
   }
-  k_row_hist<2, false><<<dim3(gg, N), TPB, 0, st>>>(p, nullptr, err);
+  k_hist<2, false><<<dim3(gh, N), TPB, 0, st>>>(p, nullptr, err);
   MV_LAUNCH_CHECK();
-  k_row_hist<3, false><<<dim3(gg, N), TPB, 0, st>>>(p, nullptr, err);
+  k_hist<3, false><<<dim3(gh, N), TPB, 0, st>>>(p, nullptr, err);
   MV_LAUNCH_CHECK();
-  k_row_count<<<dim3(gg, N), TPB, 0, st>>>(p, err);
+  k_count<<<dim3(gh, N), TPB, 0, st>>>(p, err);
   MV_LAUNCH_CHECK();
   k_chunk_scan<<<N, 1024, 0, st>>>(p);
   MV_LAUNCH_CHECK();
-  k_row_exact<<<dim3(gg, N), TPB, 0, st>>>(p, err);
+  k_row_exact<<<dim3(gh, N), TPB, 0, st>>>(p, err);
   MV_LAUNCH_CHECK();
-  k_build_votes<<<p.nchunks, TPB, 0, st>>>(p);
+  const int gb = per_row_ctas(N, (int)((p.cap + TPB * 8 - 1) / (TPB * 8)), 148 * 8);
+  k_set_bits<<<dim3(gb, N), TPB, 0, st>>>(p);
+  MV_LAUNCH_CHECK();
+  k_tie_bits<<<dim3(per_row_ctas(N, (p.nchunks + 7) / 8, 148 * 4), N), TPB, 0, st>>>(p);
+  MV_LAUNCH_CHECK();
+  k_votes<<<p.nchunks, TPB, 0, st>>>(p);
+  MV_LAUNCH_CHECK();
+  k_scan_sel<<<N, 1024, 0, st>>>(p);
+  MV_LAUNCH_CHECK();
+  k_lists<<<dim3((p.nchunks + TPB / 32 - 1) / (TPB / 32), N), TPB, 0, st>>>(p);
   MV_LAUNCH_CHECK();
   return MV_OK;
 }
