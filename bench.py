@@ -253,7 +253,8 @@ def main():
     for _ in range(args.warmup):
         ctx.mv_sparse_step(pool[step_no % pool_n], err, out_idx, out_val)
         step_no += 1
-    ctx.set_kernel_timing(True)
+    # CUDA events around the streaming kernel on one step in eight (each pair costs a few microseconds)
+    ctx.set_kernel_timing(8 if args.steps >= 8 else 1)
     sampler.wait_for_first_sample()
     barrier()
     first_row = sampler.rows_so_far()
@@ -269,7 +270,7 @@ def main():
     ms_total = ev0.elapsed_time(ev1)
     launches_per_step = ctx.last_launches()
     k_ms, k_cnt = ctx.read_kernel_timing()
-    ctx.set_kernel_timing(False)
+    ctx.set_kernel_timing(0)
     diag = ctx.read_diag(w.N)
     t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
     if dist is not None:

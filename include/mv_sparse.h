@@ -119,13 +119,23 @@ int mv_sparse_step_host(mv_ctx* ctx, const float* h_grads, int N, int64_t d, int
 int mv_read_diag(mv_ctx* ctx, int N, uint32_t* per_worker);
 
 /* Optional timing of the streaming pass (the kernel that reads grads and err and writes acc,
- * i.e. the accumulate line of Algorithm 1 fused with the candidate filter of S_top): while
- * enabled, every mv_vote / mv_sparse_step records a CUDA-event pair around that one kernel on
- * the context's stream.  mv_read_kernel_timing waits for the stream, returns the summed
- * duration in milliseconds and the number of launches it covers (at most the last 64), and
- * restarts the count.  Enabling creates the events once; nothing is recorded while disabled. */
-int mv_set_kernel_timing(mv_ctx* ctx, int enable);
+ * i.e. the accumulate line of Algorithm 1 fused with the candidate filter of S_top): with
+ * every = n >= 1, each n-th mv_vote / mv_sparse_step records a CUDA-event pair around that one
+ * kernel on the context's stream (a pair costs a few microseconds of stream time); every = 0
+ * switches it off.  mv_read_kernel_timing waits for the stream, returns the summed duration in
+ * milliseconds and the number of launches it covers (at most the last 64), and restarts the
+ * count.  The first enabling call creates the events. */
+int mv_set_kernel_timing(mv_ctx* ctx, int every);
 int mv_read_kernel_timing(mv_ctx* ctx, float* total_ms, int* launches);
+
+/* Optional per-launch timing of a whole call, for profiling without an external tool: while
+ * enabled, a CUDA event is recorded before the first and after every kernel launch of each call
+ * (the events themselves cost a little time).  mv_read_phase_times waits for the stream and
+ * returns, for the last call, the elapsed milliseconds between consecutive events: ms[i] covers
+ * the i-th kernel in launch order (Algorithm 1's steps in the order listed at the top of this
+ * file).  At most `capacity` values (and at most 47) are written; *count gets their number. */
+int mv_set_phase_timing(mv_ctx* ctx, int enable);
+int mv_read_phase_times(mv_ctx* ctx, float* ms, int capacity, int* count);
 
 /* Number of kernels the last call on this context enqueued. */
 int mv_last_launches(const mv_ctx* ctx);

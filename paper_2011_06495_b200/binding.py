@@ -67,6 +67,10 @@ def load() -> ctypes.CDLL:
     lib.mv_set_kernel_timing.argtypes = [c_vp, c_i]
     lib.mv_read_kernel_timing.restype = c_i
     lib.mv_read_kernel_timing.argtypes = [c_vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(c_i)]
+    lib.mv_set_phase_timing.restype = c_i
+    lib.mv_set_phase_timing.argtypes = [c_vp, c_i]
+    lib.mv_read_phase_times.restype = c_i
+    lib.mv_read_phase_times.argtypes = [c_vp, ctypes.POINTER(ctypes.c_float), c_i, ctypes.POINTER(c_i)]
     lib.mv_last_launches.restype = c_i
     lib.mv_last_launches.argtypes = [c_vp]
     lib.mv_status_string.restype = ctypes.c_char_p
@@ -159,8 +163,9 @@ class MvContext:
         out.copy_(torch.tensor(list(buf), dtype=torch.int64).view(N, 4))
         return out
 
-    def set_kernel_timing(self, enable: bool):
-        _check(self.lib.mv_set_kernel_timing(self.handle, int(bool(enable))), "mv_set_kernel_timing")
+    def set_kernel_timing(self, every: int):
+        """0: off; n >= 1: time the streaming pass on every n-th step."""
+        _check(self.lib.mv_set_kernel_timing(self.handle, int(every)), "mv_set_kernel_timing")
 
     def read_kernel_timing(self):
         """(total milliseconds, launches covered) of the streaming pass since the last read."""
@@ -168,6 +173,16 @@ class MvContext:
         _check(self.lib.mv_read_kernel_timing(self.handle, ctypes.byref(ms), ctypes.byref(cnt)),
                "mv_read_kernel_timing")
         return float(ms.value), int(cnt.value)
+
+    def set_phase_timing(self, enable: bool):
+        _check(self.lib.mv_set_phase_timing(self.handle, int(bool(enable))), "mv_set_phase_timing")
+
+    def read_phase_times(self):
+        """Milliseconds per kernel launch of the last call, in launch order."""
+        buf = (ctypes.c_float * 47)()
+        cnt = ctypes.c_int()
+        _check(self.lib.mv_read_phase_times(self.handle, buf, 47, ctypes.byref(cnt)), "mv_read_phase_times")
+        return [float(buf[i]) for i in range(cnt.value)]
 
     def last_launches(self) -> int:
         return int(self.lib.mv_last_launches(self.handle))

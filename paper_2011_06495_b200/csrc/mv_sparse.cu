@@ -9,11 +9,12 @@
 //                                             place, elements with key >= tau_n compacted per chunk
 //   select     k_hist<1..3>, k_count          exact K-th key T_n by radix select: on the candidates, or over
 //                                             the full row for a worker whose candidate count missed [K, cap]
-//   order      k_chunk_scan, k_row_exact      lowest-index tie quota per chunk; exact compaction for the
+//   order      (tail of k_count), k_row_exact lowest-index tie quota per chunk; exact compaction for the
 //                                             full-row workers
-//   vote       k_set_bits, k_tie_bits, k_votes  per-worker bit masks, bit-sliced vote count
-//   lists      k_scan_sel, k_lists            ascending per-worker index lists from the masks
-//   mask       k_vote_hist, k_vote_scan, k_vote_write   counting select over vote values 0..N
+//   vote       k_set_bits, k_votes            per-worker bit masks, bit-sliced vote count
+//   lists      k_scan_sel, k_lists            ascending per-worker index lists from the masks (side stream)
+//   mask       (tail of k_votes), k_vote_write  counting select over vote values 0..N (k_vote_hist when
+//                                             votes come from the caller)
 //   aggregate  k_gather                       mean on the shared mask, residual zeroed in place
 //
 // The magnitude order is the order of key(x) = bits(x) & 0x7fffffff; ties go to the lowest index.
@@ -40,6 +41,7 @@ constexpr unsigned FULL = 0xffffffffu;
 struct P {
   int N;
   int nchunks;
+  int nc_pad;             // nchunks rounded up to a multiple of 8 (row pitch of chunk_vh)
   uint32_t cap;           // candidate slots per worker
   int force_general;
   int64_t d;
@@ -50,7 +52,10 @@ struct P {
   uint32_t* hist2;        // [N][H2_BINS]
   uint32_t* hist3;        // [N][H3_BINS]
   uint32_t* cand_cnt;     // [N]
-  uint32_t* sample_done;  // [N] ticket counters
+  uint32_t* sample_done;  // [N] ticket counters (last CTA of a worker finishes the job)
+  uint32_t* count_done;   // [N]
+  uint32_t* votes_done;   // [1]
+  uint8_t* hot;           // [nc_pad] 1 if any worker kept a candidate in the chunk
   uint32_t* vote_hist;    // [256]
   uint32_t* tau;          // [N]
   uint32_t* wstate;       // [N][8]: b1, rem1, b2, rem2, T, cnt_gt, cnt_eq, need
@@ -67,10 +72,19 @@ struct P {
   uint32_t* worker_bits;  // [N][W]
   int32_t* worker_idx;    // [N][K]
   uint8_t* votes;         // [d]
-  uint16_t* chunk_vh;     // [nchunks][N+1]
+  uint16_t* chunk_vh;     // [N+1][nc_pad]: chunk_vh[v][c] = #{coordinates of chunk c with votes >= v}
   uint32_t* out_base;     // [nchunks]
   uint32_t* tie_take;     // [nchunks]
 };
+
+// Programmatic dependent launch: every kernel first waits for the kernel before it on the stream
+// to finish (all of its memory operations visible), then lets the kernel after it be scheduled.
+// Launch latency of kernel k+1 is thereby hidden behind the execution of kernel k; the order of
+// execution and the memory semantics are those of plain stream order.
+__device__ __forceinline__ void pdl_enter() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
 
 __device__ __forceinline__ uint32_t fkey(float x) { return __float_as_uint(x) & 0x7fffffffu; }
 
@@ -300,6 +314,7 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* s_w /*
 __global__ void __launch_bounds__(512) k_sample_hist(P p, const float* __restrict__ grads,
                                                      const float* __restrict__ err, uint32_t U, uint32_t L, int all,
                                                      uint32_t rank) {
+  pdl_enter();
   __shared__ uint32_t sh[SB_BINS];
   __shared__ uint32_t s_last;
   const int n = blockIdx.y;
@@ -307,11 +322,11 @@ __global__ void __launch_bounds__(512) k_sample_hist(P p, const float* __restric
   __syncthreads();
   const size_t r0 = (size_t)n * (size_t)p.d;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (uint32_t u0 = (blockIdx.x * 16u + warp) * 4u; u0 < U; u0 += gridDim.x * 64u) {
-    float a[4];
-    bool ok[4];
+  for (uint32_t u0 = (blockIdx.x * 16u + warp) * 8u; u0 < U; u0 += gridDim.x * 128u) {
+    float a[8];
+    bool ok[8];
 #pragma unroll
-    for (int q = 0; q < 4; q++) {
+    for (int q = 0; q < 8; q++) {  // sixteen loads in flight per lane
       const uint32_t u = u0 + q;
       ok[q] = false;
       a[q] = 0.f;
@@ -320,12 +335,12 @@ __global__ void __launch_bounds__(512) k_sample_hist(P p, const float* __restric
         const int64_t j = (int64_t)line * 32 + lane;
         if (j < p.d) {
           ok[q] = true;
-          a[q] = __fadd_rn(err[r0 + j], grads[r0 + j]);
+          a[q] = __fadd_rn(__ldcs(err + r0 + j), __ldcs(grads + r0 + j));
         }
       }
     }
 #pragma unroll
-    for (int q = 0; q < 4; q++)
+    for (int q = 0; q < 8; q++)
       if (ok[q]) atomicAdd(&sh[fkey(a[q]) >> SB_SHIFT], 1u);
   }
   __syncthreads();
@@ -350,6 +365,7 @@ __global__ void __launch_bounds__(512) k_sample_hist(P p, const float* __restric
 // chunk's own run of the worker's candidate buffer (one global atomic per chunk that has any)
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(TPB) k_acc_compact(P p, const float* __restrict__ grads, float* __restrict__ err) {
+  pdl_enter();
   __shared__ uint32_t s_w[9];
   __shared__ uint32_t s_base, s_total;
   const int n = blockIdx.y, c = blockIdx.x;
@@ -382,7 +398,10 @@ __global__ void __launch_bounds__(TPB) k_acc_compact(P p, const float* __restric
     uint32_t total = 0;
     for (int w = 0; w < 9; w++) total += s_w[w];
     uint32_t base = 0;
-    if (total) base = atomicAdd(&p.cand_cnt[n], total);
+    if (total) {
+      base = atomicAdd(&p.cand_cnt[n], total);
+      p.hot[c] = 1;  // same value from every worker: a plain store is enough
+    }
     p.chunk_base[(size_t)n * p.nchunks + c] = base;
     p.chunk_cnt[(size_t)n * p.nchunks + c] = total;
     s_base = base;
@@ -501,6 +520,7 @@ __device__ __forceinline__ uint32_t* hist_of(const P& p, int n) {
 // and counts every element: the first pass when sampling is switched off.
 template <int PASS, bool FUSED>
 __global__ void __launch_bounds__(TPB) k_hist(P p, const float* __restrict__ grads, float* __restrict__ err) {
+  pdl_enter();
   constexpr int NB = PASS == 1 ? H1_BINS : H2_BINS;
   __shared__ uint32_t sh[NB];
   const int n = blockIdx.y;
@@ -557,12 +577,49 @@ __global__ void __launch_bounds__(TPB) k_hist(P p, const float* __restrict__ gra
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// order: per worker, running count of threshold ties before each chunk (tie_base) and of selected
+// elements before each chunk (sel_base), given the quota `need` of ties to keep, lowest index first
+// ---------------------------------------------------------------------------------------------
+template <int NT>
+__device__ void chunk_scan(const P& p, int n, uint32_t need, bool fast) {
+  __shared__ uint32_t s_w[NT / 32 + 1];
+  const int per = (p.nchunks + NT - 1) / NT;
+  const int c0 = min(p.nchunks, (int)threadIdx.x * per), c1 = min(p.nchunks, c0 + per);
+  const size_t rb = (size_t)n * p.nchunks;
+  uint32_t esum = 0;
+  for (int c = c0; c < c1; c++) esum += __ldcg(p.chunk_eq + rb + c);
+  uint32_t tot;
+  const uint32_t epre = block_excl_scan<NT>(esum, s_w, tot);
+  uint32_t run = epre, ssum = 0;
+  for (int c = c0; c < c1; c++) {
+    const uint32_t eq = __ldcg(p.chunk_eq + rb + c);
+    const uint32_t take = run >= need ? 0u : min(eq, need - run);
+    p.tie_base[rb + c] = run;
+    run += eq;
+    if (!fast) ssum += __ldcg(p.chunk_gt + rb + c) + take;
+  }
+  if (fast) return;  // a fast worker only needs tie_base (uniform over the CTA)
+  const uint32_t spre = block_excl_scan<NT>(ssum, s_w, tot);
+  run = epre;
+  uint32_t srun = spre;
+  for (int c = c0; c < c1; c++) {
+    const uint32_t eq = __ldcg(p.chunk_eq + rb + c);
+    const uint32_t take = run >= need ? 0u : min(eq, need - run);
+    p.sel_base[rb + c] = srun;
+    run += eq;
+    srun += __ldcg(p.chunk_gt + rb + c) + take;
+  }
+}
+
 // Resolves T_n for every worker, then counts per chunk what the ordering needs:
 //   - a fast worker that keeps all of its threshold ties needs nothing here;
 //   - a fast worker that keeps only some of them needs the ties per chunk (from its candidates);
 //   - any other worker needs, from its full row, the elements above and at the threshold per chunk.
 __global__ void __launch_bounds__(TPB) k_count(P p, float* __restrict__ err) {
+  pdl_enter();
   __shared__ uint32_t s_g[TPB / 32], s_e[TPB / 32];
+  __shared__ uint32_t s_last;
   const int n = blockIdx.y;
   uint32_t need, cnt_eq;
   const uint32_t T = resolve_threshold(p, n, need, cnt_eq);
@@ -578,8 +635,7 @@ __global__ void __launch_bounds__(TPB) k_count(P p, float* __restrict__ err) {
       eq = __reduce_add_sync(FULL, eq);
       if (lane == 0) p.chunk_eq[ci] = eq;
     }
-    return;
-  }
+  } else {
   for (int c = blockIdx.x; c < p.nchunks; c += gridDim.x) {
     const Geom g = chunk_geom(n, c, p.d);
     uint32_t key[4][4], vm[4];
@@ -614,11 +670,21 @@ __global__ void __launch_bounds__(TPB) k_count(P p, float* __restrict__ err) {
       p.chunk_eq[(size_t)n * p.nchunks + c] = te;
     }
   }
+  }
+  // the last CTA of this worker to get here turns the per-chunk counts into running offsets
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) s_last = (atomicAdd(&p.count_done[n], 1u) == gridDim.x - 1) ? 1u : 0u;
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  chunk_scan<TPB>(p, n, need, worker_fast(p, n));
 }
 
 // exact compaction: writes precisely the selected elements of each chunk, in index order, at the
 // chunk's list offset (so the candidate buffer of such a worker holds its K picks, sorted)
 __global__ void __launch_bounds__(TPB) k_row_exact(P p, float* __restrict__ err) {
+  pdl_enter();
   __shared__ uint32_t s_we[9], s_ws[9];
   const int n = blockIdx.y;
   if (worker_fast(p, n)) return;
@@ -721,67 +787,120 @@ __global__ void __launch_bounds__(TPB) k_row_exact(P p, float* __restrict__ err)
       for (int w = 0; w < 9; w++) tot += s_ws[w];
       p.chunk_base[ci] = sb;
       p.chunk_cnt[ci] = tot;
+      if (tot) p.hot[c] = 1;
     }
   }
 }
 
-// ---------------------------------------------------------------------------------------------
-// order: per worker, running count of threshold ties before each chunk (tie_base) and of selected
-// elements before each chunk (sel_base), given the quota `need` of ties to keep, lowest index first
-// ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024) k_chunk_scan(P p) {
-  __shared__ uint32_t s_w[33];
-  const int n = blockIdx.x;
-  const uint32_t need = p.wstate[(size_t)n * 8 + 7];
-  const bool fast = worker_fast(p, n);
-  if (fast && need >= p.wstate[(size_t)n * 8 + 6]) return;  // keeps every tie: nothing to order
-  const int per = (p.nchunks + 1023) / 1024;
-  const int c0 = min(p.nchunks, (int)threadIdx.x * per), c1 = min(p.nchunks, c0 + per);
-  const size_t rb = (size_t)n * p.nchunks;
-  uint32_t esum = 0;
-  for (int c = c0; c < c1; c++) esum += p.chunk_eq[rb + c];
+// v* = the vote value of the K-th most voted coordinate; then per chunk the output offset and the
+// number of v*-ties it may keep (lowest index first).  Run by the last CTA that finished the
+// per-chunk vote histograms; all NT threads of that CTA call it.
+template <int NT>
+__device__ void vote_scan(const P& p) {
+  __shared__ uint32_t s_w[NT / 32 + 1];
+  __shared__ uint32_t s_v[4];
+  __shared__ uint32_t s_h[256];
+  for (int v = threadIdx.x; v <= p.N; v += NT) s_h[v] = v ? __ldcg(p.vote_hist + v) : 0u;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    uint32_t voted = 0;
+    for (int v = 1; v <= p.N; v++) voted += s_h[v];
+    s_h[0] = (uint32_t)p.d - voted;  // coordinates nobody voted for
+    uint32_t acc = 0, vstar = 0, cgt = 0, ceq = 0;
+    for (int v = p.N; v >= 0; v--) {
+      const uint32_t h = s_h[v];
+      if (acc + h >= (uint32_t)p.K) {
+        vstar = (uint32_t)v;
+        cgt = acc;
+        ceq = h;
+        break;
+      }
+      acc += h;
+    }
+    s_v[0] = vstar;
+    s_v[3] = (uint32_t)p.K - cgt;
+    p.vstate[0] = vstar;
+    p.vstate[1] = cgt;
+    p.vstate[2] = ceq;
+    p.vstate[3] = (uint32_t)p.K - cgt;
+  }
+  __syncthreads();
+  const uint32_t vstar = s_v[0], quota = s_v[3];
+  // each thread owns `per` consecutive chunks (a multiple of 8, so its counts are whole 16-byte loads)
+  const int per = (((p.nchunks + NT - 1) / NT) + 7) & ~7;
+  const int c0 = min(p.nc_pad, (int)threadIdx.x * per), c1 = min(p.nc_pad, c0 + per);
+  const uint16_t* hge = p.chunk_vh + (size_t)vstar * p.nc_pad;                                   // votes >= v*
+  const uint16_t* hgt = (int)vstar < p.N ? p.chunk_vh + (size_t)(vstar + 1) * p.nc_pad : nullptr;  // votes > v*
+  uint32_t esum = 0, gsum = 0;
+  for (int c = c0; c < c1; c += 8) {
+    const uint4 a = __ldcg(reinterpret_cast<const uint4*>(hge + c));
+    const uint4 g = hgt ? __ldcg(reinterpret_cast<const uint4*>(hgt + c)) : make_uint4(0, 0, 0, 0);
+    const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, gw[4] = {g.x, g.y, g.z, g.w};
+#pragma unroll
+    for (int q = 0; q < 8; q++) {
+      if (c + q < p.nchunks) {
+        const uint32_t ge = (aw[q >> 1] >> (16 * (q & 1))) & 0xffffu, gt = (gw[q >> 1] >> (16 * (q & 1))) & 0xffffu;
+        esum += ge - gt;
+        gsum += gt;
+      }
+    }
+  }
   uint32_t tot;
-  const uint32_t epre = block_excl_scan<1024>(esum, s_w, tot);
-  uint32_t run = epre, ssum = 0;
-  for (int c = c0; c < c1; c++) {
-    const uint32_t eq = p.chunk_eq[rb + c];
-    const uint32_t take = run >= need ? 0u : min(eq, need - run);
-    p.tie_base[rb + c] = run;
-    run += eq;
-    if (!fast) ssum += p.chunk_gt[rb + c] + take;
+  const uint32_t epre = block_excl_scan<NT>(esum, s_w, tot);
+  const uint32_t taken_before = epre < quota ? epre : quota;              // ties kept in earlier chunks
+  const uint32_t taken_here = min(epre + esum, quota) - taken_before;     // ties kept in this thread's chunks
+  const uint32_t spre = block_excl_scan<NT>(gsum + taken_here, s_w, tot);
+  uint32_t run = epre, srun = spre;
+  for (int c = c0; c < c1; c += 8) {
+    const uint4 a = __ldcg(reinterpret_cast<const uint4*>(hge + c));
+    const uint4 g = hgt ? __ldcg(reinterpret_cast<const uint4*>(hgt + c)) : make_uint4(0, 0, 0, 0);
+    const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, gw[4] = {g.x, g.y, g.z, g.w};
+#pragma unroll
+    for (int q = 0; q < 8; q++) {
+      if (c + q < p.nchunks) {
+        const uint32_t ge = (aw[q >> 1] >> (16 * (q & 1))) & 0xffffu, gt = (gw[q >> 1] >> (16 * (q & 1))) & 0xffffu;
+        const uint32_t eq = ge - gt;
+        const uint32_t take = run >= quota ? 0u : min(eq, quota - run);
+        p.tie_take[c + q] = take;
+        p.out_base[c + q] = srun;
+        run += eq;
+        srun += gt + take;
+      }
+    }
   }
-  if (fast) return;  // a fast worker only needs tie_base (uniform over the CTA)
-  const uint32_t spre = block_excl_scan<1024>(ssum, s_w, tot);
-  run = epre;
-  uint32_t srun = spre;
-  for (int c = c0; c < c1; c++) {
-    const uint32_t eq = p.chunk_eq[rb + c];
-    const uint32_t take = run >= need ? 0u : min(eq, need - run);
-    p.sel_base[rb + c] = srun;
-    run += eq;
-    srun += p.chunk_gt[rb + c] + take;
-  }
+  if (threadIdx.x == 0) p.out_base[p.nchunks] = (uint32_t)p.K;  // sentinel: end of the last chunk
+}
+
+// ticket: true in every thread of the last CTA of the grid to call it (all threads must call)
+__device__ __forceinline__ bool last_cta(uint32_t* counter, uint32_t total) {
+  __shared__ uint32_t s_last_flag;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) s_last_flag = (atomicAdd(counter, 1u) == total - 1) ? 1u : 0u;
+  __syncthreads();
+  const bool last = s_last_flag != 0;
+  if (last) __threadfence();
+  return last;
 }
 
 // s_vh[v] (v >= 1) holds how many coordinates of chunk c got exactly v votes.  Stores, per chunk,
 // the cumulative counts cum[v] = #{votes >= v} (v = 0..N) and adds the exact counts to the global
-// histogram.  All TPB threads call it.
+// histogram.  All threads of the CTA call it.
 __device__ __forceinline__ void store_vote_hist_impl(const P& p, int c, uint32_t* s_vh) {
-  const int tid = threadIdx.x;
-  if (tid <= p.N) {
+  for (int t = threadIdx.x; t <= p.N; t += blockDim.x) {
     const int64_t rem = p.d - (int64_t)c * CH;
     const uint32_t valid = (uint32_t)(rem < CH ? rem : CH);
-    uint32_t ge = 0;  // coordinates with votes >= max(tid, 1)
-    for (int v = max(tid, 1); v <= p.N; v++) ge += s_vh[v];
+    uint32_t ge = 0;  // coordinates with votes >= max(t, 1)
+    for (int v = max(t, 1); v <= p.N; v++) ge += s_vh[v];
     uint32_t exact;
-    if (tid == 0) {
+    if (t == 0) {
       exact = valid - ge;
       ge = valid;
     } else {
-      exact = s_vh[tid];
+      exact = s_vh[t];
     }
-    p.chunk_vh[(size_t)c * (p.N + 1) + tid] = (uint16_t)ge;
-    if (exact) atomicAdd(&p.vote_hist[tid], exact);
+    p.chunk_vh[(size_t)t * p.nc_pad + c] = (uint16_t)ge;
+    if (exact && t > 0) atomicAdd(&p.vote_hist[t], exact);  // the zero-vote count is derived later
   }
 }
 
@@ -794,11 +913,12 @@ __device__ __forceinline__ void store_vote_hist_impl(const P& p, int c, uint32_t
 // the N masks bit-sliced (8 counter planes per 32-coordinate word) into the vote count.
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(TPB) k_set_bits(P p) {
+  pdl_enter();
   const int n = blockIdx.y;
   const bool fast = worker_fast(p, n);
   const uint32_t* ws = p.wstate + (size_t)n * 8;
-  const uint32_t T = ws[4];
-  const bool all_ties = ws[7] >= ws[6];
+  const uint32_t T = ws[4], need = ws[7];
+  const bool all_ties = need >= ws[6];
   const uint32_t cnt = fast ? p.cand_cnt[n] : (uint32_t)p.K;  // a full-row worker's buffer holds exactly its picks
   const uint2* cd = p.cand + (size_t)n * p.cap;               // cap is a multiple of 8: rows are 64-byte aligned
   uint32_t* bits_row = p.worker_bits + (size_t)n * p.W;
@@ -824,28 +944,22 @@ __global__ void __launch_bounds__(TPB) k_set_bits(P p) {
     }
     if (acc) atomicOr(bits_row + curw, acc);
   }
-}
-
-__global__ void __launch_bounds__(TPB) k_tie_bits(P p) {
-  const int n = blockIdx.y;
-  const uint32_t* ws = p.wstate + (size_t)n * 8;
-  const uint32_t T = ws[4], need = ws[7];
-  if (!worker_fast(p, n) || need >= ws[6]) return;
+  // a worker that keeps only part of its threshold ties adds them chunk by chunk, lowest index first
+  if (!fast || all_ties) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t lt = lanemask_lt();
-  uint32_t* bits_row = p.worker_bits + (size_t)n * p.W;
   for (int c = blockIdx.x * (TPB / 32) + warp; c < p.nchunks; c += gridDim.x * (TPB / 32)) {
     const size_t ci = (size_t)n * p.nchunks + c;
-    const uint32_t cnt = p.chunk_cnt[ci];
+    const uint32_t ccnt = p.chunk_cnt[ci];
     uint32_t run = p.tie_base[ci];
-    if (cnt == 0 || run >= need) continue;
-    const uint2* cd = p.cand + (size_t)n * p.cap + p.chunk_base[ci];
-    for (uint32_t i0 = 0; i0 < cnt && run < need; i0 += 32) {
+    if (ccnt == 0 || run >= need) continue;
+    const uint2* cc = cd + p.chunk_base[ci];
+    for (uint32_t i0 = 0; i0 < ccnt && run < need; i0 += 32) {
       const uint32_t i = i0 + lane;
       uint2 kv = make_uint2(0, 0);
       bool eq = false;
-      if (i < cnt) {
-        kv = __ldcg(cd + i);
+      if (i < ccnt) {
+        kv = __ldcg(cc + i);
         eq = kv.x == T;
       }
       const uint32_t eb = __ballot_sync(FULL, eq);
@@ -855,25 +969,29 @@ __global__ void __launch_bounds__(TPB) k_tie_bits(P p) {
   }
 }
 
-__global__ void __launch_bounds__(TPB) k_votes(P p) {
+constexpr int VT = 128;  // threads of k_votes: one per mask word of the chunk
+
+// Chunks in which no worker kept a candidate are skipped: their votes, selected counts and vote
+// histograms were cleared at the start of the step.  NP = number of counter planes (2^NP > N).
+template <int NP>
+__global__ void __launch_bounds__(VT) k_votes(P p) {
+  pdl_enter();
   __shared__ uint32_t s_vh[256];
   __shared__ uint32_t s_sel[256];
-  __shared__ uint32_t s_any;
-  const int c = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31;
-  s_vh[tid] = 0;
-  s_sel[tid] = 0;
-  if (tid == 0) s_any = 0;
-  __syncthreads();
-  // a chunk in which no worker kept a candidate has all-zero masks: skip reading them
-  if (tid < p.N && p.chunk_cnt[(size_t)tid * p.nchunks + c] != 0) s_any = 1;
-  __syncthreads();
-  const int64_t jb = (int64_t)c * CH + (int64_t)tid * 32;
-  const int64_t wi = (int64_t)c * WPC + tid;
-  uint32_t planes[8];
+  for (int c = blockIdx.x; c < p.nchunks; c += gridDim.x) {
+    if (__ldcg(p.hot + c) == 0) continue;  // uniform over the CTA
+    __syncthreads();                       // previous chunk's readers are done
+    s_vh[tid] = 0;
+    s_vh[tid + VT] = 0;
+    s_sel[tid] = 0;
+    s_sel[tid + VT] = 0;
+    __syncthreads();
+    const int64_t jb = (int64_t)c * CH + (int64_t)tid * 32;
+    const int64_t wi = (int64_t)c * WPC + tid;
+    uint32_t planes[NP];
 #pragma unroll
-  for (int q = 0; q < 8; q++) planes[q] = 0;
-  if (s_any && tid < WPC) {  // warps 0..3, all lanes
+    for (int q = 0; q < NP; q++) planes[q] = 0;
     const bool inb = wi < p.W;
     const uint32_t* col = p.worker_bits + (inb ? wi : 0);
     for (int n0 = 0; n0 < p.N; n0 += 8) {
@@ -888,44 +1006,60 @@ __global__ void __launch_bounds__(TPB) k_votes(P p) {
           if (lane == 0 && pc) atomicAdd(&s_sel[n0 + q], pc);
         }
 #pragma unroll
-        for (int r = 0; r < 8; r++) {
+        for (int r = 0; r < NP; r++) {
           const uint32_t t2 = planes[r] & carry;
           planes[r] ^= carry;
           carry = t2;
         }
       }
     }
-  }
-  // expand the planes into 32 vote bytes per thread
-  if (tid < WPC && jb < p.d) {
-    uint32_t wv[8];
+    uint32_t any = 0;
 #pragma unroll
-    for (int q = 0; q < 8; q++) wv[q] = 0;
-    if (planes[0] | planes[1] | planes[2] | planes[3] | planes[4] | planes[5] | planes[6] | planes[7]) {
+    for (int q = 0; q < NP; q++) any |= planes[q];
+    // histogram of the vote values of this chunk: for each value v, the coordinates whose bit-sliced
+    // counter equals v are one AND over the planes away (no per-coordinate atomics)
+    if (__ballot_sync(FULL, any != 0)) {  // warp-uniform
+      uint32_t valid = 0xffffffffu;       // coordinates of this word that lie below d
+      if (jb >= p.d) valid = 0;
+      else if (jb + 32 > p.d) valid = (1u << (uint32_t)(p.d - jb)) - 1u;
+      for (int v = 1; v <= p.N; v++) {
+        uint32_t m = valid;
 #pragma unroll
-      for (int b = 0; b < 32; b++) {
-        uint32_t v = 0;
-#pragma unroll
-        for (int q = 0; q < 8; q++) v |= ((planes[q] >> b) & 1u) << q;
-        wv[b >> 2] |= v << (8 * (b & 3));
-        if (v && jb + b < p.d) atomicAdd(&s_vh[v], 1u);
+        for (int q = 0; q < NP; q++) m &= ((v >> q) & 1) ? planes[q] : ~planes[q];
+        const uint32_t cnt = __reduce_add_sync(FULL, (uint32_t)__popc(m));
+        if (lane == 0 && cnt) atomicAdd(&s_vh[v], cnt);
       }
     }
-    if (jb + 32 <= p.d) {
-      uint4* dst = reinterpret_cast<uint4*>(p.votes + jb);
-      dst[0] = make_uint4(wv[0], wv[1], wv[2], wv[3]);
-      dst[1] = make_uint4(wv[4], wv[5], wv[6], wv[7]);
-    } else {
-      for (int b = 0; b < 32 && jb + b < p.d; b++) p.votes[jb + b] = (uint8_t)((wv[b >> 2] >> (8 * (b & 3))) & 0xffu);
+    // expand the planes into 32 vote bytes per thread: a nibble of plane q becomes bit q of four bytes
+    if (jb < p.d) {
+      uint32_t wv[8];
+#pragma unroll
+      for (int g = 0; g < 8; g++) {
+        uint32_t x = 0;
+        if (any) {
+#pragma unroll
+          for (int q = 0; q < NP; q++) x |= ((((planes[q] >> (4 * g)) & 0xfu) * 0x00204081u) & 0x01010101u) << q;
+        }
+        wv[g] = x;
+      }
+      if (jb + 32 <= p.d) {
+        uint4* dst = reinterpret_cast<uint4*>(p.votes + jb);
+        dst[0] = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+        dst[1] = make_uint4(wv[4], wv[5], wv[6], wv[7]);
+      } else {
+        for (int b = 0; b < 32 && jb + b < p.d; b++) p.votes[jb + b] = (uint8_t)((wv[b >> 2] >> (8 * (b & 3))) & 0xffu);
+      }
     }
+    __syncthreads();
+    for (int n = tid; n < p.N; n += VT) p.chunk_sel[(size_t)n * p.nchunks + c] = s_sel[n];
+    store_vote_hist_impl(p, c, s_vh);
   }
-  __syncthreads();
-  if (tid < p.N) p.chunk_sel[(size_t)tid * p.nchunks + c] = s_sel[tid];
-  store_vote_hist_impl(p, c, s_vh);
+  if (last_cta(p.votes_done, gridDim.x)) vote_scan<VT>(p);
 }
 
 // per worker: list offset of every chunk = exclusive prefix of the selected counts
 __global__ void __launch_bounds__(1024) k_scan_sel(P p) {
+  pdl_enter();
   __shared__ uint32_t s_w[33];
   const int n = blockIdx.x;
   const int per = (p.nchunks + 1023) / 1024;
@@ -945,10 +1079,11 @@ __global__ void __launch_bounds__(1024) k_scan_sel(P p) {
 // ascending index lists from the bit masks: a warp per (worker, chunk).  In round q lane l owns mask
 // word 32*q + l; its set bits are staged in shared memory in order and copied out coalesced.
 __global__ void __launch_bounds__(TPB) k_lists(P p) {
+  pdl_enter();
   __shared__ uint16_t s_buf[TPB / 32][1024];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n = blockIdx.y;
-  const int c = blockIdx.x * (TPB / 32) + warp;
+  const int c = blockIdx.x + warp * gridDim.x;  // neighbouring chunks go to different CTAs
   if (c >= p.nchunks) return;
   const uint32_t next = c + 1 < p.nchunks ? p.chunk_sel[(size_t)n * p.nchunks + c + 1] : (uint32_t)p.K;
   uint32_t pos = p.chunk_sel[(size_t)n * p.nchunks + c];
@@ -991,6 +1126,7 @@ __global__ void __launch_bounds__(TPB) k_lists(P p) {
 // ---------------------------------------------------------------------------------------------
 // per-chunk and global histogram of vote values, from a vote vector (stand-alone mv_select)
 __global__ void __launch_bounds__(TPB) k_vote_hist(P p, const uint8_t* __restrict__ votes) {
+  pdl_enter();
   __shared__ uint32_t s_vh[256];
   const int c = blockIdx.x, tid = threadIdx.x;
   s_vh[tid] = 0;
@@ -1014,75 +1150,13 @@ __global__ void __launch_bounds__(TPB) k_vote_hist(P p, const uint8_t* __restric
   }
   __syncthreads();
   store_vote_hist_impl(p, c, s_vh);
-}
-
-// v* = the vote value of the K-th most voted coordinate; then per chunk the output offset and the
-// number of v*-ties it may keep (lowest index first)
-__global__ void __launch_bounds__(1024) k_vote_scan(P p) {
-  __shared__ uint32_t s_w[33];
-  __shared__ uint32_t s_v[4];
-  __shared__ uint32_t s_h[256];
-  if ((int)threadIdx.x <= p.N) s_h[threadIdx.x] = __ldcg(p.vote_hist + threadIdx.x);
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    uint32_t acc = 0, vstar = 0, cgt = 0, ceq = 0;
-    for (int v = p.N; v >= 0; v--) {
-      const uint32_t h = s_h[v];
-      if (acc + h >= (uint32_t)p.K) {
-        vstar = (uint32_t)v;
-        cgt = acc;
-        ceq = h;
-        break;
-      }
-      acc += h;
-    }
-    s_v[0] = vstar;
-    s_v[1] = cgt;
-    s_v[2] = ceq;
-    s_v[3] = (uint32_t)p.K - cgt;
-    p.vstate[0] = vstar;
-    p.vstate[1] = cgt;
-    p.vstate[2] = ceq;
-    p.vstate[3] = (uint32_t)p.K - cgt;
-  }
-  __syncthreads();
-  const uint32_t vstar = s_v[0], quota = s_v[3];
-  const int stride = p.N + 1;
-  const int per = (p.nchunks + 1023) / 1024;
-  const int c0 = min(p.nchunks, (int)threadIdx.x * per), c1 = min(p.nchunks, c0 + per);
-  // chunk_vh[c][v] = #{coordinates of chunk c with votes >= v}
-  uint32_t esum = 0;
-  for (int c = c0; c < c1; c++) {
-    const uint16_t* h = p.chunk_vh + (size_t)c * stride;
-    const uint32_t gt = (int)vstar < p.N ? h[vstar + 1] : 0u;
-    esum += h[vstar] - gt;
-  }
-  uint32_t tot;
-  const uint32_t epre = block_excl_scan<1024>(esum, s_w, tot);
-  uint32_t run = epre, ssum = 0;
-  for (int c = c0; c < c1; c++) {
-    const uint16_t* h = p.chunk_vh + (size_t)c * stride;
-    const uint32_t gt = (int)vstar < p.N ? h[vstar + 1] : 0u;
-    const uint32_t eq = h[vstar] - gt;
-    const uint32_t take = run >= quota ? 0u : min(eq, quota - run);
-    p.tie_take[c] = take;
-    run += eq;
-    ssum += gt + take;
-  }
-  const uint32_t spre = block_excl_scan<1024>(ssum, s_w, tot);
-  uint32_t srun = spre;
-  for (int c = c0; c < c1; c++) {
-    const uint16_t* h = p.chunk_vh + (size_t)c * stride;
-    const uint32_t gt = (int)vstar < p.N ? h[vstar + 1] : 0u;
-    p.out_base[c] = srun;
-    srun += gt + p.tie_take[c];
-  }
-  if (threadIdx.x == 0) p.out_base[p.nchunks] = (uint32_t)p.K;  // sentinel: end of the last chunk
+  if (last_cta(p.votes_done, gridDim.x)) vote_scan<TPB>(p);
 }
 
 // writes supp(M) (ascending) and optionally M as a bit mask
 __global__ void __launch_bounds__(TPB) k_vote_write(P p, const uint8_t* __restrict__ votes, int32_t* __restrict__ out_idx,
                                                     uint32_t* __restrict__ mask_bits) {
+  pdl_enter();
   __shared__ uint32_t s_w[TPB / 32 + 1];
   const int c = blockIdx.x, tid = threadIdx.x;
   const uint32_t vstar = p.vstate[0];
@@ -1154,6 +1228,7 @@ __global__ void __launch_bounds__(TPB) k_vote_write(P p, const uint8_t* __restri
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(TPB) k_gather(float* __restrict__ acc, int N, int64_t d, int64_t K,
                                                 const int32_t* __restrict__ idx, float* __restrict__ out_val) {
+  pdl_enter();
   const int64_t k = (int64_t)blockIdx.x * TPB + threadIdx.x;
   if (k >= K) return;
   const int64_t j = idx[k];
@@ -1162,22 +1237,18 @@ __global__ void __launch_bounds__(TPB) k_gather(float* __restrict__ acc, int N, 
     return;
   }
   float* col = acc + j;
+  // all loads before any store: a store to acc followed by a load from acc (another row) would
+  // otherwise be kept in program order and serialise the memory latency row by row
   double s = 0.0;
-  int n = 0;
-  for (; n + 8 <= N; n += 8) {
-    float v[8];
+  for (int n0 = 0; n0 < N; n0 += 16) {
+    float v[16];
 #pragma unroll
-    for (int q = 0; q < 8; q++) v[q] = col[(size_t)(n + q) * (size_t)d];
+    for (int q = 0; q < 16; q++) v[q] = n0 + q < N ? __ldcg(col + (size_t)(n0 + q) * (size_t)d) : 0.f;
 #pragma unroll
-    for (int q = 0; q < 8; q++) {
-      s += (double)v[q];
-      col[(size_t)(n + q) * (size_t)d] = 0.0f;
-    }
+    for (int q = 0; q < 16; q++)
+      if (n0 + q < N) s += (double)v[q];
   }
-  for (; n < N; n++) {
-    s += (double)col[(size_t)n * (size_t)d];
-    col[(size_t)n * (size_t)d] = 0.0f;
-  }
+  for (int n = 0; n < N; n++) __stcg(col + (size_t)n * (size_t)d, 0.0f);
   out_val[k] = (float)(s / (double)N);
 }
 
@@ -1189,7 +1260,7 @@ struct Layout {
   int64_t W;
   uint32_t cap;
   size_t zero_bytes;  // the leading region cleared at the start of every vote
-  size_t samp_hist, hist1, hist2, hist3, cand_cnt, sample_done, vote_hist;
+  size_t samp_hist, hist1, hist2, hist3, cand_cnt, sample_done, count_done, votes_done, hot, vote_hist;
   size_t tau, wstate, thresh, vstate, cand, chunk_base, chunk_cnt, chunk_gt, chunk_eq, tie_base, sel_base, chunk_sel;
   size_t worker_bits, worker_idx, votes, chunk_vh, out_base, tie_take;
   size_t total;
@@ -1220,6 +1291,9 @@ Layout make_layout(int N, int64_t d, int64_t K) {
   L.hist3 = take(off, n * H3_BINS * 4);
   L.cand_cnt = take(off, n * 4);
   L.sample_done = take(off, n * 4);
+  L.count_done = take(off, n * 4);
+  L.hot = take(off, (size_t)((L.nchunks + 7) & ~7));
+  L.votes_done = take(off, 4);
   L.vote_hist = take(off, 256 * 4);
   L.zero_bytes = off;
   L.tau = take(off, n * 4);
@@ -1237,7 +1311,7 @@ Layout make_layout(int N, int64_t d, int64_t K) {
   L.worker_bits = take(off, n * (size_t)L.W * 4);
   L.worker_idx = take(off, n * (size_t)K * 4);
   L.votes = take(off, nc * CH);
-  L.chunk_vh = take(off, nc * (n + 1) * 2);
+  L.chunk_vh = take(off, (size_t)(((L.nchunks + 7) & ~7)) * (n + 1) * 2);
   L.out_base = take(off, (nc + 1) * 4);
   L.tie_take = take(off, nc * 4);
   L.total = off;
@@ -1255,10 +1329,21 @@ struct mv_ctx {
   int mode;
   int launches;
   // optional CUDA-event timing of the streaming pass (ring of event pairs)
-  int timing;
+  int timing;                // 0 = off, n = record on every n-th call
+  int timing_calls;          // calls seen since timing was switched on
+  bool timing_now;           // this call records
   int timed;                 // pairs recorded since the last read
   cudaEvent_t ev[2 * 64];
   bool ev_made;
+  // index lists are written on a side stream, concurrently with mask selection and aggregation
+  cudaStream_t side;
+  cudaEvent_t ev_fork, ev_join, ev_zero;
+  int side_state;  // 0 = not tried, 1 = ready, -1 = unavailable
+  bool join_pending;
+  // optional per-launch timing of one call: pev[i] is recorded after the i-th launch (pev[0] before the first)
+  int phase_timing;
+  cudaEvent_t pev[48];
+  bool pev_made;
   // remembered for mv_read_diag
   int last_N;
   int64_t last_d, last_K;
@@ -1271,6 +1356,7 @@ P make_params(const mv_ctx* ctx, const Layout& L, int N, int64_t d, int64_t K) {
   char* b = ctx->ws;
   p.N = N;
   p.nchunks = L.nchunks;
+  p.nc_pad = (L.nchunks + 7) & ~7;
   p.cap = L.cap;
   p.force_general = ctx->mode == MV_MODE_GENERAL ? 1 : 0;
   p.d = d;
@@ -1282,6 +1368,9 @@ P make_params(const mv_ctx* ctx, const Layout& L, int N, int64_t d, int64_t K) {
   p.hist3 = (uint32_t*)(b + L.hist3);
   p.cand_cnt = (uint32_t*)(b + L.cand_cnt);
   p.sample_done = (uint32_t*)(b + L.sample_done);
+  p.count_done = (uint32_t*)(b + L.count_done);
+  p.votes_done = (uint32_t*)(b + L.votes_done);
+  p.hot = (uint8_t*)(b + L.hot);
   p.vote_hist = (uint32_t*)(b + L.vote_hist);
   p.tau = (uint32_t*)(b + L.tau);
   p.wstate = (uint32_t*)(b + L.wstate);
@@ -1304,6 +1393,21 @@ P make_params(const mv_ctx* ctx, const Layout& L, int N, int64_t d, int64_t K) {
   return p;
 }
 
+template <typename... KArgs, typename... Args>
+cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 int per_row_ctas(int N, int want, int budget) {
   int lim = budget / N;
   if (lim < 1) lim = 1;
@@ -1311,10 +1415,11 @@ int per_row_ctas(int N, int want, int budget) {
   return want < lim ? want : lim;
 }
 
-#define MV_LAUNCH_CHECK()                          \
-  do {                                             \
-    ctx->launches++;                               \
-    if (cudaGetLastError() != cudaSuccess) return MV_ERR_CUDA; \
+#define MV_LAUNCH_CHECK()                                                                        \
+  do {                                                                                           \
+    ctx->launches++;                                                                             \
+    if (cudaGetLastError() != cudaSuccess) return MV_ERR_CUDA;                                   \
+    if (ctx->phase_timing && ctx->launches < 48) cudaEventRecord(ctx->pev[ctx->launches], ctx->stream); \
   } while (0)
 
 // sample size and rank for the threshold estimate
@@ -1339,53 +1444,109 @@ void sample_plan(int64_t d, int64_t K, uint32_t& U, uint32_t& L, int& all, uint3
   rank = (uint32_t)r;
 }
 
+bool side_ready(mv_ctx* ctx) {
+  if (ctx->side_state == 0) {
+    ctx->side_state = -1;
+    if (cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking) == cudaSuccess) {
+      if (cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming) == cudaSuccess) {
+        if (cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming) == cudaSuccess) {
+          if (cudaEventCreateWithFlags(&ctx->ev_zero, cudaEventDisableTiming) == cudaSuccess)
+            ctx->side_state = 1;
+          else
+            cudaEventDestroy(ctx->ev_join);
+        }
+        if (ctx->side_state != 1) cudaEventDestroy(ctx->ev_fork);
+      }
+      if (ctx->side_state != 1) cudaStreamDestroy(ctx->side);
+    }
+  }
+  return ctx->side_state == 1;
+}
+
+// the caller's stream waits for the side stream's work of this call
+int join_side(mv_ctx* ctx) {
+  if (ctx->join_pending) {
+    ctx->join_pending = false;
+    if (cudaStreamWaitEvent(ctx->stream, ctx->ev_join, 0) != cudaSuccess) return MV_ERR_CUDA;
+  }
+  return MV_OK;
+}
+
 // steps a1-a3: accumulate, per-worker top-K, votes
 int vote_impl(mv_ctx* ctx, P p, const Layout& L, const float* grads, float* err) {
   cudaStream_t st = ctx->stream;
   const int N = p.N;
+  ctx->timing_now = ctx->timing > 0 && (ctx->timing_calls++ % ctx->timing) == 0;
   if (cudaMemsetAsync(ctx->ws, 0, L.zero_bytes, st) != cudaSuccess) return MV_ERR_CUDA;
+  // per-chunk outputs of the vote count start out cleared (only chunks with candidates are
+  // visited later); cleared on the side stream, concurrently with the sampling and streaming pass
+  cudaStream_t zs = st;
+  if (!ctx->phase_timing && side_ready(ctx) && cudaEventRecord(ctx->ev_fork, st) == cudaSuccess &&
+      cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) == cudaSuccess)
+    zs = ctx->side;
+  {
+    const size_t nc = (size_t)p.nchunks;
+    cudaError_t e = cudaMemsetAsync(p.votes, 0, (size_t)p.d, zs);
+    if (e == cudaSuccess) e = cudaMemsetAsync(p.chunk_sel, 0, (size_t)N * nc * 4, zs);
+    if (e == cudaSuccess) e = cudaMemsetAsync(p.chunk_vh, 0, (size_t)(N + 1) * (size_t)p.nc_pad * 2, zs);
+    if (e != cudaSuccess) return MV_ERR_CUDA;
+    if (zs != st && cudaEventRecord(ctx->ev_zero, zs) != cudaSuccess) return MV_ERR_CUDA;
+  }
   // CTAs per worker of the select kernels: enough for a full-row pass, not more than the candidates need
-  const int gh = per_row_ctas(N, p.force_general ? p.nchunks : (int)((p.cap + TPB * 4 - 1) / (TPB * 4)), 148 * 8);
+  const int gh = p.force_general ? per_row_ctas(N, p.nchunks, 148 * 8)
+                                 : per_row_ctas(N, (int)((p.cap + TPB * 8 - 1) / (TPB * 8)), 148 * 2);
   if (!p.force_general) {
     uint32_t U, Ls, rank;
     int all;
     sample_plan(p.d, p.K, U, Ls, all, rank);
-    const int gs = per_row_ctas(N, (int)((U + 63) / 64), 148 * 4);
-    k_sample_hist<<<dim3(gs, N), 512, 0, st>>>(p, grads, err, U, Ls, all, rank);
+    const int gs = per_row_ctas(N, (int)((U + 127) / 128), 148 * 2);
+    launch_k(k_sample_hist, dim3(dim3(gs, N)), dim3(512), st, p, grads, err, U, Ls, all, rank);
     MV_LAUNCH_CHECK();
-    if (ctx->timing) cudaEventRecord(ctx->ev[2 * (ctx->timed % 64)], st);
-    k_acc_compact<<<dim3(p.nchunks, N), TPB, 0, st>>>(p, grads, err);
+    if (ctx->timing_now) cudaEventRecord(ctx->ev[2 * (ctx->timed % 64)], st);
+    launch_k(k_acc_compact, dim3(dim3(p.nchunks, N)), dim3(TPB), st, p, grads, err);
     MV_LAUNCH_CHECK();
-    if (ctx->timing) cudaEventRecord(ctx->ev[2 * (ctx->timed++ % 64) + 1], st);
-    k_hist<1, false><<<dim3(gh, N), TPB, 0, st>>>(p, nullptr, err);
+    if (ctx->timing_now) cudaEventRecord(ctx->ev[2 * (ctx->timed++ % 64) + 1], st);
+    launch_k(k_hist<1, false>, dim3(dim3(gh, N)), dim3(TPB), st, p, nullptr, err);
     MV_LAUNCH_CHECK();
   } else {
-    if (ctx->timing) cudaEventRecord(ctx->ev[2 * (ctx->timed % 64)], st);
-    k_hist<1, true><<<dim3(gh, N), TPB, 0, st>>>(p, grads, err);
+    if (ctx->timing_now) cudaEventRecord(ctx->ev[2 * (ctx->timed % 64)], st);
+    launch_k(k_hist<1, true>, dim3(dim3(gh, N)), dim3(TPB), st, p, grads, err);
     MV_LAUNCH_CHECK();
-    if (ctx->timing) cudaEventRecord(ctx->ev[2 * (ctx->timed++ % 64) + 1], st);
+    if (ctx->timing_now) cudaEventRecord(ctx->ev[2 * (ctx->timed++ % 64) + 1], st);
   }
-  k_hist<2, false><<<dim3(gh, N), TPB, 0, st>>>(p, nullptr, err);
+  launch_k(k_hist<2, false>, dim3(dim3(gh, N)), dim3(TPB), st, p, nullptr, err);
   MV_LAUNCH_CHECK();
-  k_hist<3, false><<<dim3(gh, N), TPB, 0, st>>>(p, nullptr, err);
+  launch_k(k_hist<3, false>, dim3(dim3(gh, N)), dim3(TPB), st, p, nullptr, err);
   MV_LAUNCH_CHECK();
-  k_count<<<dim3(gh, N), TPB, 0, st>>>(p, err);
+  launch_k(k_count, dim3(dim3(gh, N)), dim3(TPB), st, p, err);
   MV_LAUNCH_CHECK();
-  k_chunk_scan<<<N, 1024, 0, st>>>(p);
+  launch_k(k_row_exact, dim3(dim3(gh, N)), dim3(TPB), st, p, err);
   MV_LAUNCH_CHECK();
-  k_row_exact<<<dim3(gh, N), TPB, 0, st>>>(p, err);
+  const int gb = per_row_ctas(N, (int)((p.cap + TPB * 16 - 1) / (TPB * 16)), 148 * 4);
+  launch_k(k_set_bits, dim3(dim3(gb, N)), dim3(TPB), st, p);
   MV_LAUNCH_CHECK();
-  const int gb = per_row_ctas(N, (int)((p.cap + TPB * 8 - 1) / (TPB * 8)), 148 * 8);
-  k_set_bits<<<dim3(gb, N), TPB, 0, st>>>(p);
+  if (zs != st && cudaStreamWaitEvent(st, ctx->ev_zero, 0) != cudaSuccess) return MV_ERR_CUDA;
+  {
+    const dim3 gv(p.nchunks < 148 * 8 ? p.nchunks : 148 * 8);
+    if (N < 4) launch_k(k_votes<2>, gv, dim3(VT), st, p);
+    else if (N < 16) launch_k(k_votes<4>, gv, dim3(VT), st, p);
+    else if (N < 64) launch_k(k_votes<6>, gv, dim3(VT), st, p);
+    else launch_k(k_votes<8>, gv, dim3(VT), st, p);
+  }
   MV_LAUNCH_CHECK();
-  k_tie_bits<<<dim3(per_row_ctas(N, (p.nchunks + 7) / 8, 148 * 4), N), TPB, 0, st>>>(p);
+  // the index lists feed nothing later in the step: write them on the side stream
+  cudaStream_t ls = st;
+  if (!ctx->phase_timing && side_ready(ctx) && cudaEventRecord(ctx->ev_fork, st) == cudaSuccess &&
+      cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) == cudaSuccess)
+    ls = ctx->side;
+  launch_k(k_scan_sel, dim3(N), dim3(1024), ls, p);
   MV_LAUNCH_CHECK();
-  k_votes<<<p.nchunks, TPB, 0, st>>>(p);
+  launch_k(k_lists, dim3(dim3((p.nchunks + TPB / 32 - 1) / (TPB / 32), N)), dim3(TPB), ls, p);
   MV_LAUNCH_CHECK();
-  k_scan_sel<<<N, 1024, 0, st>>>(p);
-  MV_LAUNCH_CHECK();
-  k_lists<<<dim3((p.nchunks + TPB / 32 - 1) / (TPB / 32), N), TPB, 0, st>>>(p);
-  MV_LAUNCH_CHECK();
+  if (ls != st) {
+    if (cudaEventRecord(ctx->ev_join, ls) != cudaSuccess) return MV_ERR_CUDA;
+    ctx->join_pending = true;
+  }
   return MV_OK;
 }
 
@@ -1394,20 +1555,18 @@ int select_impl(mv_ctx* ctx, P p, const Layout& L, const uint8_t* votes, bool ha
                 uint32_t* mask_bits) {
   cudaStream_t st = ctx->stream;
   if (!have_hist) {
-    if (cudaMemsetAsync(ctx->ws + L.vote_hist, 0, 256 * 4, st) != cudaSuccess) return MV_ERR_CUDA;
-    k_vote_hist<<<p.nchunks, TPB, 0, st>>>(p, votes);
+    if (cudaMemsetAsync(ctx->ws + L.votes_done, 0, L.zero_bytes - L.votes_done, st) != cudaSuccess) return MV_ERR_CUDA;
+    launch_k(k_vote_hist, dim3(p.nchunks), dim3(TPB), st, p, votes);
     MV_LAUNCH_CHECK();
   }
-  k_vote_scan<<<1, 1024, 0, st>>>(p);
-  MV_LAUNCH_CHECK();
-  k_vote_write<<<p.nchunks, TPB, 0, st>>>(p, votes, out_idx, mask_bits);
+  launch_k(k_vote_write, dim3(p.nchunks), dim3(TPB), st, p, votes, out_idx, mask_bits);
   MV_LAUNCH_CHECK();
   return MV_OK;
 }
 
 // steps a5-a6
 int aggregate_impl(mv_ctx* ctx, float* acc, int N, int64_t d, int64_t K, const int32_t* idx, float* out_val) {
-  k_gather<<<(unsigned)((K + TPB - 1) / TPB), TPB, 0, ctx->stream>>>(acc, N, d, K, idx, out_val);
+  launch_k(k_gather, dim3((unsigned)((K + TPB - 1) / TPB)), dim3(TPB), ctx->stream, acc, N, d, K, idx, out_val);
   MV_LAUNCH_CHECK();
   return MV_OK;
 }
@@ -1446,8 +1605,15 @@ int mv_create(mv_ctx** out, void* stream, void* workspace, size_t workspace_byte
   c->mode = MV_MODE_AUTO;
   c->launches = 0;
   c->timing = 0;
+  c->timing_calls = 0;
+  c->timing_now = false;
   c->timed = 0;
   c->ev_made = false;
+  c->phase_timing = 0;
+  c->pev_made = false;
+  c->side = nullptr;
+  c->side_state = 0;
+  c->join_pending = false;
   c->last_N = 0;
   c->last_d = 0;
   c->last_K = 0;
@@ -1459,6 +1625,14 @@ int mv_destroy(mv_ctx* ctx) {
   if (ctx == nullptr) return MV_ERR_INVALID_ARG;
   if (ctx->ev_made)
     for (int i = 0; i < 2 * 64; i++) cudaEventDestroy(ctx->ev[i]);
+  if (ctx->pev_made)
+    for (int i = 0; i < 48; i++) cudaEventDestroy(ctx->pev[i]);
+  if (ctx->side_state == 1) {
+    cudaEventDestroy(ctx->ev_fork);
+    cudaEventDestroy(ctx->ev_join);
+    cudaEventDestroy(ctx->ev_zero);
+    cudaStreamDestroy(ctx->side);
+  }
   delete ctx;
   return MV_OK;
 }
@@ -1470,8 +1644,31 @@ int mv_set_kernel_timing(mv_ctx* ctx, int enable) {
       if (cudaEventCreate(&ctx->ev[i]) != cudaSuccess) return MV_ERR_CUDA;
     ctx->ev_made = true;
   }
-  ctx->timing = enable ? 1 : 0;
+  ctx->timing = enable > 0 ? enable : 0;
+  ctx->timing_calls = 0;
   ctx->timed = 0;
+  return MV_OK;
+}
+
+int mv_set_phase_timing(mv_ctx* ctx, int enable) {
+  if (ctx == nullptr) return MV_ERR_INVALID_ARG;
+  if (enable && !ctx->pev_made) {
+    for (int i = 0; i < 48; i++)
+      if (cudaEventCreate(&ctx->pev[i]) != cudaSuccess) return MV_ERR_CUDA;
+    ctx->pev_made = true;
+  }
+  ctx->phase_timing = enable ? 1 : 0;
+  return MV_OK;
+}
+
+int mv_read_phase_times(mv_ctx* ctx, float* ms, int capacity, int* count) {
+  if (ctx == nullptr || ms == nullptr || count == nullptr || !ctx->pev_made) return MV_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return MV_ERR_CUDA;
+  int n = ctx->launches < 47 ? ctx->launches : 47;
+  if (n > capacity) n = capacity;
+  for (int i = 0; i < n; i++)
+    if (cudaEventElapsedTime(&ms[i], ctx->pev[i], ctx->pev[i + 1]) != cudaSuccess) return MV_ERR_CUDA;
+  *count = n;
   return MV_OK;
 }
 
@@ -1509,6 +1706,7 @@ int mv_vote(mv_ctx* ctx, const float* grads, float* err, int N, int64_t d, int64
       (votes && !aligned16(votes)) || (thresh && !aligned16(thresh)))
     return MV_ERR_INVALID_ARG;
   ctx->launches = 0;
+  if (ctx->phase_timing) cudaEventRecord(ctx->pev[0], ctx->stream);
   P p = make_params(ctx, L, N, d, K);
   if (worker_idx) p.worker_idx = worker_idx;
   if (worker_bits) p.worker_bits = worker_bits;
@@ -1517,7 +1715,9 @@ int mv_vote(mv_ctx* ctx, const float* grads, float* err, int N, int64_t d, int64
   ctx->last_N = N;
   ctx->last_d = d;
   ctx->last_K = K;
-  return vote_impl(ctx, p, L, grads, err);
+  const int rc2 = vote_impl(ctx, p, L, grads, err);
+  const int rc3 = join_side(ctx);
+  return rc2 != MV_OK ? rc2 : rc3;
 }
 
 int mv_select(mv_ctx* ctx, const uint8_t* votes, int N, int64_t d, int64_t K, int32_t* out_idx, uint32_t* mask_bits) {
@@ -1527,6 +1727,7 @@ int mv_select(mv_ctx* ctx, const uint8_t* votes, int N, int64_t d, int64_t K, in
   if (votes == nullptr || out_idx == nullptr || !aligned16(votes) || !aligned16(out_idx)) return MV_ERR_INVALID_ARG;
   if (mask_bits && !aligned16(mask_bits)) return MV_ERR_INVALID_ARG;
   ctx->launches = 0;
+  if (ctx->phase_timing) cudaEventRecord(ctx->pev[0], ctx->stream);
   P p = make_params(ctx, L, N, d, K);
   return select_impl(ctx, p, L, votes, false, out_idx, mask_bits);
 }
@@ -1538,6 +1739,7 @@ int mv_aggregate(mv_ctx* ctx, float* acc, int N, int64_t d, int64_t K, const int
   if (acc == nullptr || idx == nullptr || out_val == nullptr || !aligned16(acc) || !aligned16(idx) || !aligned16(out_val))
     return MV_ERR_INVALID_ARG;
   ctx->launches = 0;
+  if (ctx->phase_timing) cudaEventRecord(ctx->pev[0], ctx->stream);
   return aggregate_impl(ctx, acc, N, d, K, idx, out_val);
 }
 
@@ -1551,15 +1753,16 @@ int mv_sparse_step(mv_ctx* ctx, const float* grads, float* err, int N, int64_t d
   const size_t nb = (size_t)N * (size_t)d * 4;
   if (overlap(grads, nb, err, nb)) return MV_ERR_INVALID_ARG;
   ctx->launches = 0;
+  if (ctx->phase_timing) cudaEventRecord(ctx->pev[0], ctx->stream);
   P p = make_params(ctx, L, N, d, K);
   ctx->last_N = N;
   ctx->last_d = d;
   ctx->last_K = K;
   rc = vote_impl(ctx, p, L, grads, err);
-  if (rc != MV_OK) return rc;
-  rc = select_impl(ctx, p, L, p.votes, true, out_idx, nullptr);
-  if (rc != MV_OK) return rc;
-  return aggregate_impl(ctx, err, N, d, K, out_idx, out_val);
+  if (rc == MV_OK) rc = select_impl(ctx, p, L, p.votes, true, out_idx, nullptr);
+  if (rc == MV_OK) rc = aggregate_impl(ctx, err, N, d, K, out_idx, out_val);
+  const int rcj = join_side(ctx);
+  return rc != MV_OK ? rc : rcj;
 }
 
 int mv_sparse_step_host(mv_ctx* ctx, const float* h_grads, int N, int64_t d, int64_t K, int32_t* h_out_idx,
