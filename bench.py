@@ -191,6 +191,19 @@ def run_reference(args, w: WL.Workload):
     print(json.dumps(line), flush=True)
 
 
+def max_over_ranks(value: float, dist, device) -> float:
+    """Largest value over all ranks (the job is as slow as its slowest replica)."""
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_steps_per_s(ms_total_max: float, world: int, steps: int) -> float:
+    """Whole-job throughput of `world` independent replicas that each ran `steps` steps."""
+    return world * steps / (ms_total_max * 1e-3)
+
+
 def workload_config(w: WL.Workload):
     return {"workload": f"{w.name}: N={w.N} workers, d={w.d} fp32, K={w.K} ({w.note}), error feedback carried, "
                         f"fresh gradients every step",
@@ -272,12 +285,9 @@ def main():
     k_ms, k_cnt = ctx.read_kernel_timing()
     ctx.set_kernel_timing(0)
     diag = ctx.read_diag(w.N)
-    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, dist, dev)
     ms_step = ms_total / args.steps
-    value = world * args.steps / (ms_total * 1e-3)
+    value = job_steps_per_s(ms_total, world, args.steps)
 
     # ---- end to end through the host entry point: gradients start in pinned host memory
     e2e = None
@@ -296,10 +306,8 @@ def main():
             ctx.mv_sparse_step_host(h_pool[i % 2], h_idx, h_val, d_grads, err, out_idx, out_val)
         e1.record()
         barrier()
-        te = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
-        if dist is not None:
-            dist.all_reduce(te, op=dist.ReduceOp.MAX)
-        e2e = {"value": world * e_steps / (float(te.item()) * 1e-3), "unit": UNIT,
+        te = max_over_ranks(e0.elapsed_time(e1), dist, dev)
+        e2e = {"value": job_steps_per_s(te, world, e_steps), "unit": UNIT,
                "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": 8 * w.K, "steps": e_steps,
                "note": "mv_sparse_step_host: gradients copied from pinned host memory every step, indices and "
                        "values copied back; the residual stays on the device"}

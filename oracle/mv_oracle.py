@@ -12,7 +12,7 @@ parameter-server side collapsed onto one machine):
   2. M_n     = S_top(|acc_n|, K)                    per-worker top-K mask (Eq. 6 / S_top)
   3. votes   = sum_n M_n                            vote count per coordinate (Eq. 9)
   4. M       = S_top(votes, K)                      the K most voted coordinates (Eq. 9)
-  5. out_val = (1/N) sum_n (M (x) acc_n) on supp(M) shared-mask aggregate (Eq. 8, 1/N as in Eq. 7's G~)
+  5. out_val = (1/N) sum_n (M (x) acc_n) on supp(M) shared-mask aggregate (Eq. 8; mean as in the text)
   6. err_n   = acc_n - M (x) acc_n                  residual (Alg. 1, error update)
 
 Readings where the paper is silent (each is also listed in the design notes):
@@ -90,8 +90,8 @@ def _stop(score: np.ndarray, K: int):
     cnt_eq = int(np.count_nonzero(eq))
     need = K - cnt_gt
     assert 1 <= need <= cnt_eq
-    tie_rank = np.cumsum(eq, dtype=np.int64) - 1       # 0-based rank among the ties, by index
-    take = gt | (eq & (tie_rank < need))
+    take = gt
+    take[np.flatnonzero(eq)[:need]] = True             # the `need` lowest-index ties
     return np.flatnonzero(take).astype(np.int32), thr, cnt_gt, cnt_eq
 
 
@@ -168,30 +168,41 @@ def residual(acc: np.ndarray, idx: np.ndarray) -> np.ndarray:
 # ----------------------------------------------------------------------------
 # the whole step
 # ----------------------------------------------------------------------------
-def mv_vote(grads, err, K: int, by_sort: bool = False):
+def mv_vote(grads, err, K: int, by_sort: bool = False, threads: int = 1):
     """Steps 1-3.  Returns a dict with acc, worker_idx [N,K], worker_bits
-    [N,ceil(d/32)], votes [d] and thresh [N,3] = (T_n, cnt_gt, cnt_eq)."""
+    [N,ceil(d/32)], votes [d] and thresh [N,3] = (T_n, cnt_gt, cnt_eq).
+    The workers' rows are independent; `threads` > 1 only lets several rows be
+    selected at the same time (same functions, same results)."""
     acc = accumulate(grads, err)
     N, d = acc.shape
     topk = worker_topk_by_sort if by_sort else worker_topk
     worker_idx = np.empty((N, K), dtype=np.int32)
     worker_bits = np.empty((N, (d + 31) // 32), dtype=np.uint32)
     thresh = np.empty((N, 3), dtype=np.uint32)
-    for n in range(N):
+
+    def one_row(n):
         idx, T, cnt_gt, cnt_eq = topk(acc[n], K)
         worker_idx[n] = idx
         worker_bits[n] = support_to_bits(idx, d)
         thresh[n] = (T, cnt_gt, cnt_eq)
+
+    if threads > 1:
+        from concurrent.futures import ThreadPoolExecutor
+        with ThreadPoolExecutor(max_workers=threads) as pool:
+            list(pool.map(one_row, range(N)))
+    else:
+        for n in range(N):
+            one_row(n)
     votes = count_votes(worker_idx, d)
     return dict(acc=acc, worker_idx=worker_idx, worker_bits=worker_bits,
                 votes=votes, thresh=thresh)
 
 
-def mv_sparse_step(grads, err, K: int, by_sort: bool = False):
+def mv_sparse_step(grads, err, K: int, by_sort: bool = False, threads: int = 1):
     """One full step.  Returns a dict with everything the step defines:
     acc, worker_idx, worker_bits, votes, thresh, out_idx [K], mask_bits,
     vote_thresh = (v*, cnt_gt, cnt_eq), out_val [K] and the new err [N,d]."""
-    r = mv_vote(grads, err, K, by_sort=by_sort)
+    r = mv_vote(grads, err, K, by_sort=by_sort, threads=threads)
     sel = select_mask_by_sort if by_sort else select_mask
     out_idx, vstar, vgt, veq = sel(r["votes"], K)
     r["out_idx"] = out_idx

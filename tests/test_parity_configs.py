@@ -1,0 +1,146 @@
+"""GPU parity at the full sizes of the named configurations, in the launch configuration the
+benchmark times (mv_sparse_step on the current stream, automatic threshold mode).
+
+c2, c3, c4: every step of the run is compared with the CPU oracle (shared mask, aggregated values,
+residual), the residual being carried on both sides; the first and last step also compare the
+per-worker lists, masks, votes and thresholds.  The sweep cells (c5) compare everything for the
+small and middle sizes and, for the 2^27-coordinate cells, sampled rows and sampled outputs plus
+properties that hold at any size.  Inputs are generated on the GPU and the same bytes go to the
+oracle.
+"""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import mv_oracle as O
+from paper_2011_06495_b200 import binding as B
+from paper_2011_06495_b200 import workloads as WL
+from tests import parity as PT
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+THREADS = max(1, min(16, len(os.sched_getaffinity(0))))
+FULL = os.environ.get("MV_TEST_QUICK", "0") != "1"     # MV_TEST_QUICK=1: fewer steps and 9 of the 27 sweep cells
+
+
+def run_config(w, steps):
+    std = WL.std_vector(w, DEV) if w.segments > 1 else None
+    ctx = B.MvContext(w.N, w.d, w.K, device=DEV)
+    err = WL.initial_err(w, device=DEV)
+    err_ref = err.cpu().numpy()
+    out_idx = torch.empty(w.K, dtype=torch.int32, device=DEV)
+    out_val = torch.empty(w.K, dtype=torch.float32, device=DEV)
+    grads = torch.empty((w.N, w.d), dtype=torch.float32, device=DEV)
+    fallbacks = 0
+    for step in range(steps):
+        WL.gradients(w, step, out=grads, std=std)
+        g_np = grads.cpu().numpy()
+        ref = O.mv_sparse_step(g_np, err_ref, w.K, threads=THREADS)
+        tag = f"[{w.name} step {step}] "
+        if step in (0, steps - 1):
+            ph = PT.run_phases(ctx, grads, err, w.K)
+            PT.first_diff(PT.npy(ph["thresh"], np.uint32), ref["thresh"], tag + "thresh")
+            PT.first_diff(PT.npy(ph["worker_idx"]), ref["worker_idx"], tag + "worker_idx")
+            PT.first_diff(PT.npy(ph["worker_bits"], np.uint32), ref["worker_bits"], tag + "worker_bits")
+            PT.first_diff(PT.npy(ph["votes"]), ref["votes"], tag + "votes")
+            PT.first_diff(PT.npy(ph["mask_bits"], np.uint32), ref["mask_bits"], tag + "mask_bits")
+            del ph
+        ctx.mv_sparse_step(grads, err, out_idx, out_val)
+        torch.cuda.synchronize()
+        fallbacks += int(ctx.read_diag(w.N)[:, 2].sum())
+        PT.first_diff(PT.npy(out_idx), ref["out_idx"], tag + "out_idx")
+        PT.check_out_val(PT.npy(out_val), ref, ref["acc"], ref["out_idx"].astype(np.int64), tag + "out_val")
+        PT.first_diff(PT.bits(PT.npy(err)), PT.bits(ref["err"]), tag + "err")
+        err_ref = ref["err"]
+        del ref
+    return fallbacks
+
+
+@pytest.mark.parametrize("name", ["c2", "c3", "c4"])
+def test_named_config_every_step(name):
+    w = WL.resnet_like(name)
+    steps = w.steps if (FULL or name == "c2") else min(w.steps, 8)
+    fallbacks = run_config(w, steps)
+    assert fallbacks == 0, f"{fallbacks} worker-steps fell back to the full-row select on smooth data"
+
+
+def _cells():
+    cells = WL.sweep_cells()
+    if FULL:
+        return cells
+    keep = []
+    for i, w in enumerate(cells):       # one K per (N, d) pair, rotating through the three ratios
+        if (i % 3) == ((i // 3 + i // 9) % 3):
+            keep.append(w)
+    return keep
+
+
+@pytest.mark.parametrize("w", _cells(), ids=lambda w: w.name)
+def test_sweep_cell(w):
+    big = w.N * w.d > (1 << 28)
+    ctx = B.MvContext(w.N, w.d, w.K, device=DEV)
+    grads = WL.gradients(w, 0, device=DEV)
+    err0 = WL.initial_err(w, device=DEV)
+    if not big:
+        PT.compare_all(ctx, grads, err0, w.K, ref=O.mv_sparse_step(PT.npy(grads), PT.npy(err0), w.K, threads=THREADS),
+                       label=f"[{w.name}] ")
+        return
+    # ---- large cell: sampled rows through the oracle, the rest through size-independent properties
+    N, d, K = w.N, w.d, w.K
+    W = (d + 31) // 32
+    acc = err0.clone()
+    worker_idx = torch.empty((N, K), dtype=torch.int32, device=DEV)
+    worker_bits = torch.empty((N, W), dtype=torch.int32, device=DEV)
+    votes = torch.empty(d, dtype=torch.uint8, device=DEV)
+    thresh = torch.empty((N, 3), dtype=torch.int32, device=DEV)
+    ctx.mv_vote(grads, acc, worker_idx, worker_bits, votes, thresh)
+    torch.cuda.synchronize()
+    rows = sorted({0, N // 2, N - 1})
+    for n in rows:
+        acc_row = O.accumulate(PT.npy(grads[n])[None, :], PT.npy(err0[n])[None, :])[0]
+        PT.first_diff(PT.bits(PT.npy(acc[n])), PT.bits(acc_row), f"[{w.name}] acc row {n}")
+        idx, T, cnt_gt, cnt_eq = O.worker_topk(acc_row, K)
+        PT.first_diff(PT.npy(worker_idx[n]), idx, f"[{w.name}] worker_idx row {n}")
+        assert PT.npy(thresh[n], np.uint32).tolist() == [T, cnt_gt, cnt_eq]
+        PT.first_diff(PT.npy(worker_bits[n], np.uint32), O.support_to_bits(idx, d), f"[{w.name}] worker_bits row {n}")
+    # properties: lists strictly ascending, masks hold exactly the listed bits, votes = sum of the lists
+    assert bool((worker_idx[:, 1:] > worker_idx[:, :-1]).all())
+    tally = torch.zeros(d, dtype=torch.int32, device=DEV)
+    for n in range(N):
+        tally.index_add_(0, worker_idx[n].long(), torch.ones(K, dtype=torch.int32, device=DEV))
+    assert torch.equal(tally.to(torch.uint8), votes), "votes differ from the tally of the index lists"
+    assert int(votes.sum(dtype=torch.int64)) == N * K
+    del tally
+    # shared mask: the oracle on the full vote vector
+    out_idx = torch.empty(K, dtype=torch.int32, device=DEV)
+    mask_bits = torch.empty(W, dtype=torch.int32, device=DEV)
+    ctx.mv_select(votes, N, out_idx, mask_bits)
+    torch.cuda.synchronize()
+    ref_idx, vstar, vgt, veq = O.select_mask(PT.npy(votes), K)
+    PT.first_diff(PT.npy(out_idx), ref_idx, f"[{w.name}] out_idx")
+    PT.first_diff(PT.npy(mask_bits, np.uint32), O.support_to_bits(ref_idx, d), f"[{w.name}] mask_bits")
+    assert vstar >= 1
+    # aggregate: sampled outputs one by one, residual: sampled rows in full, the others by property
+    out_val = torch.empty(K, dtype=torch.float32, device=DEV)
+    acc_before = {n: PT.npy(acc[n]).copy() for n in rows}
+    sample_k = np.unique(np.linspace(0, K - 1, 4096).astype(np.int64))
+    cols = torch.from_numpy(ref_idx[sample_k].astype(np.int64)).to(DEV)
+    acc_cols = PT.npy(acc[:, cols])
+    ctx.mv_aggregate(acc, out_idx, out_val)
+    torch.cuda.synchronize()
+    want = O.aggregate(acc_cols, np.arange(acc_cols.shape[1]))
+    PT.check_out_val(PT.npy(out_val)[sample_k], want, acc_cols, np.arange(acc_cols.shape[1]), f"[{w.name}] out_val sample")
+    for n in rows:
+        want_row = O.residual(acc_before[n][None, :], ref_idx)[0]
+        PT.first_diff(PT.bits(PT.npy(acc[n])), PT.bits(want_row), f"[{w.name}] err row {n}")
+    assert int((acc[:, out_idx.long()].view(torch.int32) != 0).sum()) == 0, "residual not +0 on the mask"
+    # the fused step (run in place on err0) gives the same bytes as the phases
+    oi2 = torch.empty_like(out_idx)
+    ov2 = torch.empty_like(out_val)
+    ctx.mv_sparse_step(grads, err0, oi2, ov2)
+    torch.cuda.synchronize()
+    assert torch.equal(oi2, out_idx) and torch.equal(ov2.view(torch.int32), out_val.view(torch.int32))
+    assert torch.equal(err0.view(torch.int32), acc.view(torch.int32))
+    assert int(ctx.read_diag(N)[:, 2].sum()) == 0
