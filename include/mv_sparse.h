@@ -47,7 +47,8 @@ enum {
   MV_OK = 0,
   MV_ERR_INVALID_ARG = -1, /* null or misaligned pointer, N/d/K out of range, grads aliasing err */
   MV_ERR_WORKSPACE = -2,   /* workspace smaller than mv_workspace_bytes(N, d, K) */
-  MV_ERR_CUDA = -3         /* the CUDA runtime refused a launch or a copy */
+  MV_ERR_CUDA = -3,        /* the CUDA runtime refused a launch or a copy */
+  MV_ERR_TOO_LARGE = -4    /* mv_select_static only: d is larger than MV_SELECT_STATIC_MAX_D */
 };
 
 enum {
@@ -96,6 +97,34 @@ int mv_vote(mv_ctx* ctx, const float* grads, float* err, int N, int64_t d, int64
  *   mask_bits [ceil(d/32)]     out  the same set as a bit mask (may be NULL) */
 int mv_select(mv_ctx* ctx, const uint8_t* votes, int N, int64_t d, int64_t K,
               int32_t* out_idx, uint32_t* mask_bits);
+
+/* mv_select for callers that cannot hand the library a workspace.  (The paper has no counterpart
+ * to this call: it is the same selection as mv_select, packaged differently.)
+ *
+ * Who needs it: code that runs where device memory may not be allocated -- inside a region that
+ * the application has closed to cudaMalloc (a real-time loop, a plug-in whose host forbids
+ * allocation after start-up, a process whose memory pool is already fully handed out) -- and that
+ * therefore has no buffer of mv_workspace_bytes() to give to mv_create.  This call needs neither a
+ * context nor a workspace and calls no allocating routine: its scratch space is an array compiled
+ * into the library, about 2.2 MB, which every GPU that loads the library holds until the process
+ * ends.  The caller still owns and passes the input and the outputs.
+ *
+ *   stream    cudaStream_t to enqueue on (NULL = default stream)
+ *   votes     [d] uint8        in   every value must be <= N
+ *   out_idx   [K]              out  ascending
+ *   mask_bits [ceil(d/32)]     out  the same set as a bit mask (may be NULL)
+ *
+ * Limits: d <= MV_SELECT_STATIC_MAX_D (the array is sized for that; a larger d returns
+ * MV_ERR_TOO_LARGE and nothing is enqueued); N and K as for mv_select.
+ * First use: the first call on each device looks up the array's device address (with that device
+ * current) and remembers it; make that first call outside any stream capture.
+ * Sharing: all calls in the process use the one array, which keeps what the previous call left;
+ * the call itself clears the parts that must start at zero.  Two calls whose kernels overlap on
+ * the GPU (different streams without an ordering between them) would race on the array: order
+ * them.  Results are identical to mv_select's. */
+#define MV_SELECT_STATIC_MAX_D (1 << 24)
+int mv_select_static(void* stream, const uint8_t* votes, int N, int64_t d, int64_t K,
+                     int32_t* out_idx, uint32_t* mask_bits);
 
 /* Sparse communication phase (Algorithm 1 from the masked send to the aggregate; Eq. 8).
  *   acc     [N*d] in/out  acc_n on entry, the residual on exit

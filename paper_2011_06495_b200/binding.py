@@ -20,6 +20,8 @@ MV_OK = 0
 MV_ERR_INVALID_ARG = -1
 MV_ERR_WORKSPACE = -2
 MV_ERR_CUDA = -3
+MV_ERR_TOO_LARGE = -4
+MV_SELECT_STATIC_MAX_D = 1 << 24
 MV_MODE_AUTO = 0
 MV_MODE_GENERAL = 1
 
@@ -57,6 +59,8 @@ def load() -> ctypes.CDLL:
     lib.mv_vote.argtypes = [c_vp, c_vp, c_vp, c_i, c_i64, c_i64, c_vp, c_vp, c_vp, c_vp]
     lib.mv_select.restype = c_i
     lib.mv_select.argtypes = [c_vp, c_vp, c_i, c_i64, c_i64, c_vp, c_vp]
+    lib.mv_select_static.restype = c_i
+    lib.mv_select_static.argtypes = [c_vp, c_vp, c_i, c_i64, c_i64, c_vp, c_vp]
     lib.mv_aggregate.restype = c_i
     lib.mv_aggregate.argtypes = [c_vp, c_vp, c_i, c_i64, c_i64, c_vp, c_vp]
     lib.mv_sparse_step_host.restype = c_i
@@ -94,6 +98,14 @@ def _ptr(t: Optional[torch.Tensor]):
 def _check(status: int, where: str):
     if status != MV_OK:
         raise MvError(status, where)
+
+
+def mv_select_static(votes, N: int, K: int, out_idx, mask_bits=None, stream: Optional[torch.cuda.Stream] = None):
+    """mv_select without a context or a workspace (scratch is an array built into the library);
+    for callers that may not allocate device memory.  d is limited to MV_SELECT_STATIC_MAX_D."""
+    st = stream if stream is not None else torch.cuda.current_stream(votes.device)
+    _check(load().mv_select_static(ctypes.c_void_p(st.cuda_stream), _ptr(votes), int(N), votes.numel(), int(K),
+                                   _ptr(out_idx), _ptr(mask_bits)), "mv_select_static")
 
 
 class MvContext:

@@ -1812,12 +1812,87 @@ int mv_read_diag(mv_ctx* ctx, int N, uint32_t* per_worker) {
 
 int mv_last_launches(const mv_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
+// ---------------------------------------------------------------------------------------------
+// mv_select_static: the shared-mask selection with its scratch in a fixed device array
+// ---------------------------------------------------------------------------------------------
+}  // extern "C" (reopened below)
+
+namespace {
+
+constexpr int64_t STATIC_MAX_D = (int64_t)MV_SELECT_STATIC_MAX_D;
+constexpr int STATIC_MAX_CHUNKS = (int)((STATIC_MAX_D + CH - 1) / CH);
+// fixed layout inside the array (offsets in bytes, each a multiple of 256)
+constexpr size_t ST_VOTES_DONE = 0;                                   // ticket counter, must start at zero
+constexpr size_t ST_VOTE_HIST = 256;                                  // 256 counters, must start at zero
+constexpr size_t ST_VSTATE = ST_VOTE_HIST + 256 * 4;
+constexpr size_t ST_OUT_BASE = ST_VSTATE + 256;
+constexpr size_t ST_TIE_TAKE = ST_OUT_BASE + (((size_t)STATIC_MAX_CHUNKS + 1) * 4 + 255) / 256 * 256;
+constexpr size_t ST_CHUNK_VH = ST_TIE_TAKE + ((size_t)STATIC_MAX_CHUNKS * 4 + 255) / 256 * 256;
+constexpr size_t ST_TOTAL = ST_CHUNK_VH + (size_t)256 * STATIC_MAX_CHUNKS * 2;
+
+// Lives in the module's image on every GPU that loads the library, until the process exits.
+static __device__ __align__(256) unsigned char g_select_scratch[ST_TOTAL];
+
+// In host code the name g_select_scratch is only a handle for the runtime, not a device address:
+// the address a kernel can use is asked for once per device and remembered here.
+constexpr int MAX_DEVICES = 64;
+unsigned char* g_select_scratch_addr[MAX_DEVICES] = {nullptr};
+
+int select_scratch_address(unsigned char** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return MV_ERR_CUDA;
+  if (g_select_scratch_addr[dev] == nullptr) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_select_scratch) != cudaSuccess || ptr == nullptr) return MV_ERR_CUDA;
+    g_select_scratch_addr[dev] = (unsigned char*)ptr;
+  }
+  *out = g_select_scratch_addr[dev];
+  return MV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int mv_select_static(void* stream, const uint8_t* votes, int N, int64_t d, int64_t K, int32_t* out_idx,
+                     uint32_t* mask_bits) {
+  if (!sizes_ok(N, d, K)) return MV_ERR_INVALID_ARG;
+  if (d > STATIC_MAX_D) return MV_ERR_TOO_LARGE;
+  if (votes == nullptr || out_idx == nullptr || !aligned16(votes) || !aligned16(out_idx)) return MV_ERR_INVALID_ARG;
+  if (mask_bits && !aligned16(mask_bits)) return MV_ERR_INVALID_ARG;
+  unsigned char* base = nullptr;
+  const int rc = select_scratch_address(&base);
+  if (rc != MV_OK) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  P p = {};
+  p.N = N;
+  p.nchunks = (int)((d + CH - 1) / CH);
+  p.nc_pad = (p.nchunks + 7) & ~7;
+  p.d = d;
+  p.K = K;
+  p.W = (d + 31) / 32;
+  p.votes_done = (uint32_t*)(base + ST_VOTES_DONE);
+  p.vote_hist = (uint32_t*)(base + ST_VOTE_HIST);
+  p.vstate = (uint32_t*)(base + ST_VSTATE);
+  p.out_base = (uint32_t*)(base + ST_OUT_BASE);
+  p.tie_take = (uint32_t*)(base + ST_TIE_TAKE);
+  p.chunk_vh = (uint16_t*)(base + ST_CHUNK_VH);
+  // the array keeps whatever the last call left: the ticket and the vote histogram start at zero
+  if (cudaMemsetAsync(base, 0, ST_VSTATE, st) != cudaSuccess) return MV_ERR_CUDA;
+  if (launch_k(k_vote_hist, dim3(p.nchunks), dim3(TPB), st, p, votes) != cudaSuccess) return MV_ERR_CUDA;
+  if (launch_k(k_vote_write, dim3(p.nchunks), dim3(TPB), st, p, votes, out_idx, mask_bits) != cudaSuccess)
+    return MV_ERR_CUDA;
+  if (cudaGetLastError() != cudaSuccess) return MV_ERR_CUDA;
+  return MV_OK;
+}
+
 const char* mv_status_string(int status) {
   switch (status) {
     case MV_OK: return "ok";
     case MV_ERR_INVALID_ARG: return "invalid argument (null or misaligned pointer, size out of range, or grads overlapping err)";
     case MV_ERR_WORKSPACE: return "workspace smaller than mv_workspace_bytes(N, d, K)";
     case MV_ERR_CUDA: return "the CUDA runtime reported an error";
+    case MV_ERR_TOO_LARGE: return "d exceeds MV_SELECT_STATIC_MAX_D, the size the built-in scratch array of mv_select_static was compiled for";
     default: return "unknown status";
   }
 }
