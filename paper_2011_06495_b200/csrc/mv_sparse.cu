@@ -9,9 +9,10 @@
 //                                             place, elements with key >= tau_n compacted per chunk
 //   select     k_hist<1..3>, k_count          exact K-th key T_n by radix select: on the candidates, or over
 //                                             the full row for a worker whose candidate count missed [K, cap]
-//   order      (tail of k_count), k_row_exact lowest-index tie quota per chunk; exact compaction for the
-//                                             full-row workers
-//   vote       k_set_bits, k_votes            per-worker bit masks, bit-sliced vote count
+//   order      (tail of k_count)              lowest-index tie quota per chunk, for workers whose threshold
+//                                             ties are only partly kept
+//   vote       k_set_bits, k_votes            per-worker bit masks (from the candidates, or from the row for a
+//                                             full-row worker), bit-sliced vote count
 //   lists      k_scan_sel, k_lists            ascending per-worker index lists from the masks (side stream)
 //   mask       (tail of k_votes), k_vote_write  counting select over vote values 0..N (k_vote_hist when
 //                                             votes come from the caller)
@@ -58,16 +59,15 @@ struct P {
   uint8_t* hot;           // [nc_pad] 1 if any worker kept a candidate in the chunk
   uint32_t* vote_hist;    // [256]
   uint32_t* tau;          // [N]
+  uint32_t* diag_cnt;     // [N] copy of cand_cnt that survives the end-of-step clearing
   uint32_t* wstate;       // [N][8]: b1, rem1, b2, rem2, T, cnt_gt, cnt_eq, need
   uint32_t* thresh;       // [N][3]
   uint32_t* vstate;       // [4]: v*, cnt_gt, cnt_eq, quota
   uint2* cand;            // [N][cap] (key, index)
   uint32_t* chunk_base;   // [N][nchunks]
   uint32_t* chunk_cnt;
-  uint32_t* chunk_gt;
   uint32_t* chunk_eq;
   uint32_t* tie_base;
-  uint32_t* sel_base;
   uint32_t* chunk_sel;    // [N][nchunks] selected elements per chunk
   uint32_t* worker_bits;  // [N][W]
   int32_t* worker_idx;    // [N][K]
@@ -304,6 +304,18 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* s_w /*
   }
   total = tot;
   return base + x - v;
+}
+
+// ticket: true in every thread of the last CTA of the grid to call it (all threads must call)
+__device__ __forceinline__ bool last_cta(uint32_t* counter, uint32_t total) {
+  __shared__ uint32_t s_last_flag;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) s_last_flag = (atomicAdd(counter, 1u) == total - 1) ? 1u : 0u;
+  __syncthreads();
+  const bool last = s_last_flag != 0;
+  if (last) __threadfence();
+  return last;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -578,11 +590,11 @@ __global__ void __launch_bounds__(TPB) k_hist(P p, const float* __restrict__ gra
 }
 
 // ---------------------------------------------------------------------------------------------
-// order: per worker, running count of threshold ties before each chunk (tie_base) and of selected
-// elements before each chunk (sel_base), given the quota `need` of ties to keep, lowest index first
+// order: per worker, the number of threshold ties before each chunk (tie_base); a tie is kept if
+// its rank in index order is below the worker's quota
 // ---------------------------------------------------------------------------------------------
 template <int NT>
-__device__ void chunk_scan(const P& p, int n, uint32_t need, bool fast) {
+__device__ void chunk_scan(const P& p, int n) {
   __shared__ uint32_t s_w[NT / 32 + 1];
   const int per = (p.nchunks + NT - 1) / NT;
   const int c0 = min(p.nchunks, (int)threadIdx.x * per), c1 = min(p.nchunks, c0 + per);
@@ -590,42 +602,25 @@ __device__ void chunk_scan(const P& p, int n, uint32_t need, bool fast) {
   uint32_t esum = 0;
   for (int c = c0; c < c1; c++) esum += __ldcg(p.chunk_eq + rb + c);
   uint32_t tot;
-  const uint32_t epre = block_excl_scan<NT>(esum, s_w, tot);
-  uint32_t run = epre, ssum = 0;
+  uint32_t run = block_excl_scan<NT>(esum, s_w, tot);
   for (int c = c0; c < c1; c++) {
-    const uint32_t eq = __ldcg(p.chunk_eq + rb + c);
-    const uint32_t take = run >= need ? 0u : min(eq, need - run);
     p.tie_base[rb + c] = run;
-    run += eq;
-    if (!fast) ssum += __ldcg(p.chunk_gt + rb + c) + take;
-  }
-  if (fast) return;  // a fast worker only needs tie_base (uniform over the CTA)
-  const uint32_t spre = block_excl_scan<NT>(ssum, s_w, tot);
-  run = epre;
-  uint32_t srun = spre;
-  for (int c = c0; c < c1; c++) {
-    const uint32_t eq = __ldcg(p.chunk_eq + rb + c);
-    const uint32_t take = run >= need ? 0u : min(eq, need - run);
-    p.sel_base[rb + c] = srun;
-    run += eq;
-    srun += __ldcg(p.chunk_gt + rb + c) + take;
+    run += __ldcg(p.chunk_eq + rb + c);
   }
 }
 
-// Resolves T_n for every worker, then counts per chunk what the ordering needs:
-//   - a fast worker that keeps all of its threshold ties needs nothing here;
-//   - a fast worker that keeps only some of them needs the ties per chunk (from its candidates);
-//   - any other worker needs, from its full row, the elements above and at the threshold per chunk.
+// Resolves T_n for every worker.  A worker that keeps only part of its threshold ties also needs
+// the ties per chunk: counted from its candidates, or from its full row; the last CTA of the worker
+// to finish turns the counts into running offsets.
 __global__ void __launch_bounds__(TPB) k_count(P p, float* __restrict__ err) {
   pdl_enter();
-  __shared__ uint32_t s_g[TPB / 32], s_e[TPB / 32];
-  __shared__ uint32_t s_last;
+  __shared__ uint32_t s_e[TPB / 32];
   const int n = blockIdx.y;
   uint32_t need, cnt_eq;
   const uint32_t T = resolve_threshold(p, n, need, cnt_eq);
+  if (need >= cnt_eq) return;  // every tie is kept: no order needed (uniform over the worker's CTAs)
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (worker_fast(p, n)) {
-    if (need >= cnt_eq) return;  // every tie is kept: no order needed
     const uint2* cd = p.cand + (size_t)n * p.cap;
     for (int c = blockIdx.x * (TPB / 32) + warp; c < p.nchunks; c += gridDim.x * (TPB / 32)) {
       const size_t ci = (size_t)n * p.nchunks + c;
@@ -636,160 +631,30 @@ __global__ void __launch_bounds__(TPB) k_count(P p, float* __restrict__ err) {
       if (lane == 0) p.chunk_eq[ci] = eq;
     }
   } else {
-  for (int c = blockIdx.x; c < p.nchunks; c += gridDim.x) {
-    const Geom g = chunk_geom(n, c, p.d);
-    uint32_t key[4][4], vm[4];
-    load_keys<false>(g, nullptr, err, key, vm);
-    uint32_t gt = 0, eq = 0;
+    for (int c = blockIdx.x; c < p.nchunks; c += gridDim.x) {
+      const Geom g = chunk_geom(n, c, p.d);
+      uint32_t key[4][4], vm[4];
+      load_keys<false>(g, nullptr, err, key, vm);
+      uint32_t eq = 0;
 #pragma unroll
-    for (int i = 0; i < 4; i++) {
-      gt += __popc(vm[i] & gt_mask(key[i], T));
-      eq += __popc(vm[i] & eq_mask(key[i], T));
-    }
-    if (threadIdx.x == TPB - 1) {
-      uint32_t xkey[4], xvm;
-      load_extra<false>(g, nullptr, err, xkey, xvm);
-      gt += __popc(xvm & gt_mask(xkey, T));
-      eq += __popc(xvm & eq_mask(xkey, T));
-    }
-    gt = __reduce_add_sync(FULL, gt);
-    eq = __reduce_add_sync(FULL, eq);
-    __syncthreads();
-    if (lane == 0) {
-      s_g[warp] = gt;
-      s_e[warp] = eq;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      uint32_t tg = 0, te = 0;
-      for (int w = 0; w < TPB / 32; w++) {
-        tg += s_g[w];
-        te += s_e[w];
+      for (int i = 0; i < 4; i++) eq += __popc(vm[i] & eq_mask(key[i], T));
+      if (threadIdx.x == TPB - 1) {
+        uint32_t xkey[4], xvm;
+        load_extra<false>(g, nullptr, err, xkey, xvm);
+        eq += __popc(xvm & eq_mask(xkey, T));
       }
-      p.chunk_gt[(size_t)n * p.nchunks + c] = tg;
-      p.chunk_eq[(size_t)n * p.nchunks + c] = te;
+      eq = __reduce_add_sync(FULL, eq);
+      __syncthreads();
+      if (lane == 0) s_e[warp] = eq;
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        uint32_t te = 0;
+        for (int w = 0; w < TPB / 32; w++) te += s_e[w];
+        p.chunk_eq[(size_t)n * p.nchunks + c] = te;
+      }
     }
   }
-  }
-  // the last CTA of this worker to get here turns the per-chunk counts into running offsets
-  __threadfence();
-  __syncthreads();
-  if (threadIdx.x == 0) s_last = (atomicAdd(&p.count_done[n], 1u) == gridDim.x - 1) ? 1u : 0u;
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
-  chunk_scan<TPB>(p, n, need, worker_fast(p, n));
-}
-
-// exact compaction: writes precisely the selected elements of each chunk, in index order, at the
-// chunk's list offset (so the candidate buffer of such a worker holds its K picks, sorted)
-__global__ void __launch_bounds__(TPB) k_row_exact(P p, float* __restrict__ err) {
-  pdl_enter();
-  __shared__ uint32_t s_we[9], s_ws[9];
-  const int n = blockIdx.y;
-  if (worker_fast(p, n)) return;
-  const uint32_t* ws = p.wstate + (size_t)n * 8;
-  const uint32_t T = ws[4], need = ws[7];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t lt = lanemask_lt();
-  uint2* out = p.cand + (size_t)n * p.cap;
-  for (int c = blockIdx.x; c < p.nchunks; c += gridDim.x) {
-    const size_t ci = (size_t)n * p.nchunks + c;
-    const Geom g = chunk_geom(n, c, p.d);
-    uint32_t key[4][4], vm[4], em[4], sm[4];
-    load_keys<false>(g, nullptr, err, key, vm);
-    uint32_t xkey[4], xvm = 0, xem = 0, xsm = 0;
-    if (threadIdx.x == TPB - 1) {
-      load_extra<false>(g, nullptr, err, xkey, xvm);
-      xem = xvm & eq_mask(xkey, T);
-    }
-    uint32_t weq = 0;
-#pragma unroll
-    for (int i = 0; i < 4; i++) {
-      em[i] = vm[i] & eq_mask(key[i], T);
-      weq += __popc(em[i]);
-    }
-    weq = __reduce_add_sync(FULL, weq);
-    __syncthreads();  // previous chunk's readers of s_we / s_ws are done
-    if (lane == 0) s_we[warp] = weq;
-    if (threadIdx.x == TPB - 1) s_we[8] = __popc(xem);
-    __syncthreads();
-    const uint32_t tb = p.tie_base[ci];
-    uint32_t eoff = tb;
-    for (int w = 0; w < warp; w++) eoff += s_we[w];
-    uint32_t wsel = 0;
-#pragma unroll
-    for (int i = 0; i < 4; i++) {
-      uint32_t rank0, tot;
-      iter_ranks(em[i], lt, rank0, tot);
-      uint32_t take = 0;
-#pragma unroll
-      for (int e = 0; e < 4; e++) {
-        if (em[i] & (1u << e)) {
-          const uint32_t r = eoff + rank0 + __popc(em[i] & ((1u << e) - 1u));
-          if (r < need) take |= 1u << e;
-        }
-      }
-      sm[i] = (vm[i] & gt_mask(key[i], T)) | take;
-      wsel += __popc(sm[i]);
-      eoff += tot;
-    }
-    if (threadIdx.x == TPB - 1) {
-      uint32_t xoff = tb;
-      for (int w = 0; w < 8; w++) xoff += s_we[w];
-      uint32_t take = 0;
-#pragma unroll
-      for (int e = 0; e < 4; e++) {
-        if (xem & (1u << e)) {
-          const uint32_t r = xoff + __popc(xem & ((1u << e) - 1u));
-          if (r < need) take |= 1u << e;
-        }
-      }
-      xsm = (xvm & gt_mask(xkey, T)) | take;
-    }
-    wsel = __reduce_add_sync(FULL, wsel);
-    if (lane == 0) s_ws[warp] = wsel;
-    if (threadIdx.x == TPB - 1) s_ws[8] = __popc(xsm);
-    __syncthreads();
-    const uint32_t sb = p.sel_base[ci];
-    uint32_t soff = sb;
-    for (int w = 0; w < warp; w++) soff += s_ws[w];
-#pragma unroll
-    for (int i = 0; i < 4; i++) {
-      uint32_t rank0, tot;
-      iter_ranks(sm[i], lt, rank0, tot);
-      if (sm[i]) {
-        const int jf = g.j0 - g.h + 4 * (warp * 128 + i * 32 + lane);
-#pragma unroll
-        for (int e = 0; e < 4; e++) {
-          if (sm[i] & (1u << e)) {
-            const uint32_t pos = soff + rank0 + __popc(sm[i] & ((1u << e) - 1u));
-            if (pos < p.cap) out[pos] = make_uint2(key[i][e], (uint32_t)(jf + e));
-          }
-        }
-      }
-      soff += tot;
-    }
-    if (threadIdx.x == TPB - 1 && xsm) {
-      uint32_t xoff = sb;
-      for (int w = 0; w < 8; w++) xoff += s_ws[w];
-      const int jf = g.j0 - g.h + 4096;
-#pragma unroll
-      for (int e = 0; e < 4; e++) {
-        if (xsm & (1u << e)) {
-          const uint32_t pos = xoff + __popc(xsm & ((1u << e) - 1u));
-          if (pos < p.cap) out[pos] = make_uint2(xkey[e], (uint32_t)(jf + e));
-        }
-      }
-    }
-    if (threadIdx.x == 0) {
-      uint32_t tot = 0;
-      for (int w = 0; w < 9; w++) tot += s_ws[w];
-      p.chunk_base[ci] = sb;
-      p.chunk_cnt[ci] = tot;
-      if (tot) p.hot[c] = 1;
-    }
-  }
+  if (last_cta(p.count_done + n, gridDim.x)) chunk_scan<TPB>(p, n);
 }
 
 // v* = the vote value of the K-th most voted coordinate; then per chunk the output offset and the
@@ -871,18 +736,6 @@ __device__ void vote_scan(const P& p) {
   if (threadIdx.x == 0) p.out_base[p.nchunks] = (uint32_t)p.K;  // sentinel: end of the last chunk
 }
 
-// ticket: true in every thread of the last CTA of the grid to call it (all threads must call)
-__device__ __forceinline__ bool last_cta(uint32_t* counter, uint32_t total) {
-  __shared__ uint32_t s_last_flag;
-  __threadfence();
-  __syncthreads();
-  if (threadIdx.x == 0) s_last_flag = (atomicAdd(counter, 1u) == total - 1) ? 1u : 0u;
-  __syncthreads();
-  const bool last = s_last_flag != 0;
-  if (last) __threadfence();
-  return last;
-}
-
 // s_vh[v] (v >= 1) holds how many coordinates of chunk c got exactly v votes.  Stores, per chunk,
 // the cumulative counts cum[v] = #{votes >= v} (v = 0..N) and adds the exact counts to the global
 // histogram.  All threads of the CTA call it.
@@ -912,16 +765,101 @@ __device__ __forceinline__ void store_vote_hist_impl(const P& p, int c, uint32_t
 // part of their threshold ties add those, lowest index first.  (3) k_votes: one CTA per chunk adds
 // the N masks bit-sliced (8 counter planes per 32-coordinate word) into the vote count.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(TPB) k_set_bits(P p) {
+__global__ void __launch_bounds__(TPB) k_set_bits(P p, float* __restrict__ err) {
   pdl_enter();
+  __shared__ uint32_t s_we[9];
   const int n = blockIdx.y;
   const bool fast = worker_fast(p, n);
   const uint32_t* ws = p.wstate + (size_t)n * 8;
   const uint32_t T = ws[4], need = ws[7];
   const bool all_ties = need >= ws[6];
-  const uint32_t cnt = fast ? p.cand_cnt[n] : (uint32_t)p.K;  // a full-row worker's buffer holds exactly its picks
-  const uint2* cd = p.cand + (size_t)n * p.cap;               // cap is a multiple of 8: rows are 64-byte aligned
   uint32_t* bits_row = p.worker_bits + (size_t)n * p.W;
+  if (blockIdx.x == 0 && threadIdx.x == 0) p.diag_cnt[n] = p.cand_cnt[n];
+  if (!fast) {
+    // full-row worker: its picks are read off the row itself (err holds acc), chunk by chunk
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t lt = lanemask_lt();
+    for (int c = blockIdx.x; c < p.nchunks; c += gridDim.x) {
+      const Geom g = chunk_geom(n, c, p.d);
+      uint32_t key[4][4], vm[4], em[4], sm[4];
+      load_keys<false>(g, nullptr, err, key, vm);
+      uint32_t xkey[4], xvm = 0, xem = 0, xsm = 0;
+      if (threadIdx.x == TPB - 1) {
+        load_extra<false>(g, nullptr, err, xkey, xvm);
+        xem = xvm & eq_mask(xkey, T);
+      }
+#pragma unroll
+      for (int i = 0; i < 4; i++) em[i] = vm[i] & eq_mask(key[i], T);
+      if (all_ties) {
+#pragma unroll
+        for (int i = 0; i < 4; i++) sm[i] = (vm[i] & gt_mask(key[i], T)) | em[i];
+        if (threadIdx.x == TPB - 1) xsm = (xvm & gt_mask(xkey, T)) | xem;
+      } else {
+        // keep the threshold ties whose rank (in index order, over the whole row) is below `need`
+        uint32_t weq = 0;
+#pragma unroll
+        for (int i = 0; i < 4; i++) weq += __popc(em[i]);
+        weq = __reduce_add_sync(FULL, weq);
+        __syncthreads();  // previous chunk's readers of s_we are done
+        if (lane == 0) s_we[warp] = weq;
+        if (threadIdx.x == TPB - 1) s_we[8] = __popc(xem);
+        __syncthreads();
+        const uint32_t tb = p.tie_base[(size_t)n * p.nchunks + c];
+        uint32_t eoff = tb;
+        for (int w = 0; w < warp; w++) eoff += s_we[w];
+#pragma unroll
+        for (int i = 0; i < 4; i++) {
+          uint32_t rank0, tot;
+          iter_ranks(em[i], lt, rank0, tot);
+          uint32_t take = 0;
+#pragma unroll
+          for (int e = 0; e < 4; e++) {
+            if (em[i] & (1u << e)) {
+              const uint32_t r = eoff + rank0 + __popc(em[i] & ((1u << e) - 1u));
+              if (r < need) take |= 1u << e;
+            }
+          }
+          sm[i] = (vm[i] & gt_mask(key[i], T)) | take;
+          eoff += tot;
+        }
+        if (threadIdx.x == TPB - 1) {
+          uint32_t xoff = tb;
+          for (int w = 0; w < 8; w++) xoff += s_we[w];
+          uint32_t take = 0;
+#pragma unroll
+          for (int e = 0; e < 4; e++) {
+            if (xem & (1u << e)) {
+              const uint32_t r = xoff + __popc(xem & ((1u << e) - 1u));
+              if (r < need) take |= 1u << e;
+            }
+          }
+          xsm = (xvm & gt_mask(xkey, T)) | take;
+        }
+      }
+      bool any = false;
+#pragma unroll
+      for (int i = 0; i < 4; i++) {
+        if (sm[i]) {
+          any = true;
+          const int jf = g.j0 - g.h + 4 * (warp * 128 + i * 32 + lane);
+#pragma unroll
+          for (int e = 0; e < 4; e++)
+            if (sm[i] & (1u << e)) atomicOr(bits_row + ((uint32_t)(jf + e) >> 5), 1u << ((uint32_t)(jf + e) & 31u));
+        }
+      }
+      if (xsm) {
+        any = true;
+        const int jf = g.j0 - g.h + 4096;
+#pragma unroll
+        for (int e = 0; e < 4; e++)
+          if (xsm & (1u << e)) atomicOr(bits_row + ((uint32_t)(jf + e) >> 5), 1u << ((uint32_t)(jf + e) & 31u));
+      }
+      if (any) p.hot[c] = 1;  // same value from every thread
+    }
+    return;
+  }
+  const uint32_t cnt = p.cand_cnt[n];
+  const uint2* cd = p.cand + (size_t)n * p.cap;  // cap is a multiple of 8: rows are 64-byte aligned
   for (uint32_t i0 = (blockIdx.x * TPB + threadIdx.x) * 8u; i0 < cnt; i0 += gridDim.x * TPB * 8u) {
     uint4 v[4];
 #pragma unroll
@@ -931,7 +869,7 @@ __global__ void __launch_bounds__(TPB) k_set_bits(P p) {
     for (int q = 0; q < 8; q++) {
       const uint32_t key = (q & 1) ? v[q >> 1].z : v[q >> 1].x;
       const uint32_t j = (q & 1) ? v[q >> 1].w : v[q >> 1].y;
-      const bool sel = i0 + q < cnt && (!fast || key > T || (key == T && all_ties));
+      const bool sel = i0 + q < cnt && (key > T || (key == T && all_ties));
       if (sel && (int64_t)j < p.d) {
         const uint32_t w = j >> 5;
         if (w != curw) {
@@ -945,7 +883,7 @@ __global__ void __launch_bounds__(TPB) k_set_bits(P p) {
     if (acc) atomicOr(bits_row + curw, acc);
   }
   // a worker that keeps only part of its threshold ties adds them chunk by chunk, lowest index first
-  if (!fast || all_ties) return;
+  if (all_ties) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t lt = lanemask_lt();
   for (int c = blockIdx.x * (TPB / 32) + warp; c < p.nchunks; c += gridDim.x * (TPB / 32)) {
@@ -1226,9 +1164,14 @@ __global__ void __launch_bounds__(TPB) k_vote_write(P p, const uint8_t* __restri
 // ---------------------------------------------------------------------------------------------
 // aggregate: out_val[k] = fl32( (sum_n (double)acc[n][idx[k]]) / N ), then acc[n][idx[k]] = +0
 // ---------------------------------------------------------------------------------------------
+// The last kernel of a whole step also clears the leading scratch region (counters and histograms)
+// so that the next step can start without a separate memset; zero_vecs = 0 switches that off.
 __global__ void __launch_bounds__(TPB) k_gather(float* __restrict__ acc, int N, int64_t d, int64_t K,
-                                                const int32_t* __restrict__ idx, float* __restrict__ out_val) {
+                                                const int32_t* __restrict__ idx, float* __restrict__ out_val,
+                                                uint4* __restrict__ zero_ptr, uint32_t zero_vecs) {
   pdl_enter();
+  for (uint32_t i = blockIdx.x * TPB + threadIdx.x; i < zero_vecs; i += gridDim.x * TPB)
+    zero_ptr[i] = make_uint4(0, 0, 0, 0);
   const int64_t k = (int64_t)blockIdx.x * TPB + threadIdx.x;
   if (k >= K) return;
   const int64_t j = idx[k];
@@ -1261,7 +1204,7 @@ struct Layout {
   uint32_t cap;
   size_t zero_bytes;  // the leading region cleared at the start of every vote
   size_t samp_hist, hist1, hist2, hist3, cand_cnt, sample_done, count_done, votes_done, hot, vote_hist;
-  size_t tau, wstate, thresh, vstate, cand, chunk_base, chunk_cnt, chunk_gt, chunk_eq, tie_base, sel_base, chunk_sel;
+  size_t tau, diag_cnt, wstate, thresh, vstate, cand, chunk_base, chunk_cnt, chunk_eq, tie_base, chunk_sel;
   size_t worker_bits, worker_idx, votes, chunk_vh, out_base, tie_take;
   size_t total;
 };
@@ -1297,16 +1240,15 @@ Layout make_layout(int N, int64_t d, int64_t K) {
   L.vote_hist = take(off, 256 * 4);
   L.zero_bytes = off;
   L.tau = take(off, n * 4);
+  L.diag_cnt = take(off, n * 4);
   L.wstate = take(off, n * 8 * 4);
   L.thresh = take(off, n * 3 * 4);
   L.vstate = take(off, 4 * 4);
   L.cand = take(off, n * (size_t)L.cap * 8);
   L.chunk_base = take(off, n * nc * 4);
   L.chunk_cnt = take(off, n * nc * 4);
-  L.chunk_gt = take(off, n * nc * 4);
   L.chunk_eq = take(off, n * nc * 4);
   L.tie_base = take(off, n * nc * 4);
-  L.sel_base = take(off, n * nc * 4);
   L.chunk_sel = take(off, n * nc * 4);
   L.worker_bits = take(off, n * (size_t)L.W * 4);
   L.worker_idx = take(off, n * (size_t)K * 4);
@@ -1344,6 +1286,7 @@ struct mv_ctx {
   int phase_timing;
   cudaEvent_t pev[48];
   bool pev_made;
+  size_t clean_bytes;  // leading workspace bytes known to be zero (left so by the previous whole step)
   // remembered for mv_read_diag
   int last_N;
   int64_t last_d, last_K;
@@ -1373,16 +1316,15 @@ P make_params(const mv_ctx* ctx, const Layout& L, int N, int64_t d, int64_t K) {
   p.hot = (uint8_t*)(b + L.hot);
   p.vote_hist = (uint32_t*)(b + L.vote_hist);
   p.tau = (uint32_t*)(b + L.tau);
+  p.diag_cnt = (uint32_t*)(b + L.diag_cnt);
   p.wstate = (uint32_t*)(b + L.wstate);
   p.thresh = (uint32_t*)(b + L.thresh);
   p.vstate = (uint32_t*)(b + L.vstate);
   p.cand = (uint2*)(b + L.cand);
   p.chunk_base = (uint32_t*)(b + L.chunk_base);
   p.chunk_cnt = (uint32_t*)(b + L.chunk_cnt);
-  p.chunk_gt = (uint32_t*)(b + L.chunk_gt);
   p.chunk_eq = (uint32_t*)(b + L.chunk_eq);
   p.tie_base = (uint32_t*)(b + L.tie_base);
-  p.sel_base = (uint32_t*)(b + L.sel_base);
   p.chunk_sel = (uint32_t*)(b + L.chunk_sel);
   p.worker_bits = (uint32_t*)(b + L.worker_bits);
   p.worker_idx = (int32_t*)(b + L.worker_idx);
@@ -1477,7 +1419,9 @@ int vote_impl(mv_ctx* ctx, P p, const Layout& L, const float* grads, float* err)
   cudaStream_t st = ctx->stream;
   const int N = p.N;
   ctx->timing_now = ctx->timing > 0 && (ctx->timing_calls++ % ctx->timing) == 0;
-  if (cudaMemsetAsync(ctx->ws, 0, L.zero_bytes, st) != cudaSuccess) return MV_ERR_CUDA;
+  if (ctx->clean_bytes < L.zero_bytes && cudaMemsetAsync(ctx->ws, 0, L.zero_bytes, st) != cudaSuccess)
+    return MV_ERR_CUDA;
+  ctx->clean_bytes = 0;  // dirty from here on, until a whole step's last kernel has cleared it again
   // per-chunk outputs of the vote count start out cleared (only chunks with candidates are
   // visited later); cleared on the side stream, concurrently with the sampling and streaming pass
   cudaStream_t zs = st;
@@ -1520,10 +1464,8 @@ int vote_impl(mv_ctx* ctx, P p, const Layout& L, const float* grads, float* err)
   MV_LAUNCH_CHECK();
   launch_k(k_count, dim3(dim3(gh, N)), dim3(TPB), st, p, err);
   MV_LAUNCH_CHECK();
-  launch_k(k_row_exact, dim3(dim3(gh, N)), dim3(TPB), st, p, err);
-  MV_LAUNCH_CHECK();
-  const int gb = per_row_ctas(N, (int)((p.cap + TPB * 16 - 1) / (TPB * 16)), 148 * 4);
-  launch_k(k_set_bits, dim3(dim3(gb, N)), dim3(TPB), st, p);
+  const int gb = p.force_general ? gh : per_row_ctas(N, (int)((p.cap + TPB * 16 - 1) / (TPB * 16)), 148 * 4);
+  launch_k(k_set_bits, dim3(dim3(gb, N)), dim3(TPB), st, p, err);
   MV_LAUNCH_CHECK();
   if (zs != st && cudaStreamWaitEvent(st, ctx->ev_zero, 0) != cudaSuccess) return MV_ERR_CUDA;
   {
@@ -1555,6 +1497,7 @@ int select_impl(mv_ctx* ctx, P p, const Layout& L, const uint8_t* votes, bool ha
                 uint32_t* mask_bits) {
   cudaStream_t st = ctx->stream;
   if (!have_hist) {
+    ctx->clean_bytes = 0;
     if (cudaMemsetAsync(ctx->ws + L.votes_done, 0, L.zero_bytes - L.votes_done, st) != cudaSuccess) return MV_ERR_CUDA;
     launch_k(k_vote_hist, dim3(p.nchunks), dim3(TPB), st, p, votes);
     MV_LAUNCH_CHECK();
@@ -1565,9 +1508,12 @@ int select_impl(mv_ctx* ctx, P p, const Layout& L, const uint8_t* votes, bool ha
 }
 
 // steps a5-a6
-int aggregate_impl(mv_ctx* ctx, float* acc, int N, int64_t d, int64_t K, const int32_t* idx, float* out_val) {
-  launch_k(k_gather, dim3((unsigned)((K + TPB - 1) / TPB)), dim3(TPB), ctx->stream, acc, N, d, K, idx, out_val);
+int aggregate_impl(mv_ctx* ctx, float* acc, int N, int64_t d, int64_t K, const int32_t* idx, float* out_val,
+                   size_t clear_bytes) {
+  launch_k(k_gather, dim3((unsigned)((K + TPB - 1) / TPB)), dim3(TPB), ctx->stream, acc, N, d, K, idx, out_val,
+           (uint4*)ctx->ws, (uint32_t)(clear_bytes / 16));
   MV_LAUNCH_CHECK();
+  if (clear_bytes) ctx->clean_bytes = clear_bytes;
   return MV_OK;
 }
 
@@ -1604,6 +1550,7 @@ int mv_create(mv_ctx** out, void* stream, void* workspace, size_t workspace_byte
   c->ws_bytes = workspace_bytes;
   c->mode = MV_MODE_AUTO;
   c->launches = 0;
+  c->clean_bytes = 0;
   c->timing = 0;
   c->timing_calls = 0;
   c->timing_now = false;
@@ -1740,7 +1687,7 @@ int mv_aggregate(mv_ctx* ctx, float* acc, int N, int64_t d, int64_t K, const int
     return MV_ERR_INVALID_ARG;
   ctx->launches = 0;
   if (ctx->phase_timing) cudaEventRecord(ctx->pev[0], ctx->stream);
-  return aggregate_impl(ctx, acc, N, d, K, idx, out_val);
+  return aggregate_impl(ctx, acc, N, d, K, idx, out_val, 0);
 }
 
 int mv_sparse_step(mv_ctx* ctx, const float* grads, float* err, int N, int64_t d, int64_t K, int32_t* out_idx,
@@ -1760,7 +1707,7 @@ int mv_sparse_step(mv_ctx* ctx, const float* grads, float* err, int N, int64_t d
   ctx->last_K = K;
   rc = vote_impl(ctx, p, L, grads, err);
   if (rc == MV_OK) rc = select_impl(ctx, p, L, p.votes, true, out_idx, nullptr);
-  if (rc == MV_OK) rc = aggregate_impl(ctx, err, N, d, K, out_idx, out_val);
+  if (rc == MV_OK) rc = aggregate_impl(ctx, err, N, d, K, out_idx, out_val, L.zero_bytes);
   const int rcj = join_side(ctx);
   return rc != MV_OK ? rc : rcj;
 }
@@ -1792,7 +1739,7 @@ int mv_read_diag(mv_ctx* ctx, int N, uint32_t* per_worker) {
   uint32_t* cnt = (uint32_t*)malloc((size_t)N * 8);
   if (cnt == nullptr) return MV_ERR_INVALID_ARG;
   uint32_t* tau = cnt + N;
-  cudaError_t e = cudaMemcpyAsync(cnt, ctx->ws + L.cand_cnt, (size_t)N * 4, cudaMemcpyDeviceToHost, ctx->stream);
+  cudaError_t e = cudaMemcpyAsync(cnt, ctx->ws + L.diag_cnt, (size_t)N * 4, cudaMemcpyDeviceToHost, ctx->stream);
   if (e == cudaSuccess) e = cudaMemcpyAsync(tau, ctx->ws + L.tau, (size_t)N * 4, cudaMemcpyDeviceToHost, ctx->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
   if (e != cudaSuccess) {
