@@ -157,12 +157,15 @@ int mv_read_diag(mv_ctx* ctx, int N, uint32_t* per_worker);
 int mv_set_kernel_timing(mv_ctx* ctx, int every);
 int mv_read_kernel_timing(mv_ctx* ctx, float* total_ms, int* launches);
 
-/* Optional per-launch timing of a whole call, for profiling without an external tool: while
- * enabled, a CUDA event is recorded before the first and after every kernel launch of each call
- * (the events themselves cost a little time).  mv_read_phase_times waits for the stream and
- * returns, for the last call, the elapsed milliseconds between consecutive events: ms[i] covers
- * the i-th kernel in launch order (Algorithm 1's steps in the order listed at the top of this
- * file).  At most `capacity` values (and at most 47) are written; *count gets their number. */
+/* Optional per-launch timing of a whole call, for profiling without an external tool.
+ * enable = 1: a CUDA event is recorded before the first and after every kernel launch of each call
+ * (the events serialise the kernels, so the parts add up to more than the undisturbed call);
+ * mv_read_phase_times then returns, for the last call, the milliseconds between consecutive
+ * events: ms[i] covers the i-th kernel in launch order (Algorithm 1's steps in the order listed at
+ * the top of this file), at most `capacity` (and 47) values, *count their number.
+ * enable = 100 + i: only two events, before the first launch and after the i-th (1-based), which
+ * disturbs the call far less; mv_read_phase_times returns that one interval in ms[0].
+ * enable = 0: off.  While on, all work of a call stays on the context's stream. */
 int mv_set_phase_timing(mv_ctx* ctx, int enable);
 int mv_read_phase_times(mv_ctx* ctx, float* ms, int capacity, int* count);
 

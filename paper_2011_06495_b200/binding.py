@@ -186,8 +186,9 @@ class MvContext:
                "mv_read_kernel_timing")
         return float(ms.value), int(cnt.value)
 
-    def set_phase_timing(self, enable: bool):
-        _check(self.lib.mv_set_phase_timing(self.handle, int(bool(enable))), "mv_set_phase_timing")
+    def set_phase_timing(self, enable: int):
+        """0: off; 1: an event after every launch; 100 + i: only the start and the end of launch i."""
+        _check(self.lib.mv_set_phase_timing(self.handle, int(enable)), "mv_set_phase_timing")
 
     def read_phase_times(self):
         """Milliseconds per kernel launch of the last call, in launch order."""

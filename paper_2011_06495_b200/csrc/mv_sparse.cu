@@ -1361,13 +1361,18 @@ int per_row_ctas(int N, int want, int budget) {
   do {                                                                                           \
     ctx->launches++;                                                                             \
     if (cudaGetLastError() != cudaSuccess) return MV_ERR_CUDA;                                   \
-    if (ctx->phase_timing && ctx->launches < 48) cudaEventRecord(ctx->pev[ctx->launches], ctx->stream); \
+    if ((ctx->phase_timing == 1 || ctx->phase_timing == 100 + ctx->launches) && ctx->launches < 48) \
+      cudaEventRecord(ctx->pev[ctx->launches], ctx->stream);                                     \
   } while (0)
 
 // sample size and rank for the threshold estimate
 void sample_plan(int64_t d, int64_t K, uint32_t& U, uint32_t& L, int& all, uint32_t& rank) {
-  int64_t S = d / 64;
-  if (S < 131072) S = 131072;
+  // sample size: d/256, but large enough that about 100 sampled elements lie above the K-th key
+  // (the bound's slack is a few standard deviations of that count), within [32 Ki, 1 Mi]
+  int64_t S = d / 256;
+  const int64_t s_min = (int64_t)(100.0 * (double)d / (double)K);
+  if (S < s_min) S = s_min;
+  if (S < 32768) S = 32768;
   if (S > (1 << 20)) S = 1 << 20;
   if (d <= 2 * S) {
     all = 1;
@@ -1425,7 +1430,7 @@ int vote_impl(mv_ctx* ctx, P p, const Layout& L, const float* grads, float* err)
   // per-chunk outputs of the vote count start out cleared (only chunks with candidates are
   // visited later); cleared on the side stream, concurrently with the sampling and streaming pass
   cudaStream_t zs = st;
-  if (!ctx->phase_timing && side_ready(ctx) && cudaEventRecord(ctx->ev_fork, st) == cudaSuccess &&
+  if (ctx->phase_timing != 1 && side_ready(ctx) && cudaEventRecord(ctx->ev_fork, st) == cudaSuccess &&
       cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) == cudaSuccess)
     zs = ctx->side;
   {
@@ -1478,7 +1483,7 @@ int vote_impl(mv_ctx* ctx, P p, const Layout& L, const float* grads, float* err)
   MV_LAUNCH_CHECK();
   // the index lists feed nothing later in the step: write them on the side stream
   cudaStream_t ls = st;
-  if (!ctx->phase_timing && side_ready(ctx) && cudaEventRecord(ctx->ev_fork, st) == cudaSuccess &&
+  if (ctx->phase_timing != 1 && side_ready(ctx) && cudaEventRecord(ctx->ev_fork, st) == cudaSuccess &&
       cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) == cudaSuccess)
     ls = ctx->side;
   launch_k(k_scan_sel, dim3(N), dim3(1024), ls, p);
@@ -1604,13 +1609,20 @@ int mv_set_phase_timing(mv_ctx* ctx, int enable) {
       if (cudaEventCreate(&ctx->pev[i]) != cudaSuccess) return MV_ERR_CUDA;
     ctx->pev_made = true;
   }
-  ctx->phase_timing = enable ? 1 : 0;
+  ctx->phase_timing = enable > 0 ? enable : 0;  // 1: every launch; 100 + i: only the start and launch i
   return MV_OK;
 }
 
 int mv_read_phase_times(mv_ctx* ctx, float* ms, int capacity, int* count) {
   if (ctx == nullptr || ms == nullptr || count == nullptr || !ctx->pev_made) return MV_ERR_INVALID_ARG;
   if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return MV_ERR_CUDA;
+  if (ctx->phase_timing >= 100) {  // single probe: time from the start of the call to the end of launch i
+    const int i = ctx->phase_timing - 100;
+    if (i < 1 || i > ctx->launches || i > 47 || capacity < 1) return MV_ERR_INVALID_ARG;
+    if (cudaEventElapsedTime(&ms[0], ctx->pev[0], ctx->pev[i]) != cudaSuccess) return MV_ERR_CUDA;
+    *count = 1;
+    return MV_OK;
+  }
   int n = ctx->launches < 47 ? ctx->launches : 47;
   if (n > capacity) n = capacity;
   for (int i = 0; i < n; i++)

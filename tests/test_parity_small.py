@@ -24,6 +24,9 @@ def make(N, d, kind, seed):
     elif kind == "ties":
         grads = (grads * 4).round() / 4
         err = (err * 4).round() / 4
+    elif kind == "ties_fine":       # a fine grid: a handful of equal magnitudes at every level
+        grads = (grads * 2048).round() / 2048
+        err = torch.zeros(N, d)
     elif kind == "equal":
         grads = torch.full((N, d), 0.5)
         grads[::2] *= -1
@@ -118,6 +121,34 @@ def test_sampled_threshold_path(N, d, K):
     diag = ph["diag"]
     assert (diag[:, 2] == 0).all(), f"fallback used: {diag.tolist()}"
     assert (diag[:, 0] >= K).all() and (diag[:, 0] <= 4 * K + 4096).all()
+
+
+@pytest.mark.parametrize("kind", ["ties", "ties_fine"])
+@pytest.mark.parametrize("N,d,K", [(3, 300007, 2500), (2, 1000003, 300)])
+def test_sampled_threshold_path_with_ties(N, d, K, kind):
+    """Threshold ties that are only partly kept, in the sampled regime: a few of them (ranked in a small
+    list) and thousands of them (walked chunk by chunk)."""
+    grads, err = make(N, d, kind, seed=d + 17)
+    ctx = B.MvContext(N, d, K, device=DEV)
+    ref, ph, fu = PT.compare_all(ctx, grads.to(DEV), err.to(DEV), K, label=f"[sampled {kind} {N}x{d}] ")
+    assert (ref["thresh"][:, 2] > ref["thresh"][:, 1] * 0 + 1).all(), "the threshold should be tied"
+
+
+def test_threshold_beyond_the_sampled_range():
+    """The sample misses a group of huge values (they sit only in lines it does not visit), so the
+    K-th largest key lies far above the sampled bound: the candidate select must still be exact."""
+    N, d, K = 2, 400_000, 1000
+    g = torch.Generator().manual_seed(77)
+    grads = torch.randn(N, d, generator=g)
+    err = torch.zeros(N, d)
+    lines = torch.arange(d) // 32
+    hidden = torch.nonzero(lines % 2 == 1).flatten()          # the sample visits lines 0, 10, 20, ... only
+    pick = hidden[torch.randperm(hidden.numel(), generator=g)[:2000]]
+    grads[:, pick] = grads[:, pick] * 1e6 + 1e6
+    ctx = B.MvContext(N, d, K, device=DEV)
+    ref, ph, fu = PT.compare_all(ctx, grads.contiguous().to(DEV), err.to(DEV), K, label="[beyond range] ")
+    assert (ph["diag"][:, 2] == 0).all(), "the candidate path should have been kept"
+    assert (ref["thresh"][:, 0] > 0x49000000).all()            # T_n is one of the huge values
 
 
 def test_fallback_per_worker():
