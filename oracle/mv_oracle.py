@@ -211,3 +211,74 @@ def mv_sparse_step(grads, err, K: int, by_sort: bool = False, threads: int = 1):
     r["out_val"] = aggregate(r["acc"], out_idx)
     r["err"] = residual(r["acc"], out_idx)
     return r
+
+
+# ============================================================================
+# Majority voting with add-drop (Algorithm 2, MV-AD)
+#
+# Each worker keeps a vote mask Mt_n (the paper's M-tilde) from the previous
+# iteration and changes at most K_ad entries in each direction:
+#   M_n     = S_top(|acc_n|, K)                                   as before
+#   add_n   = the K_ad largest  |acc_n| among  M_n and not Mt_n   (Alg. 2, add line)
+#   drop_n  = the K_ad smallest |acc_n| among  Mt_n and not M_n   (Alg. 2, drop line)
+#   Mt_n   <- Mt_n + add_n - drop_n
+#   M_sum  <- M_sum + sum_n (add_n - drop_n)                      (Eq. 16)
+#   M       = S_top(M_sum, K)
+# followed by the same aggregation and residual as Algorithm 1.
+#
+# Readings (the paper is silent): if fewer than K_ad coordinates are eligible,
+# all of them are taken and nothing else (the selections are restricted to the
+# eligible set); ties go to the lowest index in both selections; M_sum equals
+# the per-coordinate count of the workers' current masks (true by induction when
+# it starts that way), so the server state is recomputed as that count; with
+# fewer than K voted coordinates the mask is filled up with unvoted coordinates
+# in index order, as S_top on the count vector dictates.
+# ============================================================================
+def masked_select(key: np.ndarray, eligible: np.ndarray, k: int, largest: bool) -> np.ndarray:
+    """Ascending indices of the min(k, #eligible) eligible coordinates with the largest (or
+    smallest) key, ties to the lowest index: a full stable sort of the eligible set."""
+    cand = np.flatnonzero(eligible)
+    if cand.size == 0 or k <= 0:
+        return np.zeros(0, dtype=np.int32)
+    kk = key[cand].astype(np.int64)
+    order = np.argsort(-kk if largest else kk, kind="stable")   # stable: equal keys stay in index order
+    return np.sort(cand[order[:k]]).astype(np.int32)
+
+
+def ad_vote_row(acc_row: np.ndarray, prev_row: np.ndarray, K: int, K_ad: int):
+    """One worker's add-drop vote.  prev_row: bool[d].  Returns (top-K indices, add indices,
+    drop indices, new mask bool[d])."""
+    d = acc_row.shape[0]
+    key = magnitude_key(acc_row)
+    top, _, _, _ = worker_topk(acc_row, K)
+    cur = np.zeros(d, dtype=bool)
+    cur[top] = True
+    add = masked_select(key, cur & ~prev_row, K_ad, largest=True)
+    drop = masked_select(key, prev_row & ~cur, K_ad, largest=False)
+    new = prev_row.copy()
+    new[add] = True
+    new[drop] = False
+    return top, add, drop, new
+
+
+def mv_ad_step(grads, err, prev, K: int, K_ad: int):
+    """One MV-AD step.  prev: bool[N, d] (the workers' previous vote masks).  Returns a dict with
+    acc, worker_idx [N,K], add / drop (lists of index arrays), prev (new masks, bool[N,d]),
+    msum (uint8[d]), out_idx [K], vote_thresh, out_val [K], err [N,d]."""
+    acc = accumulate(grads, err)
+    N, d = acc.shape
+    prev = np.asarray(prev, dtype=bool)
+    worker_idx = np.empty((N, K), dtype=np.int32)
+    adds, drops = [], []
+    new_prev = np.empty_like(prev)
+    for n in range(N):
+        top, add, drop, new = ad_vote_row(acc[n], prev[n], K, K_ad)
+        worker_idx[n] = top
+        adds.append(add)
+        drops.append(drop)
+        new_prev[n] = new
+    msum = new_prev.sum(axis=0).astype(np.uint8)        # Eq. 16, by induction from M_sum = count of the masks
+    out_idx, vstar, vgt, veq = select_mask(msum, K)
+    return dict(acc=acc, worker_idx=worker_idx, add=adds, drop=drops, prev=new_prev, msum=msum,
+                out_idx=out_idx, vote_thresh=(vstar, vgt, veq), out_val=aggregate(acc, out_idx),
+                err=residual(acc, out_idx))

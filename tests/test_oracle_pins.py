@@ -17,7 +17,8 @@ import torch
 
 from oracle import mv_oracle as O
 
-GOLDEN = sorted(glob.glob(os.path.join(os.path.dirname(__file__), "golden", "*.json")))
+GOLDEN = sorted(p for p in glob.glob(os.path.join(os.path.dirname(__file__), "golden", "*.json"))
+                if not os.path.basename(p).startswith("add_drop"))
 
 
 def f32_bits(x):
