@@ -219,6 +219,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2", choices=["c1", "c1_ties", "c2", "c3", "c4"])
     ap.add_argument("--mode", default="auto", choices=["auto", "general"])
+    ap.add_argument("--method", default="mv", choices=["mv", "ad"],
+                    help="mv: plain majority voting (Algorithm 1); ad: add-drop voting (Algorithm 2) with K_ad = K/10")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -262,9 +264,19 @@ def main():
 
     sampler = ClockSampler(visible_gpu_index(local_rank))
     sampler.start()
+    if args.method == "ad":
+        K_ad = max(1, w.K // 10)
+        prev_bits = torch.zeros((w.N, (w.d + 31) // 32), dtype=torch.int32, device=dev)
+
+        def one_step(g):
+            ctx.mv_ad_step(g, err, prev_bits, K_ad, out_idx, out_val)
+    else:
+        def one_step(g):
+            ctx.mv_sparse_step(g, err, out_idx, out_val)
+
     step_no = 0
     for _ in range(args.warmup):
-        ctx.mv_sparse_step(pool[step_no % pool_n], err, out_idx, out_val)
+        one_step(pool[step_no % pool_n])
         step_no += 1
     # CUDA events around the streaming kernel on one step in eight (each pair costs a few microseconds)
     ctx.set_kernel_timing(8 if args.steps >= 8 else 1)
@@ -274,7 +286,7 @@ def main():
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record()
     for _ in range(args.steps):
-        ctx.mv_sparse_step(pool[step_no % pool_n], err, out_idx, out_val)
+        one_step(pool[step_no % pool_n])
         step_no += 1
     ev1.record()
     barrier()
@@ -291,7 +303,7 @@ def main():
 
     # ---- end to end through the host entry point: gradients start in pinned host memory
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and args.method == "mv":
         h_pool = [pool[i].cpu().pin_memory() for i in range(2)]
         h_idx = torch.empty(w.K, dtype=torch.int32).pin_memory()
         h_val = torch.empty(w.K, dtype=torch.float32).pin_memory()
@@ -326,7 +338,8 @@ def main():
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
-        "data": "synthetic", "config": workload_config(w),
+        "data": "synthetic", "config": dict(workload_config(w), method=("add-drop voting, K_ad=K/10" if args.method == "ad"
+                                                                     else "majority voting")),
         "effective_gradient_gbs": w.N * w.d * 4 / (ms_step * 1e-3) / 1e9 * 1.0,
         "step_roofline_frac": alg_bytes / (ms_step * 1e-3) / 1e9 / peak,
         "roofline": {"bound": "hbm", "kernel": "k_acc_compact" if args.mode == "auto" else "k_row_hist<1,true>",

@@ -98,6 +98,24 @@ int mv_vote(mv_ctx* ctx, const float* grads, float* err, int N, int64_t d, int64
 int mv_select(mv_ctx* ctx, const uint8_t* votes, int N, int64_t d, int64_t K,
               int32_t* out_idx, uint32_t* mask_bits);
 
+/* One step of majority voting with add-drop (Algorithm 2, MV-AD; the vote update and Eq. 16).
+ * Each worker keeps a vote mask from the previous step and changes at most K_ad entries in each
+ * direction: it adds the K_ad largest |acc| among its current top-K coordinates that it did not
+ * vote for, and drops the K_ad smallest |acc| among its previous votes that are not in its current
+ * top-K (fewer if fewer are eligible; ties to the lowest index).  The shared mask is the K
+ * coordinates voted for by most workers under the updated masks (the running sum of Eq. 16 is
+ * that count), filled up in index order if fewer than K coordinates have a vote.  Aggregation and
+ * residual are those of mv_sparse_step.
+ *   grads     [N*d] in; err [N*d] in/out (residual); out_idx [K], out_val [K] out
+ *   prev_bits [N*ceil(d/32)] in/out  the workers' vote masks; at most K bits per worker and no
+ *                                    bits at or beyond d (all-zero masks are a valid start)
+ *   K_ad      1 <= K_ad <= K
+ *   add_bits, drop_bits [N*ceil(d/32)] out, may be NULL: what each worker added / dropped
+ *   msum      [d] uint8 out, may be NULL: votes per coordinate under the updated masks */
+int mv_ad_step(mv_ctx* ctx, const float* grads, float* err, uint32_t* prev_bits, int N, int64_t d, int64_t K,
+               int64_t K_ad, int32_t* out_idx, float* out_val, uint32_t* add_bits, uint32_t* drop_bits,
+               uint8_t* msum);
+
 /* mv_select for callers that cannot hand the library a workspace.  (The paper has no counterpart
  * to this call: it is the same selection as mv_select, packaged differently.)
  *

@@ -59,6 +59,8 @@ def load() -> ctypes.CDLL:
     lib.mv_vote.argtypes = [c_vp, c_vp, c_vp, c_i, c_i64, c_i64, c_vp, c_vp, c_vp, c_vp]
     lib.mv_select.restype = c_i
     lib.mv_select.argtypes = [c_vp, c_vp, c_i, c_i64, c_i64, c_vp, c_vp]
+    lib.mv_ad_step.restype = c_i
+    lib.mv_ad_step.argtypes = [c_vp, c_vp, c_vp, c_vp, c_i, c_i64, c_i64, c_i64, c_vp, c_vp, c_vp, c_vp, c_vp]
     lib.mv_select_static.restype = c_i
     lib.mv_select_static.argtypes = [c_vp, c_vp, c_i, c_i64, c_i64, c_vp, c_vp]
     lib.mv_aggregate.restype = c_i
@@ -159,6 +161,13 @@ class MvContext:
         N, d = acc.shape
         _check(self.lib.mv_aggregate(self.handle, _ptr(acc), N, d, idx.numel(), _ptr(idx), _ptr(out_val)),
                "mv_aggregate")
+
+    def mv_ad_step(self, grads, err, prev_bits, K_ad: int, out_idx, out_val, add_bits=None, drop_bits=None,
+                   msum=None, K: Optional[int] = None):
+        N, d = grads.shape
+        _check(self.lib.mv_ad_step(self.handle, _ptr(grads), _ptr(err), _ptr(prev_bits), N, d, K or self.K, int(K_ad),
+                                   _ptr(out_idx), _ptr(out_val), _ptr(add_bits), _ptr(drop_bits), _ptr(msum)),
+               "mv_ad_step")
 
     def mv_sparse_step_host(self, h_grads, h_out_idx, h_out_val, d_grads, d_err, d_out_idx, d_out_val,
                             K: Optional[int] = None):

@@ -45,6 +45,7 @@ struct P {
   int nc_pad;             // nchunks rounded up to a multiple of 8 (row pitch of chunk_vh)
   uint32_t cap;           // candidate slots per worker
   int force_general;
+  int list_mode;          // 1: the rows are plain (key, index) lists to select min(K, length) from (add-drop)
   int64_t d;
   int64_t K;
   int64_t W;              // mask words per row = ceil(d/32)
@@ -97,7 +98,15 @@ __device__ __forceinline__ uint32_t lanemask_lt() {
 __device__ __forceinline__ bool worker_fast(const P& p, int n) {
   if (p.force_general) return false;
   const uint32_t c = p.cand_cnt[n];
+  if (p.list_mode) return c > 0;
   return c >= (uint32_t)p.K && c <= p.cap;
+}
+
+// how many elements worker n selects: K, or in list mode min(K, length of its list)
+__device__ __forceinline__ uint32_t worker_K(const P& p, int n) {
+  if (!p.list_mode) return (uint32_t)p.K;
+  const uint32_t c = p.cand_cnt[n];
+  return c < (uint32_t)p.K ? c : (uint32_t)p.K;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -465,7 +474,7 @@ __device__ __forceinline__ uint32_t resolve_prefix(const P& p, int n) {
   uint32_t* ws = p.wstate + (size_t)n * 8;
   if (PASS == 2) {
     uint32_t b1, rem1;
-    block_pick<H1_BINS, TPB>(p.hist1 + (size_t)n * H1_BINS, (uint32_t)p.K, b1, rem1);
+    block_pick<H1_BINS, TPB>(p.hist1 + (size_t)n * H1_BINS, worker_K(p, n), b1, rem1);
     if (blockIdx.x == 0 && threadIdx.x == 0) {
       ws[0] = b1;
       ws[1] = rem1;
@@ -496,7 +505,7 @@ __device__ __forceinline__ uint32_t resolve_threshold(const P& p, int n, uint32_
   cnt_eq = __ldcg(p.hist3 + (size_t)n * H3_BINS + b3);
   need = rem3;
   if (blockIdx.x == 0 && threadIdx.x == 0) {
-    const uint32_t cnt_gt = (uint32_t)p.K - rem3;
+    const uint32_t cnt_gt = worker_K(p, n) - rem3;
     ws[4] = T;
     ws[5] = cnt_gt;
     ws[6] = cnt_eq;
@@ -537,6 +546,7 @@ __global__ void __launch_bounds__(TPB) k_hist(P p, const float* __restrict__ gra
   __shared__ uint32_t sh[NB];
   const int n = blockIdx.y;
   const bool fast = !FUSED && worker_fast(p, n);
+  if (p.list_mode && !fast) return;  // empty list
   const uint32_t prefix = resolve_prefix<PASS>(p, n);
   for (int b = threadIdx.x; b < NB; b += TPB) sh[b] = 0;
   __syncthreads();
@@ -616,6 +626,7 @@ __global__ void __launch_bounds__(TPB) k_count(P p, float* __restrict__ err) {
   pdl_enter();
   __shared__ uint32_t s_e[TPB / 32];
   const int n = blockIdx.y;
+  if (p.list_mode && !worker_fast(p, n)) return;  // empty list
   uint32_t need, cnt_eq;
   const uint32_t T = resolve_threshold(p, n, need, cnt_eq);
   if (need >= cnt_eq) return;  // every tie is kept: no order needed (uniform over the worker's CTAs)
@@ -770,6 +781,7 @@ __global__ void __launch_bounds__(TPB) k_set_bits(P p, float* __restrict__ err) 
   __shared__ uint32_t s_we[9];
   const int n = blockIdx.y;
   const bool fast = worker_fast(p, n);
+  if (p.list_mode && !fast) return;  // empty list
   const uint32_t* ws = p.wstate + (size_t)n * 8;
   const uint32_t T = ws[4], need = ws[7];
   const bool all_ties = need >= ws[6];
@@ -1196,6 +1208,95 @@ __global__ void __launch_bounds__(TPB) k_gather(float* __restrict__ acc, int N, 
 }
 
 // ---------------------------------------------------------------------------------------------
+// add-drop voting (Algorithm 2): from this step's top-K masks M_n and the previous vote masks Mt_n,
+//   k_ad_fill   lists, per worker, the coordinates of  M_n & ~Mt_n  (with their keys) and of
+//               Mt_n & ~M_n  (with inverted keys), in index order per chunk;
+//   k_hist<1..3>, k_count, k_set_bits (list mode, 2N rows) pick the min(K_ad, length) largest of
+//               each list -- the largest |acc| to add, the smallest |acc| to drop -- as bit masks;
+//   k_ad_apply  Mt_n <- (Mt_n | add_n) & ~drop_n.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128) k_ad_fill(P p, P a, const uint32_t* __restrict__ prev_bits,
+                                                 const float* __restrict__ acc) {
+  pdl_enter();
+  __shared__ uint32_t s_wa[4], s_wd[4], s_base[2];
+  const int n = blockIdx.y, c = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int64_t wi = (int64_t)c * WPC + tid;
+  uint32_t M = 0, Q = 0;
+  if (wi < p.W) {
+    M = __ldcg(p.worker_bits + (size_t)n * p.W + wi);
+    Q = __ldcg(prev_bits + (size_t)n * p.W + wi);
+  }
+  uint32_t A = M & ~Q, D = Q & ~M;
+  const uint32_t pa = __popc(A), pd = __popc(D);
+  uint32_t xa = pa, xd = pd;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const uint32_t ya = __shfl_up_sync(FULL, xa, off), yd = __shfl_up_sync(FULL, xd, off);
+    if (lane >= off) {
+      xa += ya;
+      xd += yd;
+    }
+  }
+  if (lane == 31) {
+    s_wa[warp] = xa;
+    s_wd[warp] = xd;
+  }
+  __syncthreads();
+  uint32_t offa = xa - pa, offd = xd - pd, tota = 0, totd = 0;
+  for (int w = 0; w < 4; w++) {
+    if (w < warp) {
+      offa += s_wa[w];
+      offd += s_wd[w];
+    }
+    tota += s_wa[w];
+    totd += s_wd[w];
+  }
+  if (tid == 0) {
+    const size_t ca = (size_t)n * p.nchunks + c, cd = (size_t)(p.N + n) * p.nchunks + c;
+    const uint32_t ba = tota ? atomicAdd(&a.cand_cnt[n], tota) : 0u;
+    const uint32_t bd = totd ? atomicAdd(&a.cand_cnt[p.N + n], totd) : 0u;
+    a.chunk_base[ca] = ba;
+    a.chunk_cnt[ca] = tota;
+    a.chunk_base[cd] = bd;
+    a.chunk_cnt[cd] = totd;
+    s_base[0] = ba;
+    s_base[1] = bd;
+  }
+  __syncthreads();
+  const float* row = acc + (size_t)n * (size_t)p.d;
+  uint2* la = a.cand + (size_t)n * a.cap;
+  uint2* ld = a.cand + (size_t)(p.N + n) * a.cap;
+  uint32_t pos = s_base[0] + offa;
+  while (A) {
+    const int b = __ffs(A) - 1;
+    A &= A - 1;
+    const int64_t j = wi * 32 + b;
+    if (j < p.d && pos < a.cap) la[pos] = make_uint2(fkey(row[j]), (uint32_t)j);
+    pos++;
+  }
+  pos = s_base[1] + offd;
+  while (D) {
+    const int b = __ffs(D) - 1;
+    D &= D - 1;
+    const int64_t j = wi * 32 + b;
+    if (j < p.d && pos < a.cap) ld[pos] = make_uint2(0x7fffffffu - fkey(row[j]), (uint32_t)j);  // smallest first
+    pos++;
+  }
+}
+
+__global__ void __launch_bounds__(TPB) k_ad_apply(uint32_t* __restrict__ prev_bits, const uint32_t* __restrict__ ad_bits,
+                                                  uint32_t* __restrict__ add_out, uint32_t* __restrict__ drop_out,
+                                                  size_t words /* N*W */) {
+  pdl_enter();
+  for (size_t i = (size_t)blockIdx.x * TPB + threadIdx.x; i < words; i += (size_t)gridDim.x * TPB) {
+    const uint32_t add = __ldcg(ad_bits + i), drop = __ldcg(ad_bits + words + i);
+    prev_bits[i] = (prev_bits[i] | add) & ~drop;
+    if (add_out) add_out[i] = add;
+    if (drop_out) drop_out[i] = drop;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------
 struct Layout {
@@ -1206,6 +1307,11 @@ struct Layout {
   size_t samp_hist, hist1, hist2, hist3, cand_cnt, sample_done, count_done, votes_done, hot, vote_hist;
   size_t tau, diag_cnt, wstate, thresh, vstate, cand, chunk_base, chunk_cnt, chunk_eq, tie_base, chunk_sel;
   size_t worker_bits, worker_idx, votes, chunk_vh, out_base, tie_take;
+  // add-drop voting: the select state once more, for 2N lists of at most ad_cap entries
+  uint32_t ad_cap;
+  size_t ad_zero, ad_zero_bytes;  // cleared at the start of every add-drop vote
+  size_t ad_hist1, ad_hist2, ad_hist3, ad_cnt, ad_count_done, ad_bits;
+  size_t ad_wstate, ad_thresh, ad_diag, ad_cand, ad_chunk_base, ad_chunk_cnt, ad_chunk_eq, ad_tie_base;
   size_t total;
 };
 
@@ -1256,6 +1362,26 @@ Layout make_layout(int N, int64_t d, int64_t K) {
   L.chunk_vh = take(off, (size_t)(((L.nchunks + 7) & ~7)) * (n + 1) * 2);
   L.out_base = take(off, (nc + 1) * 4);
   L.tie_take = take(off, nc * 4);
+  {
+    const size_t m = 2 * n;
+    L.ad_cap = (uint32_t)((K + 7) & ~(int64_t)7);
+    L.ad_zero = off;
+    L.ad_hist1 = take(off, m * H1_BINS * 4);
+    L.ad_hist2 = take(off, m * H2_BINS * 4);
+    L.ad_hist3 = take(off, m * H3_BINS * 4);
+    L.ad_cnt = take(off, m * 4);
+    L.ad_count_done = take(off, m * 4);
+    L.ad_bits = take(off, m * (size_t)L.W * 4);
+    L.ad_zero_bytes = off - L.ad_zero;
+    L.ad_wstate = take(off, m * 8 * 4);
+    L.ad_thresh = take(off, m * 3 * 4);
+    L.ad_diag = take(off, m * 4);
+    L.ad_cand = take(off, m * (size_t)L.ad_cap * 8);
+    L.ad_chunk_base = take(off, m * nc * 4);
+    L.ad_chunk_cnt = take(off, m * nc * 4);
+    L.ad_chunk_eq = take(off, m * nc * 4);
+    L.ad_tie_base = take(off, m * nc * 4);
+  }
   L.total = off;
   return L;
 }
@@ -1302,6 +1428,7 @@ P make_params(const mv_ctx* ctx, const Layout& L, int N, int64_t d, int64_t K) {
   p.nc_pad = (L.nchunks + 7) & ~7;
   p.cap = L.cap;
   p.force_general = ctx->mode == MV_MODE_GENERAL ? 1 : 0;
+  p.list_mode = 0;
   p.d = d;
   p.K = K;
   p.W = L.W;
@@ -1420,7 +1547,9 @@ int join_side(mv_ctx* ctx) {
 }
 
 // steps a1-a3: accumulate, per-worker top-K, votes
-int vote_impl(mv_ctx* ctx, P p, const Layout& L, const float* grads, float* err) {
+// `topk_only`: stop once the workers' bit masks are set (no vote count, no index lists); everything
+// then stays on the caller's stream
+int vote_impl(mv_ctx* ctx, P p, const Layout& L, const float* grads, float* err, bool topk_only = false) {
   cudaStream_t st = ctx->stream;
   const int N = p.N;
   ctx->timing_now = ctx->timing > 0 && (ctx->timing_calls++ % ctx->timing) == 0;
@@ -1430,7 +1559,7 @@ int vote_impl(mv_ctx* ctx, P p, const Layout& L, const float* grads, float* err)
   // per-chunk outputs of the vote count start out cleared (only chunks with candidates are
   // visited later); cleared on the side stream, concurrently with the sampling and streaming pass
   cudaStream_t zs = st;
-  if (ctx->phase_timing != 1 && side_ready(ctx) && cudaEventRecord(ctx->ev_fork, st) == cudaSuccess &&
+  if (!topk_only && ctx->phase_timing != 1 && side_ready(ctx) && cudaEventRecord(ctx->ev_fork, st) == cudaSuccess &&
       cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) == cudaSuccess)
     zs = ctx->side;
   {
@@ -1472,6 +1601,7 @@ int vote_impl(mv_ctx* ctx, P p, const Layout& L, const float* grads, float* err)
   const int gb = p.force_general ? gh : per_row_ctas(N, (int)((p.cap + TPB * 16 - 1) / (TPB * 16)), 148 * 4);
   launch_k(k_set_bits, dim3(dim3(gb, N)), dim3(TPB), st, p, err);
   MV_LAUNCH_CHECK();
+  if (topk_only) return MV_OK;
   if (zs != st && cudaStreamWaitEvent(st, ctx->ev_zero, 0) != cudaSuccess) return MV_ERR_CUDA;
   {
     const dim3 gv(p.nchunks < 148 * 8 ? p.nchunks : 148 * 8);
@@ -1722,6 +1852,88 @@ int mv_sparse_step(mv_ctx* ctx, const float* grads, float* err, int N, int64_t d
   if (rc == MV_OK) rc = aggregate_impl(ctx, err, N, d, K, out_idx, out_val, L.zero_bytes);
   const int rcj = join_side(ctx);
   return rc != MV_OK ? rc : rcj;
+}
+
+int mv_ad_step(mv_ctx* ctx, const float* grads, float* err, uint32_t* prev_bits, int N, int64_t d, int64_t K,
+               int64_t K_ad, int32_t* out_idx, float* out_val, uint32_t* add_bits, uint32_t* drop_bits, uint8_t* msum) {
+  Layout L;
+  int rc = check_common(ctx, N, d, K, L);
+  if (rc != MV_OK) return rc;
+  if (K_ad < 1 || K_ad > K) return MV_ERR_INVALID_ARG;
+  if (grads == nullptr || err == nullptr || prev_bits == nullptr || out_idx == nullptr || out_val == nullptr)
+    return MV_ERR_INVALID_ARG;
+  if (!aligned16(grads) || !aligned16(err) || !aligned16(prev_bits) || !aligned16(out_idx) || !aligned16(out_val))
+    return MV_ERR_INVALID_ARG;
+  if ((add_bits && !aligned16(add_bits)) || (drop_bits && !aligned16(drop_bits)) || (msum && !aligned16(msum)))
+    return MV_ERR_INVALID_ARG;
+  const size_t nb = (size_t)N * (size_t)d * 4;
+  if (overlap(grads, nb, err, nb)) return MV_ERR_INVALID_ARG;
+  ctx->launches = 0;
+  if (ctx->phase_timing) cudaEventRecord(ctx->pev[0], ctx->stream);
+  cudaStream_t st = ctx->stream;
+  P p = make_params(ctx, L, N, d, K);
+  ctx->last_N = N;
+  ctx->last_d = d;
+  ctx->last_K = K;
+  // this step's top-K masks M_n (kept in the workspace); err now holds acc
+  rc = vote_impl(ctx, p, L, grads, err, true);
+  if (rc != MV_OK) return rc;
+  // the add and drop selections: 2N lists through the select kernels in list mode
+  char* b = ctx->ws;
+  P a = p;
+  a.N = 2 * N;
+  a.K = K_ad;
+  a.cap = L.ad_cap;
+  a.list_mode = 1;
+  a.force_general = 0;
+  a.hist1 = (uint32_t*)(b + L.ad_hist1);
+  a.hist2 = (uint32_t*)(b + L.ad_hist2);
+  a.hist3 = (uint32_t*)(b + L.ad_hist3);
+  a.cand_cnt = (uint32_t*)(b + L.ad_cnt);
+  a.count_done = (uint32_t*)(b + L.ad_count_done);
+  a.worker_bits = (uint32_t*)(b + L.ad_bits);
+  a.wstate = (uint32_t*)(b + L.ad_wstate);
+  a.thresh = (uint32_t*)(b + L.ad_thresh);
+  a.diag_cnt = (uint32_t*)(b + L.ad_diag);
+  a.cand = (uint2*)(b + L.ad_cand);
+  a.chunk_base = (uint32_t*)(b + L.ad_chunk_base);
+  a.chunk_cnt = (uint32_t*)(b + L.ad_chunk_cnt);
+  a.chunk_eq = (uint32_t*)(b + L.ad_chunk_eq);
+  a.tie_base = (uint32_t*)(b + L.ad_tie_base);
+  if (cudaMemsetAsync(b + L.ad_zero, 0, L.ad_zero_bytes, st) != cudaSuccess) return MV_ERR_CUDA;
+  launch_k(k_ad_fill, dim3(dim3(p.nchunks, N)), dim3(128), st, p, a, (const uint32_t*)prev_bits, (const float*)err);
+  MV_LAUNCH_CHECK();
+  const int ga = per_row_ctas(2 * N, (int)((a.cap + TPB * 8 - 1) / (TPB * 8)), 148 * 2);
+  launch_k(k_hist<1, false>, dim3(dim3(ga, 2 * N)), dim3(TPB), st, a, nullptr, err);
+  MV_LAUNCH_CHECK();
+  launch_k(k_hist<2, false>, dim3(dim3(ga, 2 * N)), dim3(TPB), st, a, nullptr, err);
+  MV_LAUNCH_CHECK();
+  launch_k(k_hist<3, false>, dim3(dim3(ga, 2 * N)), dim3(TPB), st, a, nullptr, err);
+  MV_LAUNCH_CHECK();
+  launch_k(k_count, dim3(dim3(ga, 2 * N)), dim3(TPB), st, a, err);
+  MV_LAUNCH_CHECK();
+  launch_k(k_set_bits, dim3(dim3(ga, 2 * N)), dim3(TPB), st, a, err);
+  MV_LAUNCH_CHECK();
+  const size_t words = (size_t)N * (size_t)p.W;
+  launch_k(k_ad_apply, dim3((unsigned)((words + TPB * 4 - 1) / (TPB * 4))), dim3(TPB), st, prev_bits,
+           (const uint32_t*)a.worker_bits, add_bits, drop_bits, words);
+  MV_LAUNCH_CHECK();
+  // votes of the updated masks (= the server's running sum, Eq. 16), shared mask, aggregate
+  P v = p;
+  v.worker_bits = prev_bits;
+  if (msum) v.votes = msum;
+  if (cudaMemsetAsync(p.hot, 1, (size_t)p.nc_pad, st) != cudaSuccess) return MV_ERR_CUDA;  // every chunk may hold votes
+  {
+    const dim3 gv(p.nchunks < 148 * 8 ? p.nchunks : 148 * 8);
+    if (N < 4) launch_k(k_votes<2>, gv, dim3(VT), st, v);
+    else if (N < 16) launch_k(k_votes<4>, gv, dim3(VT), st, v);
+    else if (N < 64) launch_k(k_votes<6>, gv, dim3(VT), st, v);
+    else launch_k(k_votes<8>, gv, dim3(VT), st, v);
+  }
+  MV_LAUNCH_CHECK();
+  rc = select_impl(ctx, v, L, v.votes, false, out_idx, nullptr);  // fewer than K voted coordinates are possible here
+  if (rc != MV_OK) return rc;
+  return aggregate_impl(ctx, err, N, d, K, out_idx, out_val, L.zero_bytes);
 }
 
 int mv_sparse_step_host(mv_ctx* ctx, const float* h_grads, int N, int64_t d, int64_t K, int32_t* h_out_idx,
