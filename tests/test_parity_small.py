@@ -151,6 +151,15 @@ def test_threshold_beyond_the_sampled_range():
     assert (ref["thresh"][:, 0] > 0x49000000).all()            # T_n is one of the huge values
 
 
+@pytest.mark.parametrize("N,d,K", [(2, 500_000, 1), (2, 500_000, 499_999), (3, 400_001, 200_000), (2, 1_000_003, 7)])
+def test_sampled_regime_extreme_K(N, d, K):
+    """K = 1, K close to d and K = d/2 at sizes where the threshold bound comes from a sample: whatever
+    path each worker ends up on, the results are exact."""
+    grads, err = make(N, d, "gauss", seed=K + d)
+    ctx = B.MvContext(N, d, K, device=DEV)
+    PT.compare_all(ctx, grads.to(DEV), err.to(DEV), K, label=f"[extreme K {N}x{d} K={K}] ")
+
+
 def test_fallback_per_worker():
     """One smooth worker next to one whose values are all equal (its candidate count overflows):
     the second takes the exact multi-pass select, the first does not, results are exact."""
