@@ -1931,7 +1931,9 @@ int mv_ad_step(mv_ctx* ctx, const float* grads, float* err, uint32_t* prev_bits,
     else launch_k(k_votes<8>, gv, dim3(VT), st, v);
   }
   MV_LAUNCH_CHECK();
-  rc = select_impl(ctx, v, L, v.votes, false, out_idx, nullptr);  // fewer than K voted coordinates are possible here
+  // Fewer than K coordinates may hold a vote here (v* = 0).  k_votes visited every chunk, so its
+  // per-chunk counts include the unvoted coordinates and its scan is valid in that case too.
+  rc = select_impl(ctx, v, L, v.votes, true, out_idx, nullptr);
   if (rc != MV_OK) return rc;
   return aggregate_impl(ctx, err, N, d, K, out_idx, out_val, L.zero_bytes);
 }
