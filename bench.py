@@ -145,7 +145,7 @@ def host_cores() -> int:
         return os.cpu_count() or 1
 
 
-def oracle_steps_per_s(w: WL.Workload, steps: int, sample_workers: int, warmup: int = 0):
+def oracle_steps_per_s(w: WL.Workload, steps: int, sample_workers: int, warmup: int = 0, method: str = "mv"):
     """Times the CPU oracle as it stands on a bounded sample: the first `sample_workers` rows of
     the workload, full d and K (a majority-vote step among those workers).  Returns
     (steps/s of the sample, seconds per step, description)."""
@@ -154,11 +154,16 @@ def oracle_steps_per_s(w: WL.Workload, steps: int, sample_workers: int, warmup: 
                      segments=w.segments, std_lo=w.std_lo, std_hi=w.std_hi, rho=w.rho, err0_std=w.err0_std,
                      round_decimals=w.round_decimals)
     err = WL.initial_err(ws).numpy()
+    prev = np.zeros((ws.N, ws.d), dtype=bool)
     times = []
     for s in range(warmup + steps):
         g = WL.gradients(ws, s).numpy()
         t0 = time.perf_counter()
-        r = O.mv_sparse_step(g, err, ws.K)
+        if method == "ad":
+            r = O.mv_ad_step(g, err, prev, ws.K, max(1, ws.K // 10))
+            prev = r["prev"]
+        else:
+            r = O.mv_sparse_step(g, err, ws.K)
         dt = time.perf_counter() - t0
         err = r["err"]
         if s >= warmup:
@@ -178,7 +183,7 @@ def run_reference(args, w: WL.Workload):
     torch.set_num_threads(max(1, host_cores()))
     sample_workers = min(w.N, 2 if w.d > 1_000_000 else w.N)
     steps = max(1, min(args.steps, 3))
-    sps, sec, desc = oracle_steps_per_s(w, steps, sample_workers, warmup=min(args.warmup, 1))
+    sps, sec, desc = oracle_steps_per_s(w, steps, sample_workers, warmup=min(args.warmup, 1), method=args.method)
     line = {
         "impl": "reference", "metric": METRIC, "value": sps, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
@@ -354,7 +359,7 @@ def main():
         line["e2e"] = e2e
     if world == 1 and not args.no_cpu_baseline:
         sample_workers = min(w.N, 2 if w.d > 1_000_000 else w.N)
-        sps, sec, desc = oracle_steps_per_s(w, 1, sample_workers)
+        sps, sec, desc = oracle_steps_per_s(w, 1, sample_workers, method=args.method)
         line["cpu_baseline"] = {"value": sps, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc,
                                 "host_cores_available": host_cores()}
     print(json.dumps(line), flush=True)

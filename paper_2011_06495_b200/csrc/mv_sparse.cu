@@ -46,6 +46,9 @@ struct P {
   uint32_t cap;           // candidate slots per worker
   int force_general;
   int list_mode;          // 1: the rows are plain (key, index) lists to select min(K, length) from (add-drop)
+  int apply_rows;         // list mode: rows < apply_rows are "add" lists, the others "drop" lists
+  uint32_t* apply_bits;   // list mode, optional: the vote masks [apply_rows][W] to update in place instead of
+                          // writing the picks to worker_bits
   int64_t d;
   int64_t K;
   int64_t W;              // mask words per row = ceil(d/32)
@@ -776,6 +779,18 @@ __device__ __forceinline__ void store_vote_hist_impl(const P& p, int c, uint32_t
 // part of their threshold ties add those, lowest index first.  (3) k_votes: one CTA per chunk adds
 // the N masks bit-sliced (8 counter planes per 32-coordinate word) into the vote count.
 // ---------------------------------------------------------------------------------------------
+// Puts the picked bits `bits` of mask word w of row n where they belong: into the row's bit mask, or
+// (add-drop, in-place update) into the vote mask, set for an "add" row and cleared for a "drop" row.
+__device__ __forceinline__ void put_bits(const P& p, int n, uint32_t w, uint32_t bits) {
+  if (p.apply_bits == nullptr) {
+    atomicOr(p.worker_bits + (size_t)n * p.W + w, bits);
+  } else if (n < p.apply_rows) {
+    atomicOr(p.apply_bits + (size_t)n * p.W + w, bits);
+  } else {
+    atomicAnd(p.apply_bits + (size_t)(n - p.apply_rows) * p.W + w, ~bits);
+  }
+}
+
 __global__ void __launch_bounds__(TPB) k_set_bits(P p, float* __restrict__ err) {
   pdl_enter();
   __shared__ uint32_t s_we[9];
@@ -885,14 +900,14 @@ __global__ void __launch_bounds__(TPB) k_set_bits(P p, float* __restrict__ err) 
       if (sel && (int64_t)j < p.d) {
         const uint32_t w = j >> 5;
         if (w != curw) {
-          if (acc) atomicOr(bits_row + curw, acc);
+          if (acc) put_bits(p, n, curw, acc);
           curw = w;
           acc = 0;
         }
         acc |= 1u << (j & 31u);
       }
     }
-    if (acc) atomicOr(bits_row + curw, acc);
+    if (acc) put_bits(p, n, curw, acc);
   }
   // a worker that keeps only part of its threshold ties adds them chunk by chunk, lowest index first
   if (all_ties) return;
@@ -913,7 +928,7 @@ __global__ void __launch_bounds__(TPB) k_set_bits(P p, float* __restrict__ err) 
         eq = kv.x == T;
       }
       const uint32_t eb = __ballot_sync(FULL, eq);
-      if (eq && run + __popc(eb & lt) < need && (int64_t)kv.y < p.d) atomicOr(bits_row + (kv.y >> 5), 1u << (kv.y & 31u));
+      if (eq && run + __popc(eb & lt) < need && (int64_t)kv.y < p.d) put_bits(p, n, kv.y >> 5, 1u << (kv.y & 31u));
       run += __popc(eb);
     }
   }
@@ -1215,19 +1230,28 @@ __global__ void __launch_bounds__(TPB) k_gather(float* __restrict__ acc, int N, 
 //               each list -- the largest |acc| to add, the smallest |acc| to drop -- as bit masks;
 //   k_ad_apply  Mt_n <- (Mt_n | add_n) & ~drop_n.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(128) k_ad_fill(P p, P a, const uint32_t* __restrict__ prev_bits,
+__global__ void __launch_bounds__(TPB) k_ad_fill(P p, P a, const uint32_t* __restrict__ prev_bits,
                                                  const float* __restrict__ acc) {
   pdl_enter();
-  __shared__ uint32_t s_wa[4], s_wd[4], s_base[2];
-  const int n = blockIdx.y, c = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int64_t wi = (int64_t)c * WPC + tid;
-  uint32_t M = 0, Q = 0;
-  if (wi < p.W) {
-    M = __ldcg(p.worker_bits + (size_t)n * p.W + wi);
-    Q = __ldcg(prev_bits + (size_t)n * p.W + wi);
+  // a warp per (worker, chunk): lane l owns mask words 4l..4l+3 of the chunk, so lane order is index order
+  const int n = blockIdx.y, lane = threadIdx.x & 31;
+  const int c = blockIdx.x * (TPB / 32) + (threadIdx.x >> 5);
+  if (c >= p.nchunks) return;
+  uint32_t A[4], D[4];
+  uint32_t pa = 0, pd = 0;
+#pragma unroll
+  for (int q = 0; q < 4; q++) {
+    const int64_t wi = (int64_t)c * WPC + lane * 4 + q;
+    uint32_t M = 0, Q = 0;
+    if (wi < p.W) {
+      M = __ldcg(p.worker_bits + (size_t)n * p.W + wi);
+      Q = __ldcg(prev_bits + (size_t)n * p.W + wi);
+    }
+    A[q] = M & ~Q;
+    D[q] = Q & ~M;
+    pa += __popc(A[q]);
+    pd += __popc(D[q]);
   }
-  uint32_t A = M & ~Q, D = Q & ~M;
-  const uint32_t pa = __popc(A), pd = __popc(D);
   uint32_t xa = pa, xd = pd;
 #pragma unroll
   for (int off = 1; off < 32; off <<= 1) {
@@ -1237,50 +1261,43 @@ __global__ void __launch_bounds__(128) k_ad_fill(P p, P a, const uint32_t* __res
       xd += yd;
     }
   }
-  if (lane == 31) {
-    s_wa[warp] = xa;
-    s_wd[warp] = xd;
-  }
-  __syncthreads();
-  uint32_t offa = xa - pa, offd = xd - pd, tota = 0, totd = 0;
-  for (int w = 0; w < 4; w++) {
-    if (w < warp) {
-      offa += s_wa[w];
-      offd += s_wd[w];
-    }
-    tota += s_wa[w];
-    totd += s_wd[w];
-  }
-  if (tid == 0) {
+  const uint32_t tota = __shfl_sync(FULL, xa, 31), totd = __shfl_sync(FULL, xd, 31);
+  uint32_t ba = 0, bd = 0;
+  if (lane == 0) {
     const size_t ca = (size_t)n * p.nchunks + c, cd = (size_t)(p.N + n) * p.nchunks + c;
-    const uint32_t ba = tota ? atomicAdd(&a.cand_cnt[n], tota) : 0u;
-    const uint32_t bd = totd ? atomicAdd(&a.cand_cnt[p.N + n], totd) : 0u;
+    if (tota) ba = atomicAdd(&a.cand_cnt[n], tota);
+    if (totd) bd = atomicAdd(&a.cand_cnt[p.N + n], totd);
     a.chunk_base[ca] = ba;
     a.chunk_cnt[ca] = tota;
     a.chunk_base[cd] = bd;
     a.chunk_cnt[cd] = totd;
-    s_base[0] = ba;
-    s_base[1] = bd;
   }
-  __syncthreads();
+  if ((tota | totd) == 0) return;
+  ba = __shfl_sync(FULL, ba, 0);
+  bd = __shfl_sync(FULL, bd, 0);
   const float* row = acc + (size_t)n * (size_t)p.d;
   uint2* la = a.cand + (size_t)n * a.cap;
   uint2* ld = a.cand + (size_t)(p.N + n) * a.cap;
-  uint32_t pos = s_base[0] + offa;
-  while (A) {
-    const int b = __ffs(A) - 1;
-    A &= A - 1;
-    const int64_t j = wi * 32 + b;
-    if (j < p.d && pos < a.cap) la[pos] = make_uint2(fkey(row[j]), (uint32_t)j);
-    pos++;
-  }
-  pos = s_base[1] + offd;
-  while (D) {
-    const int b = __ffs(D) - 1;
-    D &= D - 1;
-    const int64_t j = wi * 32 + b;
-    if (j < p.d && pos < a.cap) ld[pos] = make_uint2(0x7fffffffu - fkey(row[j]), (uint32_t)j);  // smallest first
-    pos++;
+  uint32_t posa = ba + xa - pa, posd = bd + xd - pd;
+#pragma unroll
+  for (int q = 0; q < 4; q++) {
+    const int64_t j0 = ((int64_t)c * WPC + lane * 4 + q) * 32;
+    uint32_t m = A[q];
+    while (m) {
+      const int b = __ffs(m) - 1;
+      m &= m - 1;
+      const int64_t j = j0 + b;
+      if (j < p.d && posa < a.cap) la[posa] = make_uint2(fkey(row[j]), (uint32_t)j);
+      posa++;
+    }
+    m = D[q];
+    while (m) {
+      const int b = __ffs(m) - 1;
+      m &= m - 1;
+      const int64_t j = j0 + b;
+      if (j < p.d && posd < a.cap) ld[posd] = make_uint2(0x7fffffffu - fkey(row[j]), (uint32_t)j);  // smallest first
+      posd++;
+    }
   }
 }
 
@@ -1429,6 +1446,8 @@ P make_params(const mv_ctx* ctx, const Layout& L, int N, int64_t d, int64_t K) {
   p.cap = L.cap;
   p.force_general = ctx->mode == MV_MODE_GENERAL ? 1 : 0;
   p.list_mode = 0;
+  p.apply_rows = 0;
+  p.apply_bits = nullptr;
   p.d = d;
   p.K = K;
   p.W = L.W;
@@ -1900,8 +1919,15 @@ int mv_ad_step(mv_ctx* ctx, const float* grads, float* err, uint32_t* prev_bits,
   a.chunk_cnt = (uint32_t*)(b + L.ad_chunk_cnt);
   a.chunk_eq = (uint32_t*)(b + L.ad_chunk_eq);
   a.tie_base = (uint32_t*)(b + L.ad_tie_base);
-  if (cudaMemsetAsync(b + L.ad_zero, 0, L.ad_zero_bytes, st) != cudaSuccess) return MV_ERR_CUDA;
-  launch_k(k_ad_fill, dim3(dim3(p.nchunks, N)), dim3(128), st, p, a, (const uint32_t*)prev_bits, (const float*)err);
+  a.apply_rows = N;
+  // without add/drop outputs the picks update the vote masks in place (set for add, clear for drop);
+  // otherwise they are materialised as 2N masks first and applied by k_ad_apply
+  const bool direct = add_bits == nullptr && drop_bits == nullptr;
+  a.apply_bits = direct ? prev_bits : nullptr;
+  if (cudaMemsetAsync(b + L.ad_zero, 0, direct ? L.ad_bits - L.ad_zero : L.ad_zero_bytes, st) != cudaSuccess)
+    return MV_ERR_CUDA;
+  launch_k(k_ad_fill, dim3(dim3((p.nchunks + TPB / 32 - 1) / (TPB / 32), N)), dim3(TPB), st, p, a,
+           (const uint32_t*)prev_bits, (const float*)err);
   MV_LAUNCH_CHECK();
   const int ga = per_row_ctas(2 * N, (int)((a.cap + TPB * 8 - 1) / (TPB * 8)), 148 * 2);
   launch_k(k_hist<1, false>, dim3(dim3(ga, 2 * N)), dim3(TPB), st, a, nullptr, err);
@@ -1914,10 +1940,12 @@ int mv_ad_step(mv_ctx* ctx, const float* grads, float* err, uint32_t* prev_bits,
   MV_LAUNCH_CHECK();
   launch_k(k_set_bits, dim3(dim3(ga, 2 * N)), dim3(TPB), st, a, err);
   MV_LAUNCH_CHECK();
-  const size_t words = (size_t)N * (size_t)p.W;
-  launch_k(k_ad_apply, dim3((unsigned)((words + TPB * 4 - 1) / (TPB * 4))), dim3(TPB), st, prev_bits,
-           (const uint32_t*)a.worker_bits, add_bits, drop_bits, words);
-  MV_LAUNCH_CHECK();
+  if (!direct) {
+    const size_t words = (size_t)N * (size_t)p.W;
+    launch_k(k_ad_apply, dim3((unsigned)((words + TPB * 4 - 1) / (TPB * 4))), dim3(TPB), st, prev_bits,
+             (const uint32_t*)a.worker_bits, add_bits, drop_bits, words);
+    MV_LAUNCH_CHECK();
+  }
   // votes of the updated masks (= the server's running sum, Eq. 16), shared mask, aggregate
   P v = p;
   v.worker_bits = prev_bits;

@@ -27,7 +27,7 @@ def lists_to_mask(lists, d):
     return m
 
 
-def run_steps(N, d, K, K_ad, steps, kind, seed, prev0=None, mode=B.MV_MODE_AUTO):
+def run_steps(N, d, K, K_ad, steps, kind, seed, prev0=None, mode=B.MV_MODE_AUTO, want_lists=True):
     g = torch.Generator().manual_seed(seed)
     base = torch.randn(1, d, generator=g)
     W = (d + 31) // 32
@@ -47,11 +47,15 @@ def run_steps(N, d, K, K_ad, steps, kind, seed, prev0=None, mode=B.MV_MODE_AUTO)
             grads = (grads * 4).round() / 4
         grads = grads.float().contiguous()
         ref = O.mv_ad_step(grads.numpy(), err_ref, prev_ref, K, K_ad)
-        ctx.mv_ad_step(grads.to(DEV), err, prev_bits, K_ad, out_idx, out_val, add_bits, drop_bits, msum)
+        if want_lists:
+            ctx.mv_ad_step(grads.to(DEV), err, prev_bits, K_ad, out_idx, out_val, add_bits, drop_bits, msum)
+        else:       # without the add/drop outputs the vote masks are updated in place
+            ctx.mv_ad_step(grads.to(DEV), err, prev_bits, K_ad, out_idx, out_val, None, None, msum)
         torch.cuda.synchronize()
         tag = f"[ad {N}x{d} K={K} K_ad={K_ad} {kind} step {step}] "
-        PT.first_diff(PT.npy(add_bits, np.uint32), pack(lists_to_mask(ref["add"], d)), tag + "add_bits")
-        PT.first_diff(PT.npy(drop_bits, np.uint32), pack(lists_to_mask(ref["drop"], d)), tag + "drop_bits")
+        if want_lists:
+            PT.first_diff(PT.npy(add_bits, np.uint32), pack(lists_to_mask(ref["add"], d)), tag + "add_bits")
+            PT.first_diff(PT.npy(drop_bits, np.uint32), pack(lists_to_mask(ref["drop"], d)), tag + "drop_bits")
         PT.first_diff(PT.npy(prev_bits, np.uint32), pack(ref["prev"]), tag + "vote masks")
         PT.first_diff(PT.npy(msum), ref["msum"], tag + "msum")
         PT.first_diff(PT.npy(out_idx), ref["out_idx"], tag + "out_idx")
@@ -65,6 +69,12 @@ def run_steps(N, d, K, K_ad, steps, kind, seed, prev0=None, mode=B.MV_MODE_AUTO)
                                         (3, 4097, 40, 40), (33, 5000, 50, 7), (2, 300007, 3000, 300)])
 def test_add_drop_from_empty_votes(N, d, K, K_ad, kind):
     run_steps(N, d, K, K_ad, steps=5, kind=kind, seed=N * 100 + d)
+
+
+@pytest.mark.parametrize("kind", ["gauss", "ties"])
+@pytest.mark.parametrize("N,d,K,K_ad", [(3, 1000, 50, 5), (4, 10001, 300, 30), (33, 5000, 50, 7), (2, 300007, 3000, 300)])
+def test_add_drop_in_place_update(N, d, K, K_ad, kind):
+    run_steps(N, d, K, K_ad, steps=5, kind=kind, seed=N * 7 + d, want_lists=False)
 
 
 def test_add_drop_from_given_votes():
