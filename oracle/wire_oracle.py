@@ -128,3 +128,29 @@ def dequantize(codes: np.ndarray, means: np.ndarray, q: int) -> np.ndarray:
     L = 1 << (q - 1)
     mag = means[codes & (L - 1)]
     return np.where((codes >> (q - 1)) & 1, -mag, mag).astype(np.float32)
+
+
+def pack_values(codes: np.ndarray, means: np.ndarray, q: int) -> np.ndarray:
+    """Value stream: code k on stream bits [k q, k q + q) (low bit first), then the L means from the next word on."""
+    K = codes.shape[0]
+    nw = (K * q + 31) // 32
+    words = np.zeros(nw + means.shape[0], dtype=np.uint32)
+    for k in range(K):
+        for i in range(q):
+            if (int(codes[k]) >> i) & 1:
+                t = k * q + i
+                words[t >> 5] |= np.uint32(1 << (t & 31))
+    words[nw:] = means.astype(np.float32).view(np.uint32)
+    return words
+
+
+def unpack_values(words: np.ndarray, K: int, q: int):
+    nw = (K * q + 31) // 32
+    codes = np.zeros(K, dtype=np.uint8)
+    for k in range(K):
+        c = 0
+        for i in range(q):
+            t = k * q + i
+            c |= ((int(words[t >> 5]) >> (t & 31)) & 1) << i
+        codes[k] = c
+    return codes, words[nw:nw + (1 << (q - 1))].view(np.float32).copy()

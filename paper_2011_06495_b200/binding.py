@@ -81,6 +81,25 @@ def load() -> ctypes.CDLL:
     lib.mv_last_launches.argtypes = [c_vp]
     lib.mv_status_string.restype = ctypes.c_char_p
     lib.mv_status_string.argtypes = [c_i]
+    # wire formats (include/mv_wire.h)
+    lib.mv_pos_offset_bits.restype = c_i
+    lib.mv_pos_offset_bits.argtypes = [c_i64]
+    lib.mv_pos_stream_bits.restype = c_i64
+    lib.mv_pos_stream_bits.argtypes = [c_i64, c_i64, c_i64]
+    lib.mv_pos_decode_workspace_bytes.restype = c_sz
+    lib.mv_pos_decode_workspace_bytes.argtypes = [c_i64, c_i64]
+    lib.mv_pos_encode.restype = c_i
+    lib.mv_pos_encode.argtypes = [c_vp, c_vp, c_i64, c_i64, c_i64, c_vp]
+    lib.mv_pos_decode.restype = c_i
+    lib.mv_pos_decode.argtypes = [c_vp, c_vp, c_i64, c_i64, c_i64, c_vp, c_i64, c_vp, c_vp, c_sz]
+    lib.mv_quant_stream_words.restype = c_i64
+    lib.mv_quant_stream_words.argtypes = [c_i64, c_i]
+    lib.mv_quant_workspace_bytes.restype = c_sz
+    lib.mv_quant_workspace_bytes.argtypes = [c_i]
+    lib.mv_quantize.restype = c_i
+    lib.mv_quantize.argtypes = [c_vp, c_vp, c_i64, c_i, c_vp, c_vp, c_vp, c_sz]
+    lib.mv_dequantize.restype = c_i
+    lib.mv_dequantize.argtypes = [c_vp, c_vp, c_i64, c_i, c_vp]
     _lib = lib
     return lib
 
@@ -108,6 +127,52 @@ def mv_select_static(votes, N: int, K: int, out_idx, mask_bits=None, stream: Opt
     st = stream if stream is not None else torch.cuda.current_stream(votes.device)
     _check(load().mv_select_static(ctypes.c_void_p(st.cuda_stream), _ptr(votes), int(N), votes.numel(), int(K),
                                    _ptr(out_idx), _ptr(mask_bits)), "mv_select_static")
+
+
+def _stream_ptr(t: torch.Tensor, stream: Optional[torch.cuda.Stream]):
+    st = stream if stream is not None else torch.cuda.current_stream(t.device)
+    return ctypes.c_void_p(st.cuda_stream)
+
+
+def pos_offset_bits(B: int) -> int:
+    return int(load().mv_pos_offset_bits(int(B)))
+
+
+def pos_stream_bits(d: int, B: int, K: int) -> int:
+    return int(load().mv_pos_stream_bits(int(d), int(B), int(K)))
+
+
+def pos_decode_workspace_bytes(nbits: int, B: int) -> int:
+    return int(load().mv_pos_decode_workspace_bytes(int(nbits), int(B)))
+
+
+def quant_stream_words(K: int, q: int) -> int:
+    return int(load().mv_quant_stream_words(int(K), int(q)))
+
+
+def quant_workspace_bytes(q: int) -> int:
+    return int(load().mv_quant_workspace_bytes(int(q)))
+
+
+def mv_pos_encode(idx, d: int, B: int, words, stream: Optional[torch.cuda.Stream] = None):
+    """Position stream of an ascending int32 index list into `words` (uint32/int32, caller-sized)."""
+    _check(load().mv_pos_encode(_stream_ptr(words, stream), _ptr(idx), idx.numel(), int(d), int(B), _ptr(words)),
+           "mv_pos_encode")
+
+
+def mv_pos_decode(words, nbits: int, d: int, B: int, idx, result, workspace, stream: Optional[torch.cuda.Stream] = None):
+    _check(load().mv_pos_decode(_stream_ptr(words, stream), _ptr(words), int(nbits), int(d), int(B), _ptr(idx),
+                                idx.numel(), _ptr(result), _ptr(workspace), workspace.numel() * workspace.element_size()),
+           "mv_pos_decode")
+
+
+def mv_quantize(v, q: int, words, workspace, value_range=None, stream: Optional[torch.cuda.Stream] = None):
+    _check(load().mv_quantize(_stream_ptr(words, stream), _ptr(v), v.numel(), int(q), _ptr(words), _ptr(value_range),
+                              _ptr(workspace), workspace.numel() * workspace.element_size()), "mv_quantize")
+
+
+def mv_dequantize(words, K: int, q: int, out, stream: Optional[torch.cuda.Stream] = None):
+    _check(load().mv_dequantize(_stream_ptr(words, stream), _ptr(words), int(K), int(q), _ptr(out)), "mv_dequantize")
 
 
 class MvContext:

@@ -7,7 +7,8 @@ import sys
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 SRC = os.path.join(HERE, "csrc", "mv_sparse.cu")
-HDR = os.path.join(os.path.dirname(HERE), "include", "mv_sparse.h")
+SRCS = [SRC, os.path.join(HERE, "csrc", "mv_wire.cu")]
+HDRS = [os.path.join(os.path.dirname(HERE), "include", h) for h in ("mv_sparse.h", "mv_wire.h")]
 LIB = os.path.join(HERE, "libmvsparse.so")
 
 NVCC_FLAGS = [
@@ -30,13 +31,13 @@ def needs_build() -> bool:
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    return any(os.path.getmtime(f) > t for f in (SRC, HDR, os.path.abspath(__file__)))
+    return any(os.path.getmtime(f) > t for f in (*SRCS, *HDRS, os.path.abspath(__file__)))
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not needs_build():
         return LIB
-    cmd = [nvcc_path(), *NVCC_FLAGS, "-o", LIB, SRC]
+    cmd = [nvcc_path(), *NVCC_FLAGS, "-o", LIB, *SRCS]
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")

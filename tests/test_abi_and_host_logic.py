@@ -10,7 +10,7 @@ from paper_2011_06495_b200 import binding as B
 from paper_2011_06495_b200 import build as BUILD
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-HEADER = os.path.join(ROOT, "include", "mv_sparse.h")
+HEADERS = sorted(os.path.join(ROOT, "include", f) for f in os.listdir(os.path.join(ROOT, "include")) if f.endswith(".h"))
 
 
 @pytest.fixture(scope="module")
@@ -20,17 +20,20 @@ def lib():
 
 
 def declared_functions():
-    text = open(HEADER).read()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(mv_[a-z_]+)\s*\(", text)))
+    names = set()
+    for header in HEADERS:
+        text = re.sub(r"/\*.*?\*/", "", open(header).read(), flags=re.S)
+        names |= set(re.findall(r"\b(mv_[a-z_]+)\s*\(", text))
+    return sorted(names)
 
 
 def test_every_declared_symbol_is_exported(lib):
     names = declared_functions()
     assert {"mv_sparse_step", "mv_vote", "mv_select", "mv_aggregate", "mv_workspace_bytes", "mv_create",
-            "mv_destroy", "mv_sparse_step_host"} <= set(names)
+            "mv_destroy", "mv_sparse_step_host", "mv_pos_encode", "mv_pos_decode", "mv_quantize",
+            "mv_dequantize"} <= set(names)
     for name in names:
-        assert hasattr(lib, name), f"{name} is declared in mv_sparse.h but not exported"
+        assert hasattr(lib, name), f"{name} is declared in include/ but not exported"
 
 
 def test_status_strings(lib):
@@ -99,3 +102,24 @@ def test_binding_fails_loudly_without_the_library(monkeypatch, tmp_path):
     monkeypatch.setattr(B, "LIB_PATH", str(tmp_path / "missing.so"))
     with pytest.raises(ImportError):
         B.load()
+
+
+def test_wire_host_arithmetic_and_argument_checks(lib):
+    """Stream sizes are host arithmetic (Eq. 14 when K = d / B), bad arguments are refused before any launch."""
+    assert B.pos_offset_bits(1) == 0 and B.pos_offset_bits(100) == 7 and B.pos_offset_bits(128) == 7 and B.pos_offset_bits(129) == 8
+    assert B.pos_stream_bits(12, 4, 3) == 12
+    assert B.pos_stream_bits(128 * 1000, 128, 1000) == 1000 * 9            # log2(1/phi) + 2 bits per position
+    assert B.pos_stream_bits(11_173_962, 100, 111_739) == 111_739 * 8 + 111_740
+    assert B.pos_stream_bits(10, 11, 1) == -1 and B.pos_stream_bits(10, 2, 11) == -1 and B.pos_stream_bits(0, 1, 0) == -1
+    assert B.quant_stream_words(10, 4) == 2 + 8 and B.quant_stream_words(0, 1) == 1
+    assert B.quant_stream_words(10, 0) == -1 and B.quant_stream_words(10, 9) == -1
+    assert B.pos_decode_workspace_bytes(2048 * 3 + 1, 128) >= 4 * (8 * 4 + 4 + 8 + 8)
+    assert B.quant_workspace_bytes(4) > 0 and B.quant_workspace_bytes(9) == 0
+    p = ctypes.c_void_p(0x10000)
+    assert lib.mv_pos_encode(None, p, 3, 10, 11, p) == B.MV_ERR_INVALID_ARG          # B > d
+    assert lib.mv_pos_encode(None, None, 3, 10, 2, p) == B.MV_ERR_INVALID_ARG         # idx missing
+    assert lib.mv_pos_decode(None, p, 12, 12, 4, p, 3, p, p, 0) == B.MV_ERR_WORKSPACE
+    assert lib.mv_pos_decode(None, p, 12, 12, 4, p, 3, None, p, 1 << 20) == B.MV_ERR_INVALID_ARG
+    assert lib.mv_quantize(None, p, 10, 9, p, None, p, 1 << 20) == B.MV_ERR_INVALID_ARG
+    assert lib.mv_quantize(None, p, 10, 4, p, None, p, 8) == B.MV_ERR_WORKSPACE
+    assert lib.mv_dequantize(None, None, 10, 4, p) == B.MV_ERR_INVALID_ARG

@@ -123,3 +123,19 @@ def test_quantizer_degenerate_inputs():
         nz = v != 0
         assert np.array_equal(rec[nz], v[nz]) if nz.all() else np.all(np.sign(rec[nz]) == np.sign(v[nz]))
         assert np.array_equal((codes >> 3) & 1, np.signbit(v).astype(np.uint8))
+
+
+def test_value_stream_layout():
+    # q = 3: codes 5, 2, 7 -> bits 101 010 111 low bit first: stream bits 1,0,1, 0,1,0, 1,1,1 -> 0b111010101
+    means = np.array([4, 3, 2, 1], dtype=np.float32)
+    words = W.pack_values(np.array([5, 2, 7], dtype=np.uint8), means, 3)
+    assert words.size == 1 + 4 and int(words[0]) == 0b111010101
+    assert words[1:].view(np.float32).tolist() == [4, 3, 2, 1]
+    codes, m = W.unpack_values(words, 3, 3)
+    assert codes.tolist() == [5, 2, 7] and m.tolist() == [4, 3, 2, 1]
+    rng = np.random.default_rng(0)
+    for q in (1, 2, 5, 8):
+        c = rng.integers(0, 1 << q, size=77).astype(np.uint8)
+        mu = rng.random(1 << (q - 1)).astype(np.float32)
+        cc, mm = W.unpack_values(W.pack_values(c, mu, q), 77, q)
+        assert np.array_equal(cc, c) and np.array_equal(mm, mu)
