@@ -4,7 +4,7 @@
 // block of B coordinates.  The encoder is one thread per position: the token of the k-th position
 // starts at bit k (1 + w) + (its block number), because exactly that many closing bits precede it.
 // The decoder cannot know where tokens start without walking the stream, so it walks it in three
-// small kernels: every 2048-bit segment is parsed once for each of the w + 1 ways a token can
+// small kernels: every 512-bit segment is parsed once for each of the w + 1 ways a token can
 // straddle its left edge, a single block chains the per-segment results (which entry state is the
 // real one, how many positions and blocks precede the segment), and the segments are then parsed
 // once more, in parallel, writing the positions.
@@ -22,8 +22,9 @@
 
 namespace {
 
-constexpr int SEG_BITS = 2048;       // decoder segment
+constexpr int SEG_BITS = 512;        // decoder segment
 constexpr int LINK_TILE = 256;       // segments chained per shared-memory tile
+constexpr int LINK_CHUNK = 8;        // consecutive segments composed by one thread; LINK_TILE / LINK_CHUNK = 32 chunks
 constexpr int QBINS = 128;           // 2^(8-1): most intervals a byte-wide code can name
 
 __host__ __device__ inline int offset_bits(int64_t B) {
@@ -54,72 +55,133 @@ __global__ void k_pos_encode(const int32_t* __restrict__ idx, int64_t K, uint32_
 
 // ------------------------------------------------------------------------------------------ position decoder
 // map entry: exit state (6 bits) | positions (13 bits) | closed blocks (13 bits)
-__global__ void k_pos_scan(const uint32_t* __restrict__ words, int64_t nbits, int w, int64_t nseg, uint32_t* __restrict__ map) {
-  int64_t id = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
-  if (id >= nseg * (w + 1)) return;
-  int64_t seg = id / (w + 1);
-  int r = int(id - seg * (w + 1));                  // bits of a '1' token already consumed left of the segment
-  int64_t s = seg * SEG_BITS, e = min(s + SEG_BITS, nbits);
-  int64_t t = s + (r ? (1 + w - r) : 0);
-  uint32_t n1 = 0, n0 = 0;
-  int64_t cur_i = -1;
-  uint32_t cur = 0;
-  while (t < e) {
-    if ((t >> 5) != cur_i) { cur_i = t >> 5; cur = __ldg(words + cur_i); }
-    if ((cur >> (t & 31)) & 1u) { ++n1; t += 1 + w; } else { ++n0; ++t; }
-  }
-  uint32_t out = t > e ? uint32_t((1 + w) - (t - e)) : 0u;
-  map[id] = (out << 26) | (n1 << 13) | n0;
+//
+// Both parsing kernels stage their segments' words in shared memory first (coalesced), one padding
+// word per segment so that threads walking different segments hit different banks.
+constexpr int SEG_WORDS = SEG_BITS / 32;
+constexpr int SCAN_SEGS = 32;        // segments per block of k_pos_scan (times w + 1 threads)
+constexpr int EMIT_SEGS = 32;        // segments (= threads) per block of k_pos_emit
+
+__device__ __forceinline__ int padded(int i) { return i + i / SEG_WORDS; }
+
+__device__ __forceinline__ void stage_words(const uint32_t* __restrict__ words, int64_t nwords, int64_t first, int count,
+                                            uint32_t* sw) {
+  for (int i = threadIdx.x; i < count; i += blockDim.x) sw[padded(i)] = first + i < nwords ? __ldg(words + first + i) : 0u;
+  __syncthreads();
 }
 
-__global__ void __launch_bounds__(LINK_TILE) k_pos_link(const uint32_t* __restrict__ map, int w, int64_t nseg, int64_t nblocks,
-                                                         int64_t cap, uint32_t* __restrict__ ent_state, int64_t* __restrict__ ent_b1,
-                                                         int64_t* __restrict__ ent_b0, int64_t* __restrict__ result) {
-  extern __shared__ uint32_t tile[];
-  uint32_t st = 0;
-  int64_t b1 = 0, b0 = 0;
+__global__ void k_pos_scan(const uint32_t* __restrict__ words, int64_t nbits, int w, int64_t nseg, uint32_t* __restrict__ map) {
+  __shared__ uint32_t sw[SCAN_SEGS * (SEG_WORDS + 1) + 2];
+  const int64_t seg0 = int64_t(blockIdx.x) * SCAN_SEGS;
+  stage_words(words, (nbits + 31) >> 5, seg0 * SEG_WORDS, SCAN_SEGS * SEG_WORDS, sw);
+  const int ls = threadIdx.x / (w + 1);
+  const int r = threadIdx.x - ls * (w + 1);          // bits of a '1' token already consumed left of the segment
+  const int64_t seg = seg0 + ls;
+  if (ls >= SCAN_SEGS || seg >= nseg) return;
+  const int e = int(min(int64_t(SEG_BITS), nbits - seg * SEG_BITS));      // segment-local end
+  const int base = ls * SEG_BITS;
+  int t = r ? (1 + w - r) : 0;
+  uint32_t n1 = 0, n0 = 0;
+  while (t < e) {
+    uint32_t rest = sw[padded((base + t) >> 5)] >> (t & 31);          // this word from bit t on
+    if (rest & 1u) { ++n1; t += 1 + w; }
+    else {                                                             // a run of closing bits, up to the word's or the segment's end
+      int z = min(min(rest ? __ffs(int(rest)) - 1 : 32, 32 - (t & 31)), e - t);
+      n0 += z; t += z;
+    }
+  }
+  uint32_t out = t > e ? uint32_t((1 + w) - (t - e)) : 0u;
+  map[seg * (w + 1) + r] = (out << 26) | (n1 << 13) | n0;
+}
+
+// Chains the segments.  A segment's map is a function from entry state to (exit state, counts); the
+// chain is the composition of these functions from the left.  Per tile of 256 segments: 32 (w + 1)
+// threads each compose 8 consecutive maps from one entry state, thread 0 walks the 32 composed
+// chunks with the real state, and one thread per segment replays at most 7 maps inside its chunk.
+__device__ __forceinline__ void link_step(const uint32_t* tile, int w, int seg, uint32_t& st, int64_t& b1, int64_t& b0) {
+  uint32_t m = tile[seg * (w + 1) + st];
+  st = m >> 26; b1 += (m >> 13) & 8191u; b0 += m & 8191u;
+}
+
+__global__ void __launch_bounds__(1024) k_pos_link(const uint32_t* __restrict__ map, int w, int64_t nseg, int64_t nblocks,
+                                                    int64_t cap, uint32_t* __restrict__ ent_state, int64_t* __restrict__ ent_b1,
+                                                    int64_t* __restrict__ ent_b0, int64_t* __restrict__ result) {
+  extern __shared__ uint32_t tile[];                 // LINK_TILE * (w + 1) map entries
+  constexpr int NCHUNK = LINK_TILE / LINK_CHUNK;
+  __shared__ uint32_t c_st[NCHUNK * 32], c_n1[NCHUNK * 32], c_n0[NCHUNK * 32];     // composed chunk maps [chunk][entry state]
+  __shared__ uint32_t e_st[NCHUNK + 1];
+  __shared__ int64_t e_b1[NCHUNK + 1], e_b0[NCHUNK + 1];                             // entries of the chunks; [NCHUNK] carries on
+  if (threadIdx.x == 0) { e_st[NCHUNK] = 0; e_b1[NCHUNK] = 0; e_b0[NCHUNK] = 0; }
   for (int64_t base = 0; base < nseg; base += LINK_TILE) {
-    int cnt = int(min(int64_t(LINK_TILE), nseg - base));
-    for (int i = threadIdx.x; i < cnt * (w + 1); i += LINK_TILE) tile[i] = map[base * (w + 1) + i];
+    const int cnt = int(min(int64_t(LINK_TILE), nseg - base));
+    for (int i = threadIdx.x; i < cnt * (w + 1); i += blockDim.x) tile[i] = map[base * (w + 1) + i];
+    __syncthreads();
+    if (int(threadIdx.x) < NCHUNK * (w + 1)) {
+      const int chunk = threadIdx.x / (w + 1), r = threadIdx.x - chunk * (w + 1);
+      uint32_t st = r;
+      int64_t n1 = 0, n0 = 0;
+      for (int sgm = chunk * LINK_CHUNK; sgm < min(cnt, (chunk + 1) * LINK_CHUNK); ++sgm) link_step(tile, w, sgm, st, n1, n0);
+      c_st[chunk * 32 + r] = st; c_n1[chunk * 32 + r] = uint32_t(n1); c_n0[chunk * 32 + r] = uint32_t(n0);
+    }
     __syncthreads();
     if (threadIdx.x == 0) {
-      for (int i = 0; i < cnt; ++i) {
-        ent_state[base + i] = st; ent_b1[base + i] = b1; ent_b0[base + i] = b0;
-        uint32_t m = tile[i * (w + 1) + st];
-        st = m >> 26; b1 += (m >> 13) & 8191u; b0 += m & 8191u;
+      uint32_t st = e_st[NCHUNK];
+      int64_t b1 = e_b1[NCHUNK], b0 = e_b0[NCHUNK];
+      for (int c = 0; c < NCHUNK; ++c) {
+        e_st[c] = st; e_b1[c] = b1; e_b0[c] = b0;
+        b1 += c_n1[c * 32 + st]; b0 += c_n0[c * 32 + st]; st = c_st[c * 32 + st];
       }
+      e_st[NCHUNK] = st; e_b1[NCHUNK] = b1; e_b0[NCHUNK] = b0;
+    }
+    __syncthreads();
+    if (int(threadIdx.x) < cnt) {
+      const int chunk = threadIdx.x / LINK_CHUNK;
+      uint32_t st = e_st[chunk];
+      int64_t b1 = e_b1[chunk], b0 = e_b0[chunk];
+      for (int sgm = chunk * LINK_CHUNK; sgm < int(threadIdx.x); ++sgm) link_step(tile, w, sgm, st, b1, b0);
+      ent_state[base + threadIdx.x] = st; ent_b1[base + threadIdx.x] = b1; ent_b0[base + threadIdx.x] = b0;
     }
     __syncthreads();
   }
   if (threadIdx.x == 0) {
-    result[0] = b1; result[1] = b0;
+    result[0] = e_b1[NCHUNK]; result[1] = e_b0[NCHUNK];
     // the emit kernel may add bit 4; it runs after this kernel on the same stream
-    result[2] = (st ? 1 : 0) | (b0 != nblocks ? 2 : 0) | (b1 > cap ? 8 : 0);
+    result[2] = (e_st[NCHUNK] ? 1 : 0) | (e_b0[NCHUNK] != nblocks ? 2 : 0) | (e_b1[NCHUNK] > cap ? 8 : 0);
     result[3] = 0;
   }
 }
 
-__global__ void k_pos_emit(const uint32_t* __restrict__ words, int64_t nbits, int64_t d, uint32_t B, int w, int64_t nseg,
-                           const uint32_t* __restrict__ ent_state, const int64_t* __restrict__ ent_b1,
-                           const int64_t* __restrict__ ent_b0, int32_t* __restrict__ idx, int64_t cap, int64_t* result) {
-  int64_t seg = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+__global__ void __launch_bounds__(EMIT_SEGS) k_pos_emit(const uint32_t* __restrict__ words, int64_t nbits, int64_t d, uint32_t B, int w,
+                                                         int64_t nseg, const uint32_t* __restrict__ ent_state,
+                                                         const int64_t* __restrict__ ent_b1, const int64_t* __restrict__ ent_b0,
+                                                         int32_t* __restrict__ idx, int64_t cap, int64_t* result) {
+  __shared__ uint32_t sw[EMIT_SEGS * (SEG_WORDS + 1) + 4];
+  const int64_t seg0 = int64_t(blockIdx.x) * EMIT_SEGS;
+  // two more words than the segments hold: a token that starts in a segment may end in the next one
+  stage_words(words, (nbits + 31) >> 5, seg0 * SEG_WORDS, EMIT_SEGS * SEG_WORDS + 2, sw);
+  const int64_t seg = seg0 + threadIdx.x;
   if (seg >= nseg) return;
-  int64_t nwords = (nbits + 31) >> 5;
-  int r = int(ent_state[seg]);
+  const int r = int(ent_state[seg]);
   int64_t k = ent_b1[seg], blk = ent_b0[seg];
-  int64_t s = seg * SEG_BITS, e = min(s + SEG_BITS, nbits);
-  int64_t t = s + (r ? (1 + w - r) : 0);
+  const int e = int(min(int64_t(SEG_BITS), nbits - seg * SEG_BITS));
+  const int64_t left = nbits - seg * SEG_BITS;       // stream bits from the segment start on
+  const int base = threadIdx.x * SEG_BITS;
+  int t = r ? (1 + w - r) : 0;
   bool bad = false;
   while (t < e) {
-    uint64_t x = window(words, nwords, t);
+    int i = (base + t) >> 5;
+    uint64_t x = ((uint64_t(sw[padded(i + 1)]) << 32) | sw[padded(i)]) >> (t & 31);
     if (x & 1u) {
-      if (t + 1 + w > nbits) break;                                   // truncated token: reported by the link kernel
+      if (t + 1 + w > left) break;                                    // truncated token: reported by the link kernel
       uint32_t o = w ? (__brev(uint32_t(x >> 1)) >> (32 - w)) : 0u;
       int64_t j = blk * int64_t(B) + o;
       if (o >= B || j >= d) bad = true;
       else if (k < cap) idx[k] = int32_t(j);
       ++k; t += 1 + w;
-    } else { ++blk; ++t; }
+    } else {                                                           // a run of closing bits
+      int z = min(x ? __ffsll((long long)x) - 1 : 64, min(32 - (t & 31) + 32, e - t));
+      blk += z; t += z;
+    }
   }
   if (bad) atomicOr(reinterpret_cast<unsigned long long*>(result + 2), 4ull);
 }
@@ -298,14 +360,12 @@ int mv_pos_decode(void* stream, const uint32_t* words, int64_t nbits, int64_t d,
   int64_t* ent_b1 = reinterpret_cast<int64_t*>(base + L.b1);
   int64_t* ent_b0 = reinterpret_cast<int64_t*>(base + L.b0);
   int64_t nblocks = (d + B - 1) / B;
-  if (L.nseg > 0) {
-    int64_t threads = L.nseg * (w + 1);
-    k_pos_scan<<<unsigned((threads + 127) / 128), 128, 0, st>>>(words, nbits, w, L.nseg, map);
-  }
-  k_pos_link<<<1, LINK_TILE, size_t(LINK_TILE) * (w + 1) * 4, st>>>(map, w, L.nseg, nblocks, cap, ent_state, ent_b1, ent_b0, result);
   if (L.nseg > 0)
-    k_pos_emit<<<unsigned((L.nseg + 63) / 64), 64, 0, st>>>(words, nbits, d, uint32_t(B), w, L.nseg, ent_state, ent_b1, ent_b0,
-                                                              idx, cap, result);
+    k_pos_scan<<<unsigned((L.nseg + SCAN_SEGS - 1) / SCAN_SEGS), SCAN_SEGS * (w + 1), 0, st>>>(words, nbits, w, L.nseg, map);
+  k_pos_link<<<1, (LINK_TILE / LINK_CHUNK) * (w + 1) > LINK_TILE ? (LINK_TILE / LINK_CHUNK) * (w + 1) : LINK_TILE, size_t(LINK_TILE) * (w + 1) * 4, st>>>(map, w, L.nseg, nblocks, cap, ent_state, ent_b1, ent_b0, result);
+  if (L.nseg > 0)
+    k_pos_emit<<<unsigned((L.nseg + EMIT_SEGS - 1) / EMIT_SEGS), EMIT_SEGS, 0, st>>>(words, nbits, d, uint32_t(B), w, L.nseg, ent_state,
+                                                                                  ent_b1, ent_b0, idx, cap, result);
   return cuda_ok();
 }
 
