@@ -223,7 +223,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2", choices=["c1", "c1_ties", "c2", "c3", "c4"])
-    ap.add_argument("--mode", default="auto", choices=["auto", "general"])
+    ap.add_argument("--mode", default="track", choices=["auto", "general", "track"],
+                    help="how the per-worker candidate threshold is found: sampled every step (auto), carried from "
+                         "the previous step's key histogram (track), or none (general)")
     ap.add_argument("--method", default="mv", choices=["mv", "ad"],
                     help="mv: plain majority voting (Algorithm 1); ad: add-drop voting (Algorithm 2) with K_ad = K/10")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -265,7 +267,7 @@ def main():
     err = WL.initial_err(w, device=dev)
     out_idx = torch.empty(w.K, dtype=torch.int32, device=dev)
     out_val = torch.empty(w.K, dtype=torch.float32, device=dev)
-    ctx = B.MvContext(w.N, w.d, w.K, device=dev, mode=B.MV_MODE_GENERAL if args.mode == "general" else B.MV_MODE_AUTO)
+    ctx = B.MvContext(w.N, w.d, w.K, device=dev, mode={"auto": B.MV_MODE_AUTO, "general": B.MV_MODE_GENERAL, "track": B.MV_MODE_TRACK}[args.mode])
 
     sampler = ClockSampler(visible_gpu_index(local_rank))
     sampler.start()
@@ -344,10 +346,13 @@ def main():
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic", "config": dict(workload_config(w), method=("add-drop voting, K_ad=K/10" if args.method == "ad"
-                                                                     else "majority voting")),
+                                                                     else "majority voting"),
+                                          threshold={"track": "candidate threshold carried from the previous step's key histogram",
+                                                     "auto": "candidate threshold sampled every step",
+                                                     "general": "no candidate threshold (multi-pass select)"}[args.mode]),
         "effective_gradient_gbs": w.N * w.d * 4 / (ms_step * 1e-3) / 1e9 * 1.0,
         "step_roofline_frac": alg_bytes / (ms_step * 1e-3) / 1e9 / peak,
-        "roofline": {"bound": "hbm", "kernel": "k_acc_compact" if args.mode == "auto" else "k_row_hist<1,true>",
+        "roofline": {"bound": "hbm", "kernel": "k_acc_compact" if args.mode != "general" else "k_row_hist<1,true>",
                      "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
                      "frac": (achieved / peak) if achieved else None, "traffic": traffic,
                      "kernel_ms": k_ms_avg, "kernel_launches_timed": k_cnt, "algorithmic_bytes_per_launch": alg_bytes},

@@ -53,7 +53,12 @@ enum {
 
 enum {
   MV_MODE_AUTO = 0,    /* sampled threshold + single streaming pass, exact multi-pass select as fallback */
-  MV_MODE_GENERAL = 1  /* always the exact multi-pass radix select (no sampling) */
+  MV_MODE_GENERAL = 1, /* always the exact multi-pass radix select (no sampling) */
+  MV_MODE_TRACK = 2    /* as AUTO, but a call that follows one with the same N, d, K on the same context takes
+                          its candidate threshold from that call's key histogram instead of sampling: meant
+                          for the consecutive steps of one training run, where |acc| changes slowly.  Exact
+                          for any input: a worker whose threshold turns out unusable (fewer than K or more
+                          than 4K + 4096 candidates) takes the multi-pass select for that call. */
 };
 
 typedef struct mv_ctx mv_ctx;

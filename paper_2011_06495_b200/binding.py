@@ -24,6 +24,7 @@ MV_ERR_TOO_LARGE = -4
 MV_SELECT_STATIC_MAX_D = 1 << 24
 MV_MODE_AUTO = 0
 MV_MODE_GENERAL = 1
+MV_MODE_TRACK = 2
 
 _lib = None
 

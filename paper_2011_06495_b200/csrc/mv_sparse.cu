@@ -62,7 +62,11 @@ struct P {
   uint32_t* votes_done;   // [1]
   uint8_t* hot;           // [nc_pad] 1 if any worker kept a candidate in the chunk
   uint32_t* vote_hist;    // [256]
-  uint32_t* tau;          // [N]
+  uint32_t* tau;          // [N] candidate threshold of this call
+  uint32_t* tau_next;     // [N] threshold proposed for the next call (threshold tracking), or null
+  uint32_t track_rank;    // rank, among this call's counted keys, at which the next call's threshold is put
+  uint32_t* hist2b;       // [N][H2_BINS] second digit within the first-digit bin of track_rank (if not the K-th key's)
+  uint32_t* tstate;       // [N][2] that bin and the rank within it (0 = rank not reached)
   uint32_t* diag_cnt;     // [N] copy of cand_cnt that survives the end-of-step clearing
   uint32_t* wstate;       // [N][8]: b1, rem1, b2, rem2, T, cnt_gt, cnt_eq, need
   uint32_t* thresh;       // [N][3]
@@ -473,14 +477,27 @@ __global__ void __launch_bounds__(TPB) k_acc_compact(P p, const float* __restric
 // digit q among the elements whose higher digits match.
 // ---------------------------------------------------------------------------------------------
 template <int PASS>
-__device__ __forceinline__ uint32_t resolve_prefix(const P& p, int n) {
+__device__ __forceinline__ uint32_t resolve_prefix(const P& p, int n, uint32_t& track_bin) {
   uint32_t* ws = p.wstate + (size_t)n * 8;
+  track_bin = 0xffffffffu;  // no second tracked bin unless pass 2 finds one
   if (PASS == 2) {
     uint32_t b1, rem1;
     block_pick<H1_BINS, TPB>(p.hist1 + (size_t)n * H1_BINS, worker_K(p, n), b1, rem1);
     if (blockIdx.x == 0 && threadIdx.x == 0) {
       ws[0] = b1;
       ws[1] = rem1;
+    }
+    if (p.tau_next != nullptr) {
+      // threshold tracking: the next call's candidate threshold is put at rank K + margin among the
+      // keys counted in this call (the candidates, or the whole row).  This pass finds the first
+      // digit of that rank; the second digit is counted alongside the K-th key's.
+      uint32_t tb, trem;
+      block_pick<H1_BINS, TPB>(p.hist1 + (size_t)n * H1_BINS, p.track_rank, tb, trem);
+      if (blockIdx.x == 0 && threadIdx.x == 0) {
+        p.tstate[n * 2 + 0] = tb;
+        p.tstate[n * 2 + 1] = trem;
+      }
+      if (trem != 0 && tb != b1) track_bin = tb;
     }
     return b1;
   }
@@ -491,6 +508,17 @@ __device__ __forceinline__ uint32_t resolve_prefix(const P& p, int n) {
     if (blockIdx.x == 0 && threadIdx.x == 0) {
       ws[2] = b2;
       ws[3] = rem2;
+    }
+    if (p.tau_next != nullptr && blockIdx.x == 0) {  // CTA-uniform: one CTA settles the next call's threshold
+      const uint32_t tb = p.tstate[n * 2 + 0], trem = p.tstate[n * 2 + 1];
+      uint32_t tb2 = 0, trem2 = 0;
+      if (trem != 0)  // uniform over the CTA
+        block_pick<H2_BINS, TPB>((tb == b1 ? p.hist2 : p.hist2b) + (size_t)n * H2_BINS, trem, tb2, trem2);
+      if (threadIdx.x == 0) {
+        // rank not reached by the counted keys: one first-digit bin below this call's threshold
+        const uint32_t cur = p.tau[n] >> 20;
+        p.tau_next[n] = trem != 0 ? ((tb << 20) | (tb2 << 10)) : (cur ? ((cur - 1) << 20) : 0u);
+      }
     }
     return (b1 << 10) | b2;
   }
@@ -521,11 +549,12 @@ __device__ __forceinline__ uint32_t resolve_threshold(const P& p, int n, uint32_
 }
 
 template <int PASS>
-__device__ __forceinline__ void hist_add(uint32_t* sh, uint32_t key, uint32_t prefix) {
+__device__ __forceinline__ void hist_add(uint32_t* sh, uint32_t key, uint32_t prefix, uint32_t* sh2, uint32_t track_bin) {
   if (PASS == 1) {
     atomicAdd(&sh[key >> 20], 1u);
   } else if (PASS == 2) {
     if ((key >> 20) == prefix) atomicAdd(&sh[(key >> 10) & 1023u], 1u);
+    else if ((key >> 20) == track_bin) atomicAdd(&sh2[(key >> 10) & 1023u], 1u);
   } else {
     if ((key >> 10) == prefix) atomicAdd(&sh[key & 1023u], 1u);
   }
@@ -550,8 +579,12 @@ __global__ void __launch_bounds__(TPB) k_hist(P p, const float* __restrict__ gra
   const int n = blockIdx.y;
   const bool fast = !FUSED && worker_fast(p, n);
   if (p.list_mode && !fast) return;  // empty list
-  const uint32_t prefix = resolve_prefix<PASS>(p, n);
+  __shared__ uint32_t sh2[PASS == 2 ? H2_BINS : 1];
+  uint32_t track_bin;
+  const uint32_t prefix = resolve_prefix<PASS>(p, n, track_bin);
   for (int b = threadIdx.x; b < NB; b += TPB) sh[b] = 0;
+  if (PASS == 2 && track_bin != 0xffffffffu)
+    for (int b = threadIdx.x; b < H2_BINS; b += TPB) sh2[b] = 0;
   __syncthreads();
   if (fast) {
     const uint32_t cnt = p.cand_cnt[n];
@@ -568,7 +601,7 @@ __global__ void __launch_bounds__(TPB) k_hist(P p, const float* __restrict__ gra
 #pragma unroll
       for (int q = 0; q < 4; q++) {
         if (b0 + q * stride >= cnt) break;  // warp-uniform
-        if (b0 + q * stride + lane < cnt) hist_add<PASS>(sh, k[q], prefix);
+        if (b0 + q * stride + lane < cnt) hist_add<PASS>(sh, k[q], prefix, sh2, track_bin);
       }
     }
   } else {
@@ -584,13 +617,13 @@ __global__ void __launch_bounds__(TPB) k_hist(P p, const float* __restrict__ gra
       for (int i = 0; i < 4; i++)
 #pragma unroll
         for (int e = 0; e < 4; e++)
-          if (vm[i] & (1u << e)) hist_add<PASS>(sh, key[i][e], prefix);
+          if (vm[i] & (1u << e)) hist_add<PASS>(sh, key[i][e], prefix, sh2, track_bin);
       if (threadIdx.x == TPB - 1) {
         uint32_t xkey[4], xvm;
         load_extra<FUSED>(g, grads, err, xkey, xvm);
 #pragma unroll
         for (int e = 0; e < 4; e++)
-          if (xvm & (1u << e)) hist_add<PASS>(sh, xkey[e], prefix);
+          if (xvm & (1u << e)) hist_add<PASS>(sh, xkey[e], prefix, sh2, track_bin);
       }
     }
   }
@@ -599,6 +632,13 @@ __global__ void __launch_bounds__(TPB) k_hist(P p, const float* __restrict__ gra
   for (int b = threadIdx.x; b < NB; b += TPB) {
     const uint32_t v = sh[b];
     if (v) atomicAdd(&gh[b], v);
+  }
+  if (PASS == 2 && track_bin != 0xffffffffu) {
+    uint32_t* gh2 = p.hist2b + (size_t)n * H2_BINS;
+    for (int b = threadIdx.x; b < H2_BINS; b += TPB) {
+      const uint32_t v = sh2[b];
+      if (v) atomicAdd(&gh2[b], v);
+    }
   }
 }
 
@@ -1321,8 +1361,8 @@ struct Layout {
   int64_t W;
   uint32_t cap;
   size_t zero_bytes;  // the leading region cleared at the start of every vote
-  size_t samp_hist, hist1, hist2, hist3, cand_cnt, sample_done, count_done, votes_done, hot, vote_hist;
-  size_t tau, diag_cnt, wstate, thresh, vstate, cand, chunk_base, chunk_cnt, chunk_eq, tie_base, chunk_sel;
+  size_t samp_hist, hist1, hist2, hist2b, hist3, cand_cnt, sample_done, count_done, votes_done, hot, vote_hist;
+  size_t tau, tau_alt, tstate, diag_cnt, wstate, thresh, vstate, cand, chunk_base, chunk_cnt, chunk_eq, tie_base, chunk_sel;
   size_t worker_bits, worker_idx, votes, chunk_vh, out_base, tie_take;
   // add-drop voting: the select state once more, for 2N lists of at most ad_cap entries
   uint32_t ad_cap;
@@ -1355,6 +1395,7 @@ Layout make_layout(int N, int64_t d, int64_t K) {
   L.hist1 = take(off, n * H1_BINS * 4);
   L.hist2 = take(off, n * H2_BINS * 4);
   L.hist3 = take(off, n * H3_BINS * 4);
+  L.hist2b = take(off, n * H2_BINS * 4);
   L.cand_cnt = take(off, n * 4);
   L.sample_done = take(off, n * 4);
   L.count_done = take(off, n * 4);
@@ -1363,6 +1404,8 @@ Layout make_layout(int N, int64_t d, int64_t K) {
   L.vote_hist = take(off, 256 * 4);
   L.zero_bytes = off;
   L.tau = take(off, n * 4);
+  L.tau_alt = take(off, n * 4);
+  L.tstate = take(off, n * 2 * 4);
   L.diag_cnt = take(off, n * 4);
   L.wstate = take(off, n * 8 * 4);
   L.thresh = take(off, n * 3 * 4);
@@ -1433,6 +1476,11 @@ struct mv_ctx {
   // remembered for mv_read_diag
   int last_N;
   int64_t last_d, last_K;
+  // threshold tracking (MV_MODE_TRACK): the two tau arrays alternate between "this call" and "next call"
+  int tau_flip;       // which array holds the thresholds of the current (or last) call
+  bool track_valid;   // the previous call left thresholds for (track_N, track_d, track_K)
+  int track_N;
+  int64_t track_d, track_K;
 };
 
 namespace {
@@ -1461,7 +1509,11 @@ P make_params(const mv_ctx* ctx, const Layout& L, int N, int64_t d, int64_t K) {
   p.votes_done = (uint32_t*)(b + L.votes_done);
   p.hot = (uint8_t*)(b + L.hot);
   p.vote_hist = (uint32_t*)(b + L.vote_hist);
-  p.tau = (uint32_t*)(b + L.tau);
+  p.tau = (uint32_t*)(b + (ctx->tau_flip ? L.tau_alt : L.tau));
+  p.tau_next = nullptr;
+  p.track_rank = 0;
+  p.hist2b = (uint32_t*)(b + L.hist2b);
+  p.tstate = (uint32_t*)(b + L.tstate);
   p.diag_cnt = (uint32_t*)(b + L.diag_cnt);
   p.wstate = (uint32_t*)(b + L.wstate);
   p.thresh = (uint32_t*)(b + L.thresh);
@@ -1593,12 +1645,30 @@ int vote_impl(mv_ctx* ctx, P p, const Layout& L, const float* grads, float* err,
   const int gh = p.force_general ? per_row_ctas(N, p.nchunks, 148 * 8)
                                  : per_row_ctas(N, (int)((p.cap + TPB * 8 - 1) / (TPB * 8)), 148 * 2);
   if (!p.force_general) {
-    uint32_t U, Ls, rank;
-    int all;
-    sample_plan(p.d, p.K, U, Ls, all, rank);
-    const int gs = per_row_ctas(N, (int)((U + 127) / 128), 148 * 2);
-    launch_k(k_sample_hist, dim3(dim3(gs, N)), dim3(512), st, p, grads, err, U, Ls, all, rank);
-    MV_LAUNCH_CHECK();
+    // threshold tracking: the previous call on this context, if it had the same N, d and K, left a
+    // threshold per worker in the other tau array; this call reads it instead of sampling and
+    // leaves its own proposal in the array it does not read
+    const bool track = ctx->mode == MV_MODE_TRACK;
+    const bool tracked = track && ctx->track_valid && ctx->track_N == N && ctx->track_d == p.d && ctx->track_K == p.K;
+    if (tracked) ctx->tau_flip ^= 1;
+    p.tau = (uint32_t*)(ctx->ws + (ctx->tau_flip ? L.tau_alt : L.tau));
+    if (track) {
+      p.tau_next = (uint32_t*)(ctx->ws + (ctx->tau_flip ? L.tau : L.tau_alt));
+      const double r = ceil((double)p.K * 1.25 + 6.0 * sqrt((double)p.K) + 8.0);
+      p.track_rank = (uint32_t)(r < (double)p.d ? r : (double)p.d);
+      ctx->track_valid = true;
+      ctx->track_N = N;
+      ctx->track_d = p.d;
+      ctx->track_K = p.K;
+    }
+    if (!tracked) {
+      uint32_t U, Ls, rank;
+      int all;
+      sample_plan(p.d, p.K, U, Ls, all, rank);
+      const int gs = per_row_ctas(N, (int)((U + 127) / 128), 148 * 2);
+      launch_k(k_sample_hist, dim3(dim3(gs, N)), dim3(512), st, p, grads, err, U, Ls, all, rank);
+      MV_LAUNCH_CHECK();
+    }
     if (ctx->timing_now) cudaEventRecord(ctx->ev[2 * (ctx->timed % 64)], st);
     launch_k(k_acc_compact, dim3(dim3(p.nchunks, N)), dim3(TPB), st, p, grads, err);
     MV_LAUNCH_CHECK();
@@ -1703,6 +1773,8 @@ int mv_create(mv_ctx** out, void* stream, void* workspace, size_t workspace_byte
   c->ws = (char*)workspace;
   c->ws_bytes = workspace_bytes;
   c->mode = MV_MODE_AUTO;
+  c->tau_flip = 0;
+  c->track_valid = false;
   c->launches = 0;
   c->clean_bytes = 0;
   c->timing = 0;
@@ -1797,8 +1869,10 @@ int mv_read_kernel_timing(mv_ctx* ctx, float* total_ms, int* launches) {
 }
 
 int mv_set_mode(mv_ctx* ctx, int mode) {
-  if (ctx == nullptr || (mode != MV_MODE_AUTO && mode != MV_MODE_GENERAL)) return MV_ERR_INVALID_ARG;
+  if (ctx == nullptr || (mode != MV_MODE_AUTO && mode != MV_MODE_GENERAL && mode != MV_MODE_TRACK))
+    return MV_ERR_INVALID_ARG;
   ctx->mode = mode;
+  ctx->track_valid = false;
   return MV_OK;
 }
 
@@ -1994,7 +2068,8 @@ int mv_read_diag(mv_ctx* ctx, int N, uint32_t* per_worker) {
   if (cnt == nullptr) return MV_ERR_INVALID_ARG;
   uint32_t* tau = cnt + N;
   cudaError_t e = cudaMemcpyAsync(cnt, ctx->ws + L.diag_cnt, (size_t)N * 4, cudaMemcpyDeviceToHost, ctx->stream);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(tau, ctx->ws + L.tau, (size_t)N * 4, cudaMemcpyDeviceToHost, ctx->stream);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(tau, ctx->ws + (ctx->tau_flip ? L.tau_alt : L.tau), (size_t)N * 4, cudaMemcpyDeviceToHost, ctx->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
   if (e != cudaSuccess) {
     free(cnt);

@@ -25,15 +25,15 @@ THREADS = max(1, min(16, len(os.sched_getaffinity(0))))
 FULL = os.environ.get("MV_TEST_QUICK", "0") != "1"     # MV_TEST_QUICK=1: fewer steps and 9 of the 27 sweep cells
 
 
-def run_config(w, steps):
+def run_config(w, steps, mode=B.MV_MODE_AUTO):
     std = WL.std_vector(w, DEV) if w.segments > 1 else None
-    ctx = B.MvContext(w.N, w.d, w.K, device=DEV)
+    ctx = B.MvContext(w.N, w.d, w.K, device=DEV, mode=mode)
     err = WL.initial_err(w, device=DEV)
     err_ref = err.cpu().numpy()
     out_idx = torch.empty(w.K, dtype=torch.int32, device=DEV)
     out_val = torch.empty(w.K, dtype=torch.float32, device=DEV)
     grads = torch.empty((w.N, w.d), dtype=torch.float32, device=DEV)
-    fallbacks = 0
+    fallbacks = []
     for step in range(steps):
         WL.gradients(w, step, out=grads, std=std)
         g_np = grads.cpu().numpy()
@@ -49,7 +49,7 @@ def run_config(w, steps):
             del ph
         ctx.mv_sparse_step(grads, err, out_idx, out_val)
         torch.cuda.synchronize()
-        fallbacks += int(ctx.read_diag(w.N)[:, 2].sum())
+        fallbacks.append(int(ctx.read_diag(w.N)[:, 2].sum()))
         PT.first_diff(PT.npy(out_idx), ref["out_idx"], tag + "out_idx")
         PT.check_out_val(PT.npy(out_val), ref, ref["acc"], ref["out_idx"].astype(np.int64), tag + "out_val")
         PT.first_diff(PT.bits(PT.npy(err)), PT.bits(ref["err"]), tag + "err")
@@ -58,12 +58,18 @@ def run_config(w, steps):
     return fallbacks
 
 
+@pytest.mark.parametrize("mode", [B.MV_MODE_AUTO, B.MV_MODE_TRACK], ids=["auto", "track"])
 @pytest.mark.parametrize("name", ["c2", "c3", "c4"])
-def test_named_config_every_step(name):
+def test_named_config_every_step(name, mode):
     w = WL.resnet_like(name)
     steps = w.steps if (FULL or name == "c2") else min(w.steps, 8)
-    fallbacks = run_config(w, steps)
-    assert fallbacks == 0, f"{fallbacks} worker-steps fell back to the full-row select on smooth data"
+    if mode == B.MV_MODE_TRACK and name != "c2":
+        steps = min(steps, 12)
+    fallbacks = run_config(w, steps, mode)
+    # a tracked threshold may miss while the residuals build up from zero (|acc| grows by tens of
+    # per cent per step there); from then on, and always with a sampled threshold, nobody falls back
+    settled = fallbacks[4:] if mode == B.MV_MODE_TRACK else fallbacks
+    assert sum(settled) == 0, f"worker-steps that fell back to the full-row select on smooth data, per step: {fallbacks}"
 
 
 def _cells():

@@ -12,7 +12,8 @@ from tests import parity as PT
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
-MODES = [B.MV_MODE_AUTO, B.MV_MODE_GENERAL]
+MODES = [B.MV_MODE_AUTO, B.MV_MODE_GENERAL, B.MV_MODE_TRACK]
+MODE_IDS = ["auto", "general", "track"]
 
 
 def make(N, d, kind, seed):
@@ -56,7 +57,7 @@ SHAPES = [
 ]
 
 
-@pytest.mark.parametrize("mode", MODES, ids=["auto", "general"])
+@pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
 @pytest.mark.parametrize("kind", ["gauss", "ties", "layers"])
 @pytest.mark.parametrize("N,d,K", SHAPES)
 def test_shapes(N, d, K, kind, mode):
@@ -65,7 +66,7 @@ def test_shapes(N, d, K, kind, mode):
     PT.compare_all(ctx, grads.to(DEV), err.to(DEV), K, by_sort=(d <= 20000), label=f"[{N}x{d} K={K} {kind}] ")
 
 
-@pytest.mark.parametrize("mode", MODES, ids=["auto", "general"])
+@pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
 @pytest.mark.parametrize("kind", ["equal", "zeros", "sparse"])
 @pytest.mark.parametrize("N,d,K", [(3, 5000, 17), (4, 20011, 300), (2, 300007, 10)])
 def test_degenerate(N, d, K, kind, mode):
@@ -82,7 +83,7 @@ def test_max_workers():
 
 
 @pytest.mark.parametrize("name", ["c1", "c1_ties"])
-@pytest.mark.parametrize("mode", MODES, ids=["auto", "general"])
+@pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
 def test_config_c1(name, mode):
     w = WL.resnet_like(name)
     grads = WL.gradients(w, 0)
@@ -190,6 +191,77 @@ def test_error_feedback_over_steps():
         PT.check_out_val(PT.npy(out_val), ref, ref["acc"], ref["out_idx"].astype(np.int64), f"step {step} out_val")
         PT.first_diff(PT.bits(PT.npy(err_gpu)), PT.bits(ref["err"]), f"step {step} err")
         err_ref = ref["err"]
+
+
+@pytest.mark.parametrize("N,d,K", [(6, 200003, 2000), (3, 1000003, 250), (4, 50000, 5000), (2, 4097, 7)])
+def test_threshold_tracking_over_steps(N, d, K):
+    """MV_MODE_TRACK: after the first call the candidate threshold comes from the previous call's key
+    histogram (one kernel fewer); every step stays bit-identical to the oracle, and on slowly
+    changing data no worker needs the fallback."""
+    w = WL.scaled(WL.resnet_like("c2"), d=d, N=N, K=K, steps=7)
+    ctx = B.MvContext(w.N, w.d, w.K, device=DEV, mode=B.MV_MODE_TRACK)
+    err_gpu = WL.initial_err(w).to(DEV)
+    err_ref = WL.initial_err(w).numpy()
+    out_idx = torch.empty(w.K, dtype=torch.int32, device=DEV)
+    out_val = torch.empty(w.K, dtype=torch.float32, device=DEV)
+    launches = []
+    for step in range(w.steps):
+        grads = WL.gradients(w, step)
+        ref = O.mv_sparse_step(grads.numpy(), err_ref, w.K)
+        ctx.mv_sparse_step(grads.to(DEV), err_gpu, out_idx, out_val)
+        torch.cuda.synchronize()
+        launches.append(ctx.last_launches())
+        diag = ctx.read_diag(w.N)
+        PT.first_diff(PT.npy(out_idx), ref["out_idx"], f"step {step} out_idx")
+        PT.check_out_val(PT.npy(out_val), ref, ref["acc"], ref["out_idx"].astype(np.int64), f"step {step} out_val")
+        PT.first_diff(PT.bits(PT.npy(err_gpu)), PT.bits(ref["err"]), f"step {step} err")
+        if step >= 2:
+            assert (diag[:, 2] == 0).all(), f"step {step}: fallback with a tracked threshold: {diag.tolist()}"
+        err_ref = ref["err"]
+    assert launches[0] == launches[1] + 1 and len(set(launches[1:])) == 1      # the sampling kernel runs once
+
+
+def test_threshold_tracking_survives_a_change_of_scale():
+    """The tracked threshold is only a guess: when the data jumps by orders of magnitude between two
+    calls the affected workers take the exact multi-pass select for that call and results stay exact;
+    the call after that is back on the fast path.  Another (d, K) on the same context samples again."""
+    N, d, K = 4, 300007, 3000
+    ctx = B.MvContext(N, d, K, device=DEV, mode=B.MV_MODE_TRACK)
+    grads, err = make(N, d, "gauss", seed=31)
+    scales = [1.0, 1.0, 1e3, 1e3, 1e-4, 1e-4, 1.0]
+    fell_back = []
+    for step, sc in enumerate(scales):
+        g = (grads * sc).roll(step, dims=1).contiguous()
+        e = (err * sc).contiguous()
+        g[1] = grads[1].roll(step)                      # worker 1 keeps its scale throughout
+        e[1] = err[1]
+        ref = O.mv_sparse_step(g.numpy(), e.numpy(), K)
+        fu = PT.run_step(ctx, g.to(DEV), e.to(DEV), K)
+        fell_back.append(ctx.read_diag(N)[:, 2].tolist())
+        PT.first_diff(PT.npy(fu["out_idx"]), ref["out_idx"], f"step {step} out_idx")
+        PT.check_out_val(PT.npy(fu["out_val"]), ref, ref["acc"], ref["out_idx"].astype(np.int64), f"step {step} out_val")
+        PT.first_diff(PT.bits(PT.npy(fu["err"])), PT.bits(ref["err"]), f"step {step} err")
+    assert fell_back[0] == [0, 0, 0, 0] and fell_back[1] == [0, 0, 0, 0]
+    assert fell_back[2] == [1, 0, 1, 1] and fell_back[4] == [1, 0, 1, 1] and fell_back[6] == [1, 0, 1, 1]
+    assert fell_back[3] == [0, 0, 0, 0] and fell_back[5] == [0, 0, 0, 0]
+    # a smaller problem on the same context: nothing is carried over
+    d2, K2 = 100003, 500
+    g2, e2 = make(N, d2, "gauss", seed=32)
+    ref = O.mv_sparse_step(g2.numpy(), e2.numpy(), K2)
+    out_idx = torch.empty(K2, dtype=torch.int32, device=DEV)
+    out_val = torch.empty(K2, dtype=torch.float32, device=DEV)
+    e2g = e2.to(DEV)
+    before = None
+    for rep in range(2):
+        e2g.copy_(e2)
+        ctx.mv_sparse_step(g2.to(DEV), e2g, out_idx, out_val, K=K2)
+        torch.cuda.synchronize()
+        PT.first_diff(PT.npy(out_idx), ref["out_idx"], f"second problem, call {rep}")
+        PT.first_diff(PT.bits(PT.npy(e2g)), PT.bits(ref["err"]), f"second problem, call {rep} err")
+        assert (ctx.read_diag(N)[:, 2] == 0).all()
+        if rep == 0:
+            before = ctx.last_launches()
+    assert ctx.last_launches() == before - 1
 
 
 def test_checkpoint_resume():
