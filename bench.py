@@ -29,6 +29,7 @@ import torch  # noqa: E402
 
 from paper_2011_06495_b200 import workloads as WL  # noqa: E402
 
+RS_SEED = 201106495
 METRIC = "majority-vote sparse steps/s"
 UNIT = "steps/s"
 FALLBACK_HBM_GBS = 6650.0
@@ -162,6 +163,9 @@ def oracle_steps_per_s(w: WL.Workload, steps: int, sample_workers: int, warmup: 
         if method == "ad":
             r = O.mv_ad_step(g, err, prev, ws.K, max(1, ws.K // 10))
             prev = r["prev"]
+        elif method == "rs":
+            from oracle import rs_oracle as R
+            r = R.mv_rs_step(g, err, ws.K, RS_SEED, s)
         else:
             r = O.mv_sparse_step(g, err, ws.K)
         dt = time.perf_counter() - t0
@@ -226,8 +230,9 @@ def main():
     ap.add_argument("--mode", default="track", choices=["auto", "general", "track"],
                     help="how the per-worker candidate threshold is found: sampled every step (auto), carried from "
                          "the previous step's key histogram (track), or none (general)")
-    ap.add_argument("--method", default="mv", choices=["mv", "ad"],
-                    help="mv: plain majority voting (Algorithm 1); ad: add-drop voting (Algorithm 2) with K_ad = K/10")
+    ap.add_argument("--method", default="mv", choices=["mv", "ad", "rs"],
+                    help="mv: plain majority voting (Algorithm 1); ad: add-drop voting (Algorithm 2) with K_ad = K/10; "
+                         "rs: random selection proportional to the votes (Algorithm 1, second variant)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -277,6 +282,12 @@ def main():
 
         def one_step(g):
             ctx.mv_ad_step(g, err, prev_bits, K_ad, out_idx, out_val)
+    elif args.method == "rs":
+        draw = [0]
+
+        def one_step(g):
+            ctx.mv_rs_step(g, err, RS_SEED, draw[0], out_idx, out_val)
+            draw[0] += 1
     else:
         def one_step(g):
             ctx.mv_sparse_step(g, err, out_idx, out_val)
@@ -345,8 +356,8 @@ def main():
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
-        "data": "synthetic", "config": dict(workload_config(w), method=("add-drop voting, K_ad=K/10" if args.method == "ad"
-                                                                     else "majority voting"),
+        "data": "synthetic", "config": dict(workload_config(w), method={"ad": "add-drop voting, K_ad=K/10", "rs": "random selection proportional to the votes",
+                                                  "mv": "majority voting"}[args.method],
                                           threshold={"track": "candidate threshold carried from the previous step's key histogram",
                                                      "auto": "candidate threshold sampled every step",
                                                      "general": "no candidate threshold (multi-pass select)"}[args.mode]),

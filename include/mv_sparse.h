@@ -121,6 +121,30 @@ int mv_ad_step(mv_ctx* ctx, const float* grads, float* err, uint32_t* prev_bits,
                int64_t K_ad, int32_t* out_idx, float* out_val, uint32_t* add_bits, uint32_t* drop_bits,
                uint8_t* msum);
 
+/* Majority voting with random selection (SSGD-MV-RS: Algorithm 1 with the S_rand-weighted line; Section
+ * 4.1 words it as "select indices at random using the votes until K unique indices are selected").
+ * The shared mask is a draw of successive sampling proportional to the votes, taken with one random
+ * number per coordinate (exponential clocks): coordinate j with v_j > 0 votes gets the ring time
+ * t_j = E_j / v_j, E_j = -ln((x_j + 1/2) / 2^32), x_j = first output word of Philox4x32-10 with key
+ * (seed low, seed high) and counter (j, 0, draw low, draw high); the K smallest t_j win.  So that a
+ * CPU statement of the same rule gives the same indices, every deciding operation is fixed: -ln by
+ * the binary64 recipe v = 2x+1, e = floor(log2 v), m = v/2^e (halved and e+1 if m > sqrt 2),
+ * s = (m-1)/(m+1), ln m = 2s(1 + s^2/3 + ... + s^22/23) by Horner from the 1/23 end,
+ * E = (33-e) ln2 - ln m; t_j is one binary64 division rounded once to binary32; equal t_j go to the
+ * lowest index.  Coordinates without a vote are never selected; if fewer than K hold a vote, the
+ * tail of out_idx is filled with -1.  The same (seed, draw) gives the same mask; use a new `draw`
+ * every step.
+ *
+ * mv_select_rs: votes [d] uint8 in: the count of at most N workers voting for at most K coordinates each
+ *              (so at most N K coordinates hold a vote; with more than that nothing is selected and
+ *              out_idx is all -1); out_idx [K] out ascending; mask_bits may be NULL.
+ * mv_rs_step:  as mv_sparse_step with this selection in place of the K most voted (the union of the
+ *              workers' top-K sets always holds at least K coordinates, so out_idx is full). */
+int mv_select_rs(mv_ctx* ctx, const uint8_t* votes, int N, int64_t d, int64_t K, uint64_t seed, uint64_t draw,
+                 int32_t* out_idx, uint32_t* mask_bits);
+int mv_rs_step(mv_ctx* ctx, const float* grads, float* err, int N, int64_t d, int64_t K, uint64_t seed, uint64_t draw,
+               int32_t* out_idx, float* out_val);
+
 /* mv_select for callers that cannot hand the library a workspace.  (The paper has no counterpart
  * to this call: it is the same selection as mv_select, packaged differently.)
  *

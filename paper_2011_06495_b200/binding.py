@@ -82,6 +82,11 @@ def load() -> ctypes.CDLL:
     lib.mv_last_launches.argtypes = [c_vp]
     lib.mv_status_string.restype = ctypes.c_char_p
     lib.mv_status_string.argtypes = [c_i]
+    c_u64 = ctypes.c_uint64
+    lib.mv_select_rs.restype = c_i
+    lib.mv_select_rs.argtypes = [c_vp, c_vp, c_i, c_i64, c_i64, c_u64, c_u64, c_vp, c_vp]
+    lib.mv_rs_step.restype = c_i
+    lib.mv_rs_step.argtypes = [c_vp, c_vp, c_vp, c_i, c_i64, c_i64, c_u64, c_u64, c_vp, c_vp]
     # wire formats (include/mv_wire.h)
     lib.mv_pos_offset_bits.restype = c_i
     lib.mv_pos_offset_bits.argtypes = [c_i64]
@@ -234,6 +239,15 @@ class MvContext:
         _check(self.lib.mv_ad_step(self.handle, _ptr(grads), _ptr(err), _ptr(prev_bits), N, d, K or self.K, int(K_ad),
                                    _ptr(out_idx), _ptr(out_val), _ptr(add_bits), _ptr(drop_bits), _ptr(msum)),
                "mv_ad_step")
+
+    def mv_select_rs(self, votes, N: int, seed: int, draw: int, out_idx, mask_bits=None, K: Optional[int] = None):
+        _check(self.lib.mv_select_rs(self.handle, _ptr(votes), int(N), votes.numel(), int(K or self.K), int(seed), int(draw),
+                                     _ptr(out_idx), _ptr(mask_bits)), "mv_select_rs")
+
+    def mv_rs_step(self, grads, err, seed: int, draw: int, out_idx, out_val, K: Optional[int] = None):
+        N, d = grads.shape
+        _check(self.lib.mv_rs_step(self.handle, _ptr(grads), _ptr(err), int(N), int(d), int(K or self.K), int(seed), int(draw),
+                                   _ptr(out_idx), _ptr(out_val)), "mv_rs_step")
 
     def mv_sparse_step_host(self, h_grads, h_out_idx, h_out_val, d_grads, d_err, d_out_idx, d_out_val,
                             K: Optional[int] = None):

@@ -105,7 +105,7 @@ __device__ __forceinline__ uint32_t lanemask_lt() {
 __device__ __forceinline__ bool worker_fast(const P& p, int n) {
   if (p.force_general) return false;
   const uint32_t c = p.cand_cnt[n];
-  if (p.list_mode) return c > 0;
+  if (p.list_mode) return c > 0 && c <= p.cap;  // a list that overflowed its room counts as empty
   return c >= (uint32_t)p.K && c <= p.cap;
 }
 
@@ -1341,6 +1341,110 @@ __global__ void __launch_bounds__(TPB) k_ad_fill(P p, P a, const uint32_t* __res
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// random selection (SSGD-MV-RS: Algorithm 1 with the S_rand-weighted line).  Coordinate j with
+// v_j > 0 votes rings at time E_j / v_j, E_j = -ln u_j, u_j = (x_j + 1/2) / 2^32, x_j the first word
+// of Philox4x32-10 (key = seed, counter = (j, 0, draw)); the K earliest ring times are a draw of
+// "sample proportionally to the votes until K distinct indices" (exponential clocks, Efraimidis and
+// Spirakis).  Everything that decides an index is a fixed sequence of IEEE operations: the
+// logarithm below uses binary64 +, *, / only, the ring time is one binary64 division rounded once
+// to binary32, equal times go to the lowest index.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t philox4x32_10_first(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0,
+                                                        uint32_t k1) {
+#pragma unroll
+  for (int r = 0; r < 10; r++) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    c0 = hi1 ^ c1 ^ k0;
+    c1 = lo1;
+    c2 = hi0 ^ c3 ^ k1;
+    c3 = lo0;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  return c0;
+}
+
+__device__ __forceinline__ double neg_log_u(uint32_t x) {
+  const unsigned long long v = 2ull * x + 1ull;  // u = v / 2^33
+  int e = 63 - __clzll((long long)v);
+  double m = __ddiv_rn((double)v, (double)(1ull << e));  // [1, 2), exact
+  if (m > 1.4142135623730951) {
+    m = __dmul_rn(m, 0.5);
+    e += 1;
+  }
+  const double s = __ddiv_rn(__dadd_rn(m, -1.0), __dadd_rn(m, 1.0));
+  const double z = __dmul_rn(s, s);
+  double poly = 1.0 / 23.0;
+#pragma unroll
+  for (int k = 21; k >= 1; k -= 2) poly = __dadd_rn(__dmul_rn(poly, z), 1.0 / (double)k);
+  const double logm = __dmul_rn(__dmul_rn(2.0, s), poly);
+  return __dsub_rn(__dmul_rn((double)(33 - e), 0.6931471805599453), logm);
+}
+
+// A CTA per chunk: thread t owns coordinates 16t .. 16t+15 of the chunk, so thread order is index
+// order.  Voted coordinates are appended to the single list `a` (row 0) as (0x7fffffff - ring time
+// bits, index): the list-mode select then keeps the K largest keys, i.e. the K earliest times.
+__global__ void __launch_bounds__(TPB) k_rs_fill(P p, P a, const uint8_t* __restrict__ votes, uint32_t seed_lo,
+                                                 uint32_t seed_hi, uint32_t draw_lo, uint32_t draw_hi) {
+  pdl_enter();
+  __shared__ uint32_t s_w[TPB / 32 + 1];
+  __shared__ uint32_t s_base;
+  const int c = blockIdx.x;
+  const int64_t j0 = (int64_t)c * CH + threadIdx.x * 16;
+  uint8_t v[16];
+  if (j0 + 16 <= p.d) {
+    const uint4 q = __ldcg(reinterpret_cast<const uint4*>(votes + j0));
+    const uint32_t w4[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int i = 0; i < 16; i++) v[i] = (uint8_t)(w4[i >> 2] >> (8 * (i & 3)));
+  } else {
+#pragma unroll
+    for (int i = 0; i < 16; i++) v[i] = j0 + i < p.d ? votes[j0 + i] : (uint8_t)0;
+  }
+  uint32_t cnt = 0;
+#pragma unroll
+  for (int i = 0; i < 16; i++) cnt += v[i] != 0;
+  uint32_t total;
+  uint32_t pos = block_excl_scan<TPB>(cnt, s_w, total);
+  if (threadIdx.x == 0) {
+    const uint32_t base = total ? atomicAdd(&a.cand_cnt[0], total) : 0u;
+    s_base = base;
+    a.chunk_base[c] = base;
+    a.chunk_cnt[c] = total;
+  }
+  __syncthreads();
+  if (cnt == 0) return;
+  pos += s_base;
+#pragma unroll
+  for (int i = 0; i < 16; i++) {
+    if (v[i] == 0) continue;
+    const uint32_t j = (uint32_t)(j0 + i);
+    const uint32_t x = philox4x32_10_first(j, 0u, draw_lo, draw_hi, seed_lo, seed_hi);
+    const double t = __ddiv_rn(neg_log_u(x), (double)v[i]);
+    const uint32_t tb = __float_as_uint(__double2float_rn(t));
+    if (pos < a.cap) a.cand[pos] = make_uint2(0x7fffffffu - tb, j);
+    pos++;
+  }
+}
+
+// selected coordinates per chunk of one bit-mask row (a warp per chunk)
+__global__ void __launch_bounds__(TPB) k_chunk_popc(const uint32_t* __restrict__ bits, int64_t W, int nchunks,
+                                                    uint32_t* __restrict__ chunk_sel) {
+  pdl_enter();
+  const int c = blockIdx.x * (TPB / 32) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (c >= nchunks) return;
+  uint32_t s = 0;
+#pragma unroll
+  for (int q = 0; q < 4; q++) {
+    const int64_t wi = (int64_t)c * WPC + q * 32 + lane;
+    if (wi < W) s += __popc(__ldcg(bits + wi));
+  }
+  s = __reduce_add_sync(FULL, s);
+  if (lane == 0) chunk_sel[c] = s;
+}
+
 __global__ void __launch_bounds__(TPB) k_ad_apply(uint32_t* __restrict__ prev_bits, const uint32_t* __restrict__ ad_bits,
                                                   uint32_t* __restrict__ add_out, uint32_t* __restrict__ drop_out,
                                                   size_t words /* N*W */) {
@@ -1368,6 +1472,7 @@ struct Layout {
   uint32_t ad_cap;
   size_t ad_zero, ad_zero_bytes;  // cleared at the start of every add-drop vote
   size_t ad_hist1, ad_hist2, ad_hist3, ad_cnt, ad_count_done, ad_bits;
+  size_t rs_chunk_sel;  // [nchunks] random selection: selected coordinates per chunk, then their offsets
   size_t ad_wstate, ad_thresh, ad_diag, ad_cand, ad_chunk_base, ad_chunk_cnt, ad_chunk_eq, ad_tie_base;
   size_t total;
 };
@@ -1437,6 +1542,7 @@ Layout make_layout(int N, int64_t d, int64_t K) {
     L.ad_thresh = take(off, m * 3 * 4);
     L.ad_diag = take(off, m * 4);
     L.ad_cand = take(off, m * (size_t)L.ad_cap * 8);
+    L.rs_chunk_sel = take(off, nc * 4);
     L.ad_chunk_base = take(off, m * nc * 4);
     L.ad_chunk_cnt = take(off, m * nc * 4);
     L.ad_chunk_eq = take(off, m * nc * 4);
@@ -2038,6 +2144,124 @@ int mv_ad_step(mv_ctx* ctx, const float* grads, float* err, uint32_t* prev_bits,
   rc = select_impl(ctx, v, L, v.votes, true, out_idx, nullptr);
   if (rc != MV_OK) return rc;
   return aggregate_impl(ctx, err, N, d, K, out_idx, out_val, L.zero_bytes);
+}
+
+}  // extern "C" (reopened below)
+
+namespace {
+
+// P for the add-drop / random-selection lists: the select state once more, over `rows` lists
+P list_params(const mv_ctx* ctx, const Layout& L, const P& p, int rows, int64_t K_list, uint32_t cap) {
+  char* b = ctx->ws;
+  P a = p;
+  a.N = rows;
+  a.K = K_list;
+  a.cap = cap;
+  a.list_mode = 1;
+  a.force_general = 0;
+  a.tau_next = nullptr;
+  a.hist1 = (uint32_t*)(b + L.ad_hist1);
+  a.hist2 = (uint32_t*)(b + L.ad_hist2);
+  a.hist3 = (uint32_t*)(b + L.ad_hist3);
+  a.cand_cnt = (uint32_t*)(b + L.ad_cnt);
+  a.count_done = (uint32_t*)(b + L.ad_count_done);
+  a.worker_bits = (uint32_t*)(b + L.ad_bits);
+  a.wstate = (uint32_t*)(b + L.ad_wstate);
+  a.thresh = (uint32_t*)(b + L.ad_thresh);
+  a.diag_cnt = (uint32_t*)(b + L.ad_diag);
+  a.cand = (uint2*)(b + L.ad_cand);
+  a.chunk_base = (uint32_t*)(b + L.ad_chunk_base);
+  a.chunk_cnt = (uint32_t*)(b + L.ad_chunk_cnt);
+  a.chunk_eq = (uint32_t*)(b + L.ad_chunk_eq);
+  a.tie_base = (uint32_t*)(b + L.ad_tie_base);
+  a.apply_rows = 0;
+  a.apply_bits = nullptr;
+  return a;
+}
+
+// S_rand-weighted: voted coordinates with their ring times into one list, the K earliest through the
+// list-mode select into a bit mask, the mask into an ascending index list
+int rs_select_impl(mv_ctx* ctx, const P& p, const Layout& L, const uint8_t* votes, uint64_t seed, uint64_t draw,
+                   int32_t* out_idx, uint32_t* mask_bits) {
+  cudaStream_t st = ctx->stream;
+  char* b = ctx->ws;
+  // one list that can hold every voted coordinate (at most min(d, N K) of them)
+  const uint64_t room = (uint64_t)2 * (uint64_t)p.N * (uint64_t)L.ad_cap;
+  P a = list_params(ctx, L, p, 1, p.K, (uint32_t)(room < 0xfffffff8ull ? room : 0xfffffff8ull));
+  if (cudaMemsetAsync(b + L.ad_zero, 0, (L.ad_bits - L.ad_zero) + (size_t)p.W * 4, st) != cudaSuccess) return MV_ERR_CUDA;
+  if (cudaMemsetAsync(out_idx, 0xff, (size_t)p.K * 4, st) != cudaSuccess) return MV_ERR_CUDA;
+  launch_k(k_rs_fill, dim3(p.nchunks), dim3(TPB), st, p, a, votes, (uint32_t)seed, (uint32_t)(seed >> 32), (uint32_t)draw,
+           (uint32_t)(draw >> 32));
+  MV_LAUNCH_CHECK();
+  uint64_t most = (uint64_t)p.N * (uint64_t)p.K;
+  if (most > (uint64_t)p.d) most = (uint64_t)p.d;
+  const int ga = per_row_ctas(1, (int)((most + TPB * 8 - 1) / (TPB * 8)), 148 * 2);
+  launch_k(k_hist<1, false>, dim3(dim3(ga, 1)), dim3(TPB), st, a, nullptr, nullptr);
+  MV_LAUNCH_CHECK();
+  launch_k(k_hist<2, false>, dim3(dim3(ga, 1)), dim3(TPB), st, a, nullptr, nullptr);
+  MV_LAUNCH_CHECK();
+  launch_k(k_hist<3, false>, dim3(dim3(ga, 1)), dim3(TPB), st, a, nullptr, nullptr);
+  MV_LAUNCH_CHECK();
+  launch_k(k_count, dim3(dim3(ga, 1)), dim3(TPB), st, a, nullptr);
+  MV_LAUNCH_CHECK();
+  launch_k(k_set_bits, dim3(dim3(ga, 1)), dim3(TPB), st, a, nullptr);
+  MV_LAUNCH_CHECK();
+  P r = a;
+  r.list_mode = 0;
+  r.chunk_sel = (uint32_t*)(b + L.rs_chunk_sel);
+  r.worker_idx = out_idx;
+  launch_k(k_chunk_popc, dim3((p.nchunks + TPB / 32 - 1) / (TPB / 32)), dim3(TPB), st, (const uint32_t*)a.worker_bits, p.W,
+           p.nchunks, r.chunk_sel);
+  MV_LAUNCH_CHECK();
+  launch_k(k_scan_sel, dim3(1), dim3(1024), st, r);
+  MV_LAUNCH_CHECK();
+  launch_k(k_lists, dim3(dim3((p.nchunks + TPB / 32 - 1) / (TPB / 32), 1)), dim3(TPB), st, r);
+  MV_LAUNCH_CHECK();
+  if (mask_bits &&
+      cudaMemcpyAsync(mask_bits, a.worker_bits, (size_t)p.W * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return MV_ERR_CUDA;
+  return MV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int mv_select_rs(mv_ctx* ctx, const uint8_t* votes, int N, int64_t d, int64_t K, uint64_t seed, uint64_t draw,
+                 int32_t* out_idx, uint32_t* mask_bits) {
+  Layout L;
+  const int rc = check_common(ctx, N, d, K, L);
+  if (rc != MV_OK) return rc;
+  if (votes == nullptr || out_idx == nullptr || !aligned16(votes) || !aligned16(out_idx)) return MV_ERR_INVALID_ARG;
+  if (mask_bits && !aligned16(mask_bits)) return MV_ERR_INVALID_ARG;
+  ctx->launches = 0;
+  if (ctx->phase_timing) cudaEventRecord(ctx->pev[0], ctx->stream);
+  const P p = make_params(ctx, L, N, d, K);
+  return rs_select_impl(ctx, p, L, votes, seed, draw, out_idx, mask_bits);
+}
+
+int mv_rs_step(mv_ctx* ctx, const float* grads, float* err, int N, int64_t d, int64_t K, uint64_t seed, uint64_t draw,
+               int32_t* out_idx, float* out_val) {
+  Layout L;
+  int rc = check_common(ctx, N, d, K, L);
+  if (rc != MV_OK) return rc;
+  if (grads == nullptr || err == nullptr || out_idx == nullptr || out_val == nullptr) return MV_ERR_INVALID_ARG;
+  if (!aligned16(grads) || !aligned16(err) || !aligned16(out_idx) || !aligned16(out_val)) return MV_ERR_INVALID_ARG;
+  const size_t nb = (size_t)N * (size_t)d * 4;
+  if (overlap(grads, nb, err, nb)) return MV_ERR_INVALID_ARG;
+  ctx->launches = 0;
+  if (ctx->phase_timing) cudaEventRecord(ctx->pev[0], ctx->stream);
+  P p = make_params(ctx, L, N, d, K);
+  ctx->last_N = N;
+  ctx->last_d = d;
+  ctx->last_K = K;
+  rc = vote_impl(ctx, p, L, grads, err);
+  // the union of N top-K sets holds at least K coordinates, so the mask is always full
+  if (rc == MV_OK) rc = rs_select_impl(ctx, p, L, p.votes, seed, draw, out_idx, nullptr);
+  // the vote count's own scan is not consumed here: the gather clears its state with the rest
+  if (rc == MV_OK) rc = aggregate_impl(ctx, err, N, d, K, out_idx, out_val, L.zero_bytes);
+  const int rcj = join_side(ctx);
+  return rc != MV_OK ? rc : rcj;
 }
 
 int mv_sparse_step_host(mv_ctx* ctx, const float* h_grads, int N, int64_t d, int64_t K, int32_t* h_out_idx,
