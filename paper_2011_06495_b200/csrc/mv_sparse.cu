@@ -298,6 +298,60 @@ __device__ void block_pick(const uint32_t* __restrict__ hist, uint32_t rank, uin
   __syncthreads();
 }
 
+// block_pick for two ranks of the same histogram in one sweep (same contract for each rank).
+template <int NB, int NT>
+__device__ void block_pick2(const uint32_t* __restrict__ hist, uint32_t rank_a, uint32_t rank_b, uint32_t& bin_a,
+                            uint32_t& rem_a, uint32_t& bin_b, uint32_t& rem_b) {
+  constexpr int PER = NB / NT;
+  __shared__ uint32_t s_wsum[NT / 32];
+  __shared__ uint32_t s_res[4];
+  const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+  uint32_t loc[PER];
+  uint32_t sum = 0;
+#pragma unroll
+  for (int k = 0; k < PER; k++) {
+    loc[k] = __ldcg(hist + t * PER + k);
+    sum += loc[k];
+  }
+  if (t < 4) s_res[t] = 0;
+  uint32_t x = sum;  // inclusive suffix sum within the warp
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const uint32_t y = __shfl_down_sync(FULL, x, off);
+    if (lane + off < 32) x += y;
+  }
+  if (lane == 0) s_wsum[warp] = x;
+  __syncthreads();
+  uint32_t above0 = x - sum;
+  for (int w = warp + 1; w < NT / 32; w++) above0 += s_wsum[w];
+#pragma unroll
+  for (int which = 0; which < 2; which++) {
+    const uint32_t rank = which ? rank_b : rank_a;
+    uint32_t above = above0;
+    if (above < rank && rank <= above + sum) {
+      bool done = false;
+#pragma unroll
+      for (int k = PER - 1; k >= 0; k--) {
+        if (!done) {
+          if (above + loc[k] >= rank) {
+            s_res[2 * which] = (uint32_t)(t * PER + k);
+            s_res[2 * which + 1] = rank - above;
+            done = true;
+          } else {
+            above += loc[k];
+          }
+        }
+      }
+    }
+  }
+  __syncthreads();
+  bin_a = s_res[0];
+  rem_a = s_res[1];
+  bin_b = s_res[2];
+  rem_b = s_res[3];
+  __syncthreads();
+}
+
 // Exclusive prefix sum over the threads of a CTA (NT = 256 or 1024); `total` gets the CTA sum.
 template <int NT>
 __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* s_w /*NT/32 + 1*/, uint32_t& total) {
@@ -482,39 +536,46 @@ __device__ __forceinline__ uint32_t resolve_prefix(const P& p, int n, uint32_t& 
   track_bin = 0xffffffffu;  // no second tracked bin unless pass 2 finds one
   if (PASS == 2) {
     uint32_t b1, rem1;
-    block_pick<H1_BINS, TPB>(p.hist1 + (size_t)n * H1_BINS, worker_K(p, n), b1, rem1);
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-      ws[0] = b1;
-      ws[1] = rem1;
-    }
-    if (p.tau_next != nullptr) {
+    if (p.tau_next == nullptr) {
+      block_pick<H1_BINS, TPB>(p.hist1 + (size_t)n * H1_BINS, worker_K(p, n), b1, rem1);
+    } else {
       // threshold tracking: the next call's candidate threshold is put at rank K + margin among the
       // keys counted in this call (the candidates, or the whole row).  This pass finds the first
       // digit of that rank; the second digit is counted alongside the K-th key's.
       uint32_t tb, trem;
-      block_pick<H1_BINS, TPB>(p.hist1 + (size_t)n * H1_BINS, p.track_rank, tb, trem);
+      block_pick2<H1_BINS, TPB>(p.hist1 + (size_t)n * H1_BINS, worker_K(p, n), p.track_rank, b1, rem1, tb, trem);
       if (blockIdx.x == 0 && threadIdx.x == 0) {
         p.tstate[n * 2 + 0] = tb;
         p.tstate[n * 2 + 1] = trem;
       }
       if (trem != 0 && tb != b1) track_bin = tb;
     }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+      ws[0] = b1;
+      ws[1] = rem1;
+    }
     return b1;
   }
   if (PASS == 3) {
     const uint32_t b1 = ws[0], rem1 = ws[1];
     uint32_t b2, rem2;
-    block_pick<H2_BINS, TPB>(p.hist2 + (size_t)n * H2_BINS, rem1, b2, rem2);
+    // threshold tracking: CTA 0 also settles the next call's threshold (second digit of its rank)
+    const bool settle = p.tau_next != nullptr && blockIdx.x == 0;  // CTA-uniform
+    uint32_t tb = 0, trem = 0, tb2 = 0, trem2 = 0;
+    if (settle) {
+      tb = p.tstate[n * 2 + 0];
+      trem = p.tstate[n * 2 + 1];
+    }
+    if (settle && trem != 0 && tb == b1) {  // the usual case: both ranks in the same first-digit bin
+      block_pick2<H2_BINS, TPB>(p.hist2 + (size_t)n * H2_BINS, rem1, trem, b2, rem2, tb2, trem2);
+    } else {
+      block_pick<H2_BINS, TPB>(p.hist2 + (size_t)n * H2_BINS, rem1, b2, rem2);
+      if (settle && trem != 0) block_pick<H2_BINS, TPB>(p.hist2b + (size_t)n * H2_BINS, trem, tb2, trem2);
+    }
     if (blockIdx.x == 0 && threadIdx.x == 0) {
       ws[2] = b2;
       ws[3] = rem2;
-    }
-    if (p.tau_next != nullptr && blockIdx.x == 0) {  // CTA-uniform: one CTA settles the next call's threshold
-      const uint32_t tb = p.tstate[n * 2 + 0], trem = p.tstate[n * 2 + 1];
-      uint32_t tb2 = 0, trem2 = 0;
-      if (trem != 0)  // uniform over the CTA
-        block_pick<H2_BINS, TPB>((tb == b1 ? p.hist2 : p.hist2b) + (size_t)n * H2_BINS, trem, tb2, trem2);
-      if (threadIdx.x == 0) {
+      if (settle) {
         // rank not reached by the counted keys: one first-digit bin below this call's threshold
         const uint32_t cur = p.tau[n] >> 20;
         p.tau_next[n] = trem != 0 ? ((tb << 20) | (tb2 << 10)) : (cur ? ((cur - 1) << 20) : 0u);
