@@ -446,10 +446,42 @@ __global__ void __launch_bounds__(512) k_sample_hist(P p, const float* __restric
 // stream: acc = err + grads in place; elements with key >= tau_n appended, in index order, to the
 // chunk's own run of the worker's candidate buffer (one global atomic per chunk that has any)
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(TPB) k_acc_compact(P p, const float* __restrict__ grads, float* __restrict__ err) {
+// Writes this thread's candidates at CTA-local positions off + (ordered rank) through `put(pos, entry)`.
+template <typename PUT>
+__device__ __forceinline__ void emit_candidates(const Geom& g, const uint32_t (&key)[4][4], const uint32_t (&cm)[4],
+                                                const uint32_t (&xkey)[4], uint32_t xcm, const uint32_t* s_w, PUT put) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  uint32_t off = 0;
+  for (int w = 0; w < warp; w++) off += s_w[w];
+  const uint32_t lt = lanemask_lt();
+#pragma unroll
+  for (int i = 0; i < 4; i++) {
+    uint32_t rank0, tot;
+    iter_ranks(cm[i], lt, rank0, tot);
+    if (cm[i]) {
+      const int jf = g.j0 - g.h + 4 * (warp * 128 + i * 32 + lane);
+#pragma unroll
+      for (int e = 0; e < 4; e++)
+        if (cm[i] & (1u << e)) put(off + rank0 + __popc(cm[i] & ((1u << e) - 1u)), make_uint2(key[i][e], (uint32_t)(jf + e)));
+    }
+    off += tot;
+  }
+  if (threadIdx.x == TPB - 1 && xcm) {
+    uint32_t xoff = 0;
+    for (int w = 0; w < 8; w++) xoff += s_w[w];
+    const int jf = g.j0 - g.h + 4096;
+#pragma unroll
+    for (int e = 0; e < 4; e++)
+      if (xcm & (1u << e)) put(xoff + __popc(xcm & ((1u << e) - 1u)), make_uint2(xkey[e], (uint32_t)(jf + e)));
+  }
+}
+
+__global__ void __launch_bounds__(TPB, 4) k_acc_compact(P p, const float* __restrict__ grads, float* __restrict__ err) {
   pdl_enter();
+  constexpr uint32_t QCAP = 1024;  // candidates of a chunk staged in shared memory (more: written directly)
   __shared__ uint32_t s_w[9];
-  __shared__ uint32_t s_base, s_total;
+  __shared__ uint32_t s_base;
+  __shared__ uint2 s_q[QCAP];
   const int n = blockIdx.y, c = blockIdx.x;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const Geom g = chunk_geom(n, c, p.d);
@@ -460,7 +492,7 @@ __global__ void __launch_bounds__(TPB) k_acc_compact(P p, const float* __restric
     const int64_t wi = (int64_t)c * WPC + threadIdx.x;
     if (wi < p.W) p.worker_bits[(size_t)n * p.W + wi] = 0u;
   }
-  uint32_t xkey[4], xcm = 0;
+  uint32_t xkey[4] = {0, 0, 0, 0}, xcm = 0;
   if (threadIdx.x == TPB - 1) {
     uint32_t xvm;
     load_extra<true>(g, grads, err, xkey, xvm);
@@ -476,52 +508,44 @@ __global__ void __launch_bounds__(TPB) k_acc_compact(P p, const float* __restric
   if (lane == 0) s_w[warp] = wsum;
   if (threadIdx.x == TPB - 1) s_w[8] = __popc(xcm);
   __syncthreads();
+  uint32_t total = 0;
+#pragma unroll
+  for (int w = 0; w < 9; w++) total += s_w[w];
+  // the chunk's run in the worker's candidate buffer: one reservation per chunk that has any,
+  // issued now and consumed after the staging, so that its round trip overlaps with it
+  uint32_t base_r = 0;
   if (threadIdx.x == 0) {
-    uint32_t total = 0;
-    for (int w = 0; w < 9; w++) total += s_w[w];
-    uint32_t base = 0;
     if (total) {
-      base = atomicAdd(&p.cand_cnt[n], total);
+      base_r = atomicAdd(&p.cand_cnt[n], total);
       p.hot[c] = 1;  // same value from every worker: a plain store is enough
     }
-    p.chunk_base[(size_t)n * p.nchunks + c] = base;
     p.chunk_cnt[(size_t)n * p.nchunks + c] = total;
-    s_base = base;
-    s_total = total;
+    if (total == 0) p.chunk_base[(size_t)n * p.nchunks + c] = 0;
   }
-  __syncthreads();
-  if (s_total == 0) return;
-  uint32_t off = s_base;
-  for (int w = 0; w < warp; w++) off += s_w[w];
+  if (total == 0) return;  // uniform over the CTA
   uint2* out = p.cand + (size_t)n * p.cap;
-  const uint32_t lt = lanemask_lt();
-#pragma unroll
-  for (int i = 0; i < 4; i++) {
-    uint32_t rank0, tot;
-    iter_ranks(cm[i], lt, rank0, tot);
-    if (cm[i]) {
-      const int jf = g.j0 - g.h + 4 * (warp * 128 + i * 32 + lane);
-#pragma unroll
-      for (int e = 0; e < 4; e++) {
-        if (cm[i] & (1u << e)) {
-          const uint32_t pos = off + rank0 + __popc(cm[i] & ((1u << e) - 1u));
-          if (pos < p.cap) out[pos] = make_uint2(key[i][e], (uint32_t)(jf + e));
-        }
-      }
+  if (total <= QCAP) {
+    // stage in index order, then copy out coalesced: whole sectors instead of 8-byte pieces
+    emit_candidates(g, key, cm, xkey, xcm, s_w, [&](uint32_t pos, uint2 v) { s_q[pos] = v; });
+    if (threadIdx.x == 0) {
+      s_base = base_r;
+      p.chunk_base[(size_t)n * p.nchunks + c] = base_r;
     }
-    off += tot;
-  }
-  if (threadIdx.x == TPB - 1 && xcm) {
-    uint32_t xoff = s_base;
-    for (int w = 0; w < 8; w++) xoff += s_w[w];
-    const int jf = g.j0 - g.h + 4096;
-#pragma unroll
-    for (int e = 0; e < 4; e++) {
-      if (xcm & (1u << e)) {
-        const uint32_t pos = xoff + __popc(xcm & ((1u << e) - 1u));
-        if (pos < p.cap) out[pos] = make_uint2(xkey[e], (uint32_t)(jf + e));
-      }
+    __syncthreads();
+    const uint32_t base = s_base;
+    for (uint32_t i = threadIdx.x; i < total; i += TPB)
+      if (base + i < p.cap) out[base + i] = s_q[i];
+  } else {
+    if (threadIdx.x == 0) {
+      s_base = base_r;
+      p.chunk_base[(size_t)n * p.nchunks + c] = base_r;
     }
+    __syncthreads();
+    const uint32_t base = s_base;
+    const uint32_t cap = p.cap;
+    emit_candidates(g, key, cm, xkey, xcm, s_w, [&](uint32_t pos, uint2 v) {
+      if (base + pos < cap) out[base + pos] = v;
+    });
   }
 }
 
@@ -576,9 +600,19 @@ __device__ __forceinline__ uint32_t resolve_prefix(const P& p, int n, uint32_t& 
       ws[2] = b2;
       ws[3] = rem2;
       if (settle) {
-        // rank not reached by the counted keys: one first-digit bin below this call's threshold
-        const uint32_t cur = p.tau[n] >> 20;
-        p.tau_next[n] = trem != 0 ? ((tb << 20) | (tb2 << 10)) : (cur ? ((cur - 1) << 20) : 0u);
+        uint32_t next = (tb << 20) | (tb2 << 10);
+        if (trem == 0) {
+          // The counted keys (c candidates, all >= tau) do not reach the rank: go below tau by linear
+          // extrapolation in key space from the two ranks that are known, (K, K-th key) and (c, tau),
+          // with a quarter to spare; at least 2^10 and at most half a first-digit bin per call.
+          const uint32_t tau = p.tau[n], c = p.cand_cnt[n], K = worker_K(p, n);
+          const uint32_t t21 = (b1 << 20) | (b2 << 10);
+          const float slope = (t21 > tau && c >= K) ? (float)(t21 - tau) / (float)(c - K + 1u) : 0.f;
+          float drop = 1.25f * slope * (float)(p.track_rank > c ? p.track_rank - c : 1u);
+          drop = fminf(fmaxf(drop, 1024.f), 524288.f);
+          next = tau > (uint32_t)drop ? tau - (uint32_t)drop : 0u;
+        }
+        p.tau_next[n] = next;
       }
     }
     return (b1 << 10) | b2;
@@ -1821,7 +1855,7 @@ int vote_impl(mv_ctx* ctx, P p, const Layout& L, const float* grads, float* err,
     p.tau = (uint32_t*)(ctx->ws + (ctx->tau_flip ? L.tau_alt : L.tau));
     if (track) {
       p.tau_next = (uint32_t*)(ctx->ws + (ctx->tau_flip ? L.tau : L.tau_alt));
-      const double r = ceil((double)p.K * 1.25 + 6.0 * sqrt((double)p.K) + 8.0);
+      const double r = ceil((double)p.K * 1.35 + 6.0 * sqrt((double)p.K) + 8.0);
       p.track_rank = (uint32_t)(r < (double)p.d ? r : (double)p.d);
       ctx->track_valid = true;
       ctx->track_N = N;

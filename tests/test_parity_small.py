@@ -221,6 +221,36 @@ def test_threshold_tracking_over_steps(N, d, K):
     assert launches[0] == launches[1] + 1 and len(set(launches[1:])) == 1      # the sampling kernel runs once
 
 
+@pytest.mark.parametrize("name,N,d,K", [("c3", 8, 400_009, 400), ("c2", 6, 300_007, 3000), ("c4", 4, 500_003, 125)])
+def test_threshold_tracking_long_run(name, N, d, K):
+    """Hundreds of consecutive steps: the tracked threshold neither drifts out of the usable range
+    (no fallback once the residuals have built up) nor oscillates; the last step is compared with
+    the oracle from the device's own residual state."""
+    w = WL.scaled(WL.resnet_like(name), d=d, N=N, K=K, steps=1)
+    ctx = B.MvContext(w.N, w.d, w.K, device=DEV, mode=B.MV_MODE_TRACK)
+    pool = [WL.gradients(w, s, device=DEV) for s in range(5)]
+    err = WL.initial_err(w, device=DEV)
+    out_idx = torch.empty(w.K, dtype=torch.int32, device=DEV)
+    out_val = torch.empty(w.K, dtype=torch.float32, device=DEV)
+    fallbacks, ratio = [], []
+    steps = 600
+    for step in range(steps):
+        if step == steps - 1:
+            err_before = err.cpu().numpy()
+        ctx.mv_sparse_step(pool[step % 5], err, out_idx, out_val)
+        if step % 7 == 0 or step == steps - 1:
+            diag = ctx.read_diag(w.N)
+            fallbacks.append(int(diag[:, 2].sum()))
+            ratio.append(float(diag[:, 0].max()) / w.K)
+    torch.cuda.synchronize()
+    assert sum(fallbacks[2:]) == 0, f"fallbacks at sampled steps: {fallbacks}"
+    assert max(ratio[2:]) < 3.5 and min(ratio[2:]) >= 1.0, f"candidates per K out of range: {ratio}"
+    ref = O.mv_sparse_step(PT.npy(pool[(steps - 1) % 5]), err_before, w.K)
+    PT.first_diff(PT.npy(out_idx), ref["out_idx"], "last step out_idx")
+    PT.check_out_val(PT.npy(out_val), ref, ref["acc"], ref["out_idx"].astype(np.int64), "last step out_val")
+    PT.first_diff(PT.bits(PT.npy(err)), PT.bits(ref["err"]), "last step err")
+
+
 def test_threshold_tracking_survives_a_change_of_scale():
     """The tracked threshold is only a guess: when the data jumps by orders of magnitude between two
     calls the affected workers take the exact multi-pass select for that call and results stay exact;
