@@ -15,6 +15,7 @@ import argparse
 import hashlib
 import json
 import os
+import re
 import subprocess
 import sys
 import tempfile
@@ -45,9 +46,34 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
+STREAM_KERNEL_FUNCTIONS = ("pdl_enter", "fkey", "lanemask_lt", "chunk_geom", "load_keys", "load_extra", "iter_ranks",
+                           "ge_mask", "emit_candidates", "k_acc_compact")
+
+
+def function_text(text: str, name: str) -> str:
+    """Source text of the first __device__/__global__ function called `name` (signature through closing brace)."""
+    for m in re.finditer(r"^[^\n;{}]*\b" + re.escape(name) + r"\s*\(", text, flags=re.M):
+        line_start = text.rfind("\n", 0, m.start()) + 1
+        head = text[max(0, line_start - 200):m.end()]
+        if "__device__" not in head and "__global__" not in head:
+            continue
+        i = text.index("{", m.end())
+        depth, j = 1, i + 1
+        while depth:
+            depth += {"{": 1, "}": -1}.get(text[j], 0)
+            j += 1
+        return text[line_start:j]
+    raise KeyError(name)
+
+
 def kernel_source_hash():
+    """Hash of the streaming kernel and of the device functions it calls (the counters in
+    profiles/traffic.json belong to exactly this text)."""
     src = os.path.join(ROOT, "paper_2011_06495_b200", "csrc", "mv_sparse.cu")
-    return hashlib.sha256(open(src, "rb").read()).hexdigest()[:16]
+    text = open(src).read()
+    consts = "".join(re.findall(r"^constexpr[^\n]*\n", text, flags=re.M))
+    body = consts + "".join(function_text(text, f) for f in STREAM_KERNEL_FUNCTIONS)
+    return hashlib.sha256(body.encode()).hexdigest()[:16]
 
 
 def recorded_traffic(workload: str, n_units: int):
