@@ -121,6 +121,22 @@ int mv_ad_step(mv_ctx* ctx, const float* grads, float* err, uint32_t* prev_bits,
                int64_t K_ad, int32_t* out_idx, float* out_val, uint32_t* add_bits, uint32_t* drop_bits,
                uint8_t* msum);
 
+/* Worker-sharded step (the paper's remark under Eq. 8 that a shared mask lets the values be summed by
+ * an all-reduce): when the N workers are spread over several GPUs, each rank runs mv_vote on its
+ * N_local rows, the vote counts (uint8 [d]) are summed over the ranks, every rank runs mv_select on
+ * the summed votes with N = the total number of workers, mv_aggregate_partial gives the rank's
+ * binary64 partial sums on the shared mask (and zeroes its workers' residual there), the partial
+ * sums are summed over the ranks and mv_finish_mean divides by the total number of workers and
+ * rounds once to binary32.  The two sums over ranks are the caller's collectives; the library only
+ * provides the two kernels that a single-GPU step does not need.
+ *   out_sum [K] double out: sum over this rank's workers, in worker order, of acc[n][idx[k]]
+ *   sum     [K] double in : the sum of all ranks' out_sum;  out_val [K] float out
+ * Differences from the single-GPU mean: only the order in which the binary64 terms of different
+ * ranks are added (fixed by the collective), i.e. at most a last-bit difference after rounding. */
+int mv_aggregate_partial(mv_ctx* ctx, float* acc, int N_local, int64_t d, int64_t K, const int32_t* idx,
+                         double* out_sum);
+int mv_finish_mean(void* stream, const double* sum, int64_t K, int N_total, float* out_val);
+
 /* Majority voting with random selection (SSGD-MV-RS: Algorithm 1 with the S_rand-weighted line; Section
  * 4.1 words it as "select indices at random using the votes until K unique indices are selected").
  * The shared mask is a draw of successive sampling proportional to the votes, taken with one random

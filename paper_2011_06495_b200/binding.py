@@ -87,6 +87,10 @@ def load() -> ctypes.CDLL:
     lib.mv_select_rs.argtypes = [c_vp, c_vp, c_i, c_i64, c_i64, c_u64, c_u64, c_vp, c_vp]
     lib.mv_rs_step.restype = c_i
     lib.mv_rs_step.argtypes = [c_vp, c_vp, c_vp, c_i, c_i64, c_i64, c_u64, c_u64, c_vp, c_vp]
+    lib.mv_aggregate_partial.restype = c_i
+    lib.mv_aggregate_partial.argtypes = [c_vp, c_vp, c_i, c_i64, c_i64, c_vp, c_vp]
+    lib.mv_finish_mean.restype = c_i
+    lib.mv_finish_mean.argtypes = [c_vp, c_vp, c_i64, c_i, c_vp]
     # wire formats (include/mv_wire.h)
     lib.mv_pos_offset_bits.restype = c_i
     lib.mv_pos_offset_bits.argtypes = [c_i64]
@@ -248,6 +252,15 @@ class MvContext:
         N, d = grads.shape
         _check(self.lib.mv_rs_step(self.handle, _ptr(grads), _ptr(err), int(N), int(d), int(K or self.K), int(seed), int(draw),
                                    _ptr(out_idx), _ptr(out_val)), "mv_rs_step")
+
+    def mv_aggregate_partial(self, acc, idx, out_sum):
+        N, d = acc.shape
+        _check(self.lib.mv_aggregate_partial(self.handle, _ptr(acc), N, d, idx.numel(), _ptr(idx), _ptr(out_sum)),
+               "mv_aggregate_partial")
+
+    def mv_finish_mean(self, total, N_total: int, out_val):
+        _check(self.lib.mv_finish_mean(ctypes.c_void_p(self.stream.cuda_stream), _ptr(total), total.numel(), int(N_total),
+                                       _ptr(out_val)), "mv_finish_mean")
 
     def mv_sparse_step_host(self, h_grads, h_out_idx, h_out_val, d_grads, d_err, d_out_idx, d_out_val,
                             K: Optional[int] = None):

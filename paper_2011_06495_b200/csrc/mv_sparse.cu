@@ -1330,7 +1330,8 @@ __global__ void __launch_bounds__(TPB) k_vote_write(P p, const uint8_t* __restri
 // so that the next step can start without a separate memset; zero_vecs = 0 switches that off.
 __global__ void __launch_bounds__(TPB) k_gather(float* __restrict__ acc, int N, int64_t d, int64_t K,
                                                 const int32_t* __restrict__ idx, float* __restrict__ out_val,
-                                                uint4* __restrict__ zero_ptr, uint32_t zero_vecs) {
+                                                uint4* __restrict__ zero_ptr, uint32_t zero_vecs,
+                                                double* __restrict__ out_sum) {
   pdl_enter();
   for (uint32_t i = blockIdx.x * TPB + threadIdx.x; i < zero_vecs; i += gridDim.x * TPB)
     zero_ptr[i] = make_uint4(0, 0, 0, 0);
@@ -1338,7 +1339,8 @@ __global__ void __launch_bounds__(TPB) k_gather(float* __restrict__ acc, int N, 
   if (k >= K) return;
   const int64_t j = idx[k];
   if (j < 0 || j >= d) {
-    out_val[k] = 0.f;
+    if (out_sum) out_sum[k] = 0.0;
+    else out_val[k] = 0.f;
     return;
   }
   float* col = acc + j;
@@ -1354,7 +1356,16 @@ __global__ void __launch_bounds__(TPB) k_gather(float* __restrict__ acc, int N, 
       if (n0 + q < N) s += (double)v[q];
   }
   for (int n = 0; n < N; n++) __stcg(col + (size_t)n * (size_t)d, 0.0f);
-  out_val[k] = (float)(s / (double)N);
+  // a rank that holds only some of the workers hands back its binary64 partial sum instead
+  if (out_sum) out_sum[k] = s;
+  else out_val[k] = (float)(s / (double)N);
+}
+
+// worker-sharded step: mean over all workers from the summed partial sums
+__global__ void __launch_bounds__(TPB) k_finish_mean(const double* __restrict__ sum, int64_t K, double n_total,
+                                                     float* __restrict__ out_val) {
+  const int64_t k = (int64_t)blockIdx.x * TPB + threadIdx.x;
+  if (k < K) out_val[k] = (float)(sum[k] / n_total);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1934,9 +1945,9 @@ int select_impl(mv_ctx* ctx, P p, const Layout& L, const uint8_t* votes, bool ha
 
 // steps a5-a6
 int aggregate_impl(mv_ctx* ctx, float* acc, int N, int64_t d, int64_t K, const int32_t* idx, float* out_val,
-                   size_t clear_bytes) {
+                   size_t clear_bytes, double* out_sum = nullptr) {
   launch_k(k_gather, dim3((unsigned)((K + TPB - 1) / TPB)), dim3(TPB), ctx->stream, acc, N, d, K, idx, out_val,
-           (uint4*)ctx->ws, (uint32_t)(clear_bytes / 16));
+           (uint4*)ctx->ws, (uint32_t)(clear_bytes / 16), out_sum);
   MV_LAUNCH_CHECK();
   if (clear_bytes) ctx->clean_bytes = clear_bytes;
   return MV_OK;
@@ -2124,6 +2135,25 @@ int mv_aggregate(mv_ctx* ctx, float* acc, int N, int64_t d, int64_t K, const int
   ctx->launches = 0;
   if (ctx->phase_timing) cudaEventRecord(ctx->pev[0], ctx->stream);
   return aggregate_impl(ctx, acc, N, d, K, idx, out_val, 0);
+}
+
+int mv_aggregate_partial(mv_ctx* ctx, float* acc, int N_local, int64_t d, int64_t K, const int32_t* idx,
+                         double* out_sum) {
+  Layout L;
+  const int rc = check_common(ctx, N_local, d, K, L);
+  if (rc != MV_OK) return rc;
+  if (acc == nullptr || idx == nullptr || out_sum == nullptr || !aligned16(acc) || !aligned16(idx) || !aligned16(out_sum))
+    return MV_ERR_INVALID_ARG;
+  ctx->launches = 0;
+  if (ctx->phase_timing) cudaEventRecord(ctx->pev[0], ctx->stream);
+  return aggregate_impl(ctx, acc, N_local, d, K, idx, nullptr, 0, out_sum);
+}
+
+int mv_finish_mean(void* stream, const double* sum, int64_t K, int N_total, float* out_val) {
+  if (sum == nullptr || out_val == nullptr || K < 1 || N_total < 1 || !aligned16(sum) || !aligned16(out_val))
+    return MV_ERR_INVALID_ARG;
+  k_finish_mean<<<(unsigned)((K + TPB - 1) / TPB), TPB, 0, (cudaStream_t)stream>>>(sum, K, (double)N_total, out_val);
+  return cudaGetLastError() == cudaSuccess ? MV_OK : MV_ERR_CUDA;
 }
 
 int mv_sparse_step(mv_ctx* ctx, const float* grads, float* err, int N, int64_t d, int64_t K, int32_t* out_idx,

@@ -51,3 +51,76 @@ def test_reference_arm_runs_on_rank_zero_only():
     assert line["impl"] == "reference" and line["unit"] == "steps/s" and line["value"] > 0
     assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
     assert line["n_gpus"] == 2 and line["config"]["N"] == 4
+
+
+# ---------------------------------------------------------------------------------------------
+# worker-sharded step: the orchestration (which calls, which collectives, which N) under gloo,
+# world size 2, with a CPU stand-in for the CUDA context that computes each call from the oracle
+# ---------------------------------------------------------------------------------------------
+class _OracleContext:
+    """The four calls ShardedStep makes, computed on CPU tensors by the oracle (a test double: the
+    product's context runs the same calls on the GPU)."""
+
+    def mv_vote(self, grads, err, votes=None, K=None, **_):
+        from oracle import mv_oracle as O
+        v = O.mv_vote(grads.numpy(), err.numpy(), K)
+        err.copy_(torch.from_numpy(v["acc"]))
+        votes.copy_(torch.from_numpy(v["votes"]))
+
+    def mv_select(self, votes, N, out_idx, K=None, **_):
+        from oracle import mv_oracle as O
+        assert int(votes.max()) <= N
+        out_idx.copy_(torch.from_numpy(O.select_mask(votes.numpy(), K)[0]))
+
+    def mv_aggregate_partial(self, acc, idx, out_sum):
+        cols = idx.long()
+        total = torch.zeros(idx.numel(), dtype=torch.float64)
+        for n in range(acc.shape[0]):
+            total += acc[n, cols].double()
+        out_sum.copy_(total)
+        acc[:, cols] = 0.0
+
+    def mv_finish_mean(self, total, N_total, out_val):
+        out_val.copy_((total / float(N_total)).float())
+
+
+def _sharded_rank(rank, world, port, out_dir):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    sys.path.insert(0, ROOT)
+    import numpy as np
+    from paper_2011_06495_b200.sharded import ShardedStep
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    N, d, K, steps = 6, 5003, 60, 3
+    rows = slice(rank * N // world, (rank + 1) * N // world)
+    g = torch.Generator().manual_seed(77)
+    err = torch.zeros(N, d)[rows].clone()
+    step = ShardedStep(_OracleContext(), N, d, K, "cpu")
+    out_idx = torch.empty(K, dtype=torch.int32)
+    out_val = torch.empty(K, dtype=torch.float32)
+    outs = []
+    for _ in range(steps):
+        grads = torch.randn(N, d, generator=g)          # the same stream on both ranks; each takes its rows
+        step.step(grads[rows].clone(), err, out_idx, out_val)
+        outs.append((out_idx.clone(), out_val.clone()))
+    torch.save({"outs": outs, "err": err}, os.path.join(out_dir, f"sharded{rank}.pt"))
+    dist.destroy_process_group()
+
+
+def test_worker_sharded_step_equals_the_unsharded_step(tmp_path):
+    import numpy as np
+    from oracle import mv_oracle as O
+    world = 2
+    mp.spawn(_sharded_rank, args=(world, 29633, str(tmp_path)), nprocs=world, join=True)
+    res = [torch.load(tmp_path / f"sharded{r}.pt") for r in range(world)]
+    N, d, K, steps = 6, 5003, 60, 3
+    g = torch.Generator().manual_seed(77)
+    err = np.zeros((N, d), dtype=np.float32)
+    for s in range(steps):
+        ref = O.mv_sparse_step(torch.randn(N, d, generator=g).numpy(), err, K)
+        err = ref["err"]
+        for r in range(world):
+            idx, val = res[r]["outs"][s]
+            assert np.array_equal(idx.numpy(), ref["out_idx"])                       # every rank holds the same mask
+            np.testing.assert_allclose(val.numpy(), ref["out_val"], rtol=1e-6, atol=1e-12)
+    got_err = np.concatenate([res[r]["err"].numpy() for r in range(world)], axis=0)
+    assert np.array_equal(got_err.view(np.uint32), err.view(np.uint32))              # residuals, rank by rank
