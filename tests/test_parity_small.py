@@ -82,6 +82,72 @@ def test_max_workers():
     PT.compare_all(ctx, grads.to(DEV), err.to(DEV), K, label="[N=255] ")
 
 
+def test_longest_row():
+    """d at the documented limit (2^31 - 8193) with two workers, so that coordinates, flat offsets
+    n*d + j and chunk numbers reach their largest values.  The expected result follows from the
+    definition alone: a background of small values, a few hundred planted distinct large magnitudes
+    (always selected) and a few thousand planted equal magnitudes of which only the lowest indices
+    fit - placed at the very start, the very end and around 2^30 and 2^31 - 2^13 as well."""
+    N, K = 2, 2000
+    d = (1 << 31) - 8193
+    rng = np.random.default_rng(31)
+    ctx = B.MvContext(N, d, K, device=DEV)
+    grads = torch.empty((N, d), dtype=torch.float32, device=DEV)
+    err = torch.empty((N, d), dtype=torch.float32, device=DEV)
+    g = torch.Generator(device=DEV).manual_seed(31)
+    for n in range(N):
+        grads[n].normal_(0.0, 0.01, generator=g)
+        err[n].normal_(0.0, 0.001, generator=g)
+    special = np.array([0, 1, 31, 4095, 4096, (1 << 30) - 1, 1 << 30, (1 << 31) - 16384, d - 4097, d - 4096, d - 33, d - 2, d - 1])
+    planted = []
+    for n in range(N):
+        pos = np.unique(np.concatenate([special, rng.integers(0, d, size=3200)]))
+        rng.shuffle(pos)
+        big, tied = np.sort(pos[:500]), np.sort(pos[500:3000])
+        if n == 1:                                                  # half of worker 1's distinct picks coincide with worker 0's
+            big = np.unique(np.concatenate([planted[0][0][::2], big[:250]]))
+            tied = np.setdiff1d(tied, big)
+        planted.append((big, tied))
+        tpos = torch.from_numpy(np.concatenate([big, tied])).to(DEV)
+        vals = torch.cat([torch.arange(big.size, device=DEV, dtype=torch.float32) * (1 if n == 0 else -1) + (200.0 if n == 0 else -200.0),
+                          torch.full((tied.size,), -100.0 if n == 0 else 100.0, device=DEV)])
+        grads[n, tpos] = vals
+        err[n, tpos] = 0.0
+    # the definition, on the planted positions only: each worker keeps its distinct values and the lowest-index ties
+    worker_sets = [np.sort(np.concatenate([b, t[:K - b.size]])) for b, t in planted]
+    pos, votes = np.unique(np.concatenate(worker_sets), return_counts=True)
+    order = np.lexsort((pos, -votes))                               # votes descending, index ascending
+    want_idx = np.sort(pos[order[:K]]).astype(np.int64)
+    out_idx = torch.empty(K, dtype=torch.int32, device=DEV)
+    out_val = torch.empty(K, dtype=torch.float32, device=DEV)
+    widx = torch.empty((N, K), dtype=torch.int32, device=DEV)
+    acc_at = (grads[:, torch.from_numpy(want_idx).to(DEV)] + err[:, torch.from_numpy(want_idx).to(DEV)]).double().cpu().numpy()
+    probe = torch.from_numpy(np.concatenate([special, rng.integers(0, d, size=100_000)])).to(DEV)
+    acc_probe = grads[:, probe] + err[:, probe]
+    e = err.clone()
+    ctx.mv_vote(grads, e, worker_idx=widx)                          # sampled threshold
+    torch.cuda.synchronize()
+    for n in range(N):
+        PT.first_diff(PT.npy(widx[n]).astype(np.int64), worker_sets[n].astype(np.int64), f"worker {n} top-K")
+    ctx.set_mode(B.MV_MODE_TRACK)
+    launches = []
+    for call in range(2):                                           # the second call runs with a carried threshold
+        e.copy_(err)
+        ctx.mv_sparse_step(grads, e, out_idx, out_val)
+        torch.cuda.synchronize()
+        launches.append(ctx.last_launches())
+        # K/d is 1e-6 here: a sample of 2^20 elements cannot bracket the K-th key (both workers take the
+        # full-row select on the first call); the carried threshold of the second call can
+        assert ctx.read_diag(N)[:, 2].tolist() == ([1, 1] if call == 0 else [0, 0])
+        PT.first_diff(PT.npy(out_idx).astype(np.int64), want_idx, f"call {call} out_idx")
+        np.testing.assert_allclose(PT.npy(out_val).astype(np.float64), acc_at.sum(axis=0) / N, rtol=1e-6, atol=0)
+        got = e[:, probe]
+        in_mask = torch.from_numpy(np.isin(PT.npy(probe), want_idx)).to(DEV)
+        assert bool((got[:, in_mask] == 0).all()) and torch.equal(got[:, ~in_mask], acc_probe[:, ~in_mask])
+        assert int((e[:, torch.from_numpy(want_idx).to(DEV)] != 0).sum()) == 0
+    assert launches[1] == launches[0] - 1
+
+
 @pytest.mark.parametrize("name", ["c1", "c1_ties"])
 @pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
 def test_config_c1(name, mode):
