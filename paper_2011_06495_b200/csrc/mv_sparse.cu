@@ -18,6 +18,13 @@
 //                                             votes come from the caller)
 //   aggregate  k_gather                       mean on the shared mask, residual zeroed in place
 //
+// With threshold tracking the sample is skipped after the first call: while a call resolves its
+// K-th key, the same histogram sweeps locate a slightly larger rank, and that key prefix is the
+// next call's tau_n.  Variants reuse the select kernels in "list mode" over explicit (key, index)
+// lists: add-drop voting (k_ad_fill, k_ad_apply; Algorithm 2) and random selection proportional to
+// the votes (k_rs_fill, k_chunk_popc; Algorithm 1, second variant).  A rank that holds only some
+// of the workers gets binary64 partial sums from k_gather and finishes with k_finish_mean.
+//
 // The magnitude order is the order of key(x) = bits(x) & 0x7fffffff; ties go to the lowest index.
 #include <cuda_runtime.h>
 #include <stdint.h>
