@@ -91,6 +91,12 @@ def test_add_drop_without_sampling():
     run_steps(3, 50021, 500, 50, steps=3, kind="gauss", seed=9, mode=B.MV_MODE_GENERAL)
 
 
+@pytest.mark.parametrize("N,d,K,K_ad", [(4, 300007, 3000, 300), (6, 100003, 500, 50)])
+def test_add_drop_with_a_tracked_threshold(N, d, K, K_ad):
+    """The bench's configuration: candidate threshold carried from step to step."""
+    run_steps(N, d, K, K_ad, steps=6, kind="gauss", seed=13, mode=B.MV_MODE_TRACK, want_lists=False)
+
+
 def test_large_K_ad_equals_plain_majority_voting():
     """K_ad = K: the step gives the same bytes as mv_sparse_step."""
     N, d, K = 5, 70001, 700
@@ -116,7 +122,7 @@ def test_add_drop_at_resnet_size():
     w = WL.resnet_like("c2")
     K_ad = w.K // 10
     std = WL.std_vector(w, DEV)
-    ctx = B.MvContext(w.N, w.d, w.K, device=DEV)
+    ctx = B.MvContext(w.N, w.d, w.K, device=DEV, mode=B.MV_MODE_TRACK)
     W = (w.d + 31) // 32
     err = WL.initial_err(w, device=DEV)
     err_ref = err.cpu().numpy()
