@@ -1482,7 +1482,7 @@ __device__ __forceinline__ uint32_t philox4x32_10_first(uint32_t c0, uint32_t c1
 __device__ __forceinline__ double neg_log_u(uint32_t x) {
   const unsigned long long v = 2ull * x + 1ull;  // u = v / 2^33
   int e = 63 - __clzll((long long)v);
-  double m = __ddiv_rn((double)v, (double)(1ull << e));  // [1, 2), exact
+  double m = __dmul_rn((double)v, __longlong_as_double((long long)(1023 - e) << 52));  // v * 2^-e: [1, 2), exact
   if (m > 1.4142135623730951) {
     m = __dmul_rn(m, 0.5);
     e += 1;
@@ -1497,13 +1497,18 @@ __device__ __forceinline__ double neg_log_u(uint32_t x) {
 }
 
 // A CTA per chunk: thread t owns coordinates 16t .. 16t+15 of the chunk, so thread order is index
-// order.  Voted coordinates are appended to the single list `a` (row 0) as (0x7fffffff - ring time
-// bits, index): the list-mode select then keeps the K largest keys, i.e. the K earliest times.
+// order.  Voted coordinates are first compacted, in index order, into shared memory; the threads
+// then share them out evenly (the generator and the logarithm are the expensive part, and only about
+// one coordinate in ten holds a vote) and append them to the single list `a` (row 0) as
+// (0x7fffffff - ring time bits, index): the list-mode select then keeps the K largest keys, i.e. the
+// K earliest times.
 __global__ void __launch_bounds__(TPB) k_rs_fill(P p, P a, const uint8_t* __restrict__ votes, uint32_t seed_lo,
                                                  uint32_t seed_hi, uint32_t draw_lo, uint32_t draw_hi) {
   pdl_enter();
   __shared__ uint32_t s_w[TPB / 32 + 1];
   __shared__ uint32_t s_base;
+  __shared__ uint16_t s_off[CH];  // offset of the coordinate within the chunk
+  __shared__ uint8_t s_v[CH];     // its votes
   const int c = blockIdx.x;
   const int64_t j0 = (int64_t)c * CH + threadIdx.x * 16;
   uint8_t v[16];
@@ -1527,18 +1532,22 @@ __global__ void __launch_bounds__(TPB) k_rs_fill(P p, P a, const uint8_t* __rest
     a.chunk_base[c] = base;
     a.chunk_cnt[c] = total;
   }
-  __syncthreads();
-  if (cnt == 0) return;
-  pos += s_base;
+  if (total == 0) return;  // uniform over the CTA
 #pragma unroll
   for (int i = 0; i < 16; i++) {
     if (v[i] == 0) continue;
-    const uint32_t j = (uint32_t)(j0 + i);
-    const uint32_t x = philox4x32_10_first(j, 0u, draw_lo, draw_hi, seed_lo, seed_hi);
-    const double t = __ddiv_rn(neg_log_u(x), (double)v[i]);
-    const uint32_t tb = __float_as_uint(__double2float_rn(t));
-    if (pos < a.cap) a.cand[pos] = make_uint2(0x7fffffffu - tb, j);
+    s_off[pos] = (uint16_t)(threadIdx.x * 16 + i);
+    s_v[pos] = v[i];
     pos++;
+  }
+  __syncthreads();
+  const uint32_t base = s_base;
+  for (uint32_t i = threadIdx.x; i < total; i += TPB) {
+    const uint32_t j = (uint32_t)((int64_t)c * CH + s_off[i]);
+    const uint32_t x = philox4x32_10_first(j, 0u, draw_lo, draw_hi, seed_lo, seed_hi);
+    const double t = __ddiv_rn(neg_log_u(x), (double)s_v[i]);
+    const uint32_t tb = __float_as_uint(__double2float_rn(t));
+    if (base + i < a.cap) a.cand[base + i] = make_uint2(0x7fffffffu - tb, j);
   }
 }
 
