@@ -1387,8 +1387,10 @@ __global__ void __launch_bounds__(TPB) k_ad_fill(P p, P a, const uint32_t* __res
                                                  const float* __restrict__ acc) {
   pdl_enter();
   // a warp per (worker, chunk): lane l owns mask words 4l..4l+3 of the chunk, so lane order is index order
-  const int n = blockIdx.y, lane = threadIdx.x & 31;
-  const int c = blockIdx.x * (TPB / 32) + (threadIdx.x >> 5);
+  __shared__ uint32_t s_A[TPB / 32][WPC];    // the chunk's "add" candidates as mask words ...
+  __shared__ uint16_t s_rank[TPB / 32][WPC];  // ... and how many of them lie in earlier words
+  const int n = blockIdx.y, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int c = blockIdx.x * (TPB / 32) + warp;
   if (c >= p.nchunks) return;
   uint32_t A[4], D[4];
   uint32_t pa = 0, pd = 0;
@@ -1432,10 +1434,37 @@ __global__ void __launch_bounds__(TPB) k_ad_fill(P p, P a, const uint32_t* __res
   uint2* la = a.cand + (size_t)n * a.cap;
   uint2* ld = a.cand + (size_t)(p.N + n) * a.cap;
   uint32_t posa = ba + xa - pa, posd = bd + xd - pd;
+  // The keys of the "add" candidates: M_n is a subset of the worker's candidate buffer when the
+  // worker went through it, so the chunk's run there already holds (key, index) for every one of
+  // them, in index order: no need to gather acc.  A full-row worker gathers, like the drop list.
+  const bool from_run = tota != 0 && worker_fast(p, n);  // warp-uniform
+  if (from_run) {
+    uint32_t r = xa - pa;
+#pragma unroll
+    for (int q = 0; q < 4; q++) {
+      s_A[warp][lane * 4 + q] = A[q];
+      s_rank[warp][lane * 4 + q] = (uint16_t)r;
+      r += __popc(A[q]);
+    }
+    __syncwarp();
+    const size_t ci = (size_t)n * p.nchunks + c;
+    const uint32_t rcnt = p.chunk_cnt[ci];
+    const uint2* run = p.cand + (size_t)n * p.cap + p.chunk_base[ci];
+    for (uint32_t i = lane; i < rcnt; i += 32) {
+      const uint2 kv = __ldcg(run + i);
+      const uint32_t o = kv.y - (uint32_t)c * CH;  // offset within the chunk
+      if (o >= (uint32_t)CH) continue;             // cannot happen for a well-formed run
+      const uint32_t w = s_A[warp][o >> 5], bit = o & 31u;
+      if ((w >> bit) & 1u) {
+        const uint32_t pos = ba + s_rank[warp][o >> 5] + __popc(w & ((1u << bit) - 1u));
+        if (pos < a.cap) la[pos] = kv;
+      }
+    }
+  }
 #pragma unroll
   for (int q = 0; q < 4; q++) {
     const int64_t j0 = ((int64_t)c * WPC + lane * 4 + q) * 32;
-    uint32_t m = A[q];
+    uint32_t m = from_run ? 0u : A[q];
     while (m) {
       const int b = __ffs(m) - 1;
       m &= m - 1;
