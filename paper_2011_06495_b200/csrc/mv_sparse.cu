@@ -7,26 +7,31 @@
 //                                             lower bound tau_n on the K-th largest magnitude key
 //   stream     k_acc_compact                  the one pass over N x d: acc = err + grads written in
 //                                             place, elements with key >= tau_n compacted per chunk
-//   select     k_hist<1..3>, k_count          exact K-th key T_n by radix select: on the candidates, or over
-//                                             the full row for a worker whose candidate count missed [K, cap]
-//   order      (tail of k_count)              lowest-index tie quota per chunk, for workers whose threshold
-//                                             ties are only partly kept
-//   vote       k_set_bits, k_votes            per-worker bit masks (from the candidates, or from the row for a
-//                                             full-row worker), bit-sliced vote count
-//   lists      k_scan_sel, k_lists            ascending per-worker index lists from the masks (side stream)
-//   mask       (tail of k_votes), k_vote_write  counting select over vote values 0..N (k_vote_hist when
-//                                             votes come from the caller)
+//   select     k_select_cluster               a thread-block cluster per worker: exact K-th key T_n of the
+//                                             candidates (histograms in shared memory, merged through
+//                                             distributed shared memory), or of the full row for a worker
+//                                             whose candidate count missed [K, cap]; tie order per chunk
+//                                             for workers whose threshold ties are only partly kept; all
+//                                             CTAs first clear the bit masks and the vote bytes
+//   pick       k_set_bits                     every pick sets its bit in the worker's mask and adds one
+//                                             to its coordinate's vote byte (L2 atomics)
+//   mask       k_vote_hist, k_vote_write      counting select over vote values 0..N: per-chunk vote
+//                                             histograms, v*, output offsets; then supp(M) ascending
+//   lists      k_chunk_popc, k_scan_sel, k_lists   ascending per-worker index lists from the masks (side stream)
 //   aggregate  k_gather                       mean on the shared mask, residual zeroed in place
 //
 // With threshold tracking the sample is skipped after the first call: while a call resolves its
-// K-th key, the same histogram sweeps locate a slightly larger rank, and that key prefix is the
-// next call's tau_n.  Variants reuse the select kernels in "list mode" over explicit (key, index)
-// lists: add-drop voting (k_ad_fill, k_ad_apply; Algorithm 2) and random selection proportional to
-// the votes (k_rs_fill, k_chunk_popc; Algorithm 1, second variant).  A rank that holds only some
-// of the workers gets binary64 partial sums from k_gather and finishes with k_finish_mean.
+// K-th key, the same counts locate a slightly larger rank, and that key is the next call's tau_n.
+// MV_MODE_GENERAL (no sampling) fuses a full radix histogram into the first pass instead and uses the
+// grid-wide select kernels k_hist<1..3>, k_count, k_set_bits and the bit-sliced vote count k_votes;
+// the same select kernels serve the variants in "list mode" over explicit (key, index) lists:
+// add-drop voting (k_ad_fill, k_ad_apply; Algorithm 2) and random selection proportional to the
+// votes (k_rs_fill; Algorithm 1, second variant).  A rank that holds only some of the workers gets
+// binary64 partial sums from k_gather and finishes with k_finish_mean.
 //
 // The magnitude order is the order of key(x) = bits(x) & 0x7fffffff; ties go to the lowest index.
 #include <cuda_runtime.h>
+#include <cooperative_groups.h>
 #include <stdint.h>
 #include <stdlib.h>
 #include <math.h>
@@ -44,6 +49,8 @@ constexpr int SB_SHIFT = 18;
 constexpr int H1_BINS = 2048;        // radix digits of the 31-bit key: 11 + 10 + 10 bits
 constexpr int H2_BINS = 1024;
 constexpr int H3_BINS = 1024;
+constexpr int WIN_SHIFT = 11;        // the select first counts the candidates in [tau, tau + 2^(11+11)) in H1_BINS bins of 2^11 keys
+constexpr int WIN_LIST = 1024;       // most keys of one such bin that the select ranks directly
 constexpr unsigned FULL = 0xffffffffu;
 
 struct P {
@@ -54,6 +61,7 @@ struct P {
   int force_general;
   int list_mode;          // 1: the rows are plain (key, index) lists to select min(K, length) from (add-drop)
   int apply_rows;         // list mode: rows < apply_rows are "add" lists, the others "drop" lists
+  uint32_t* vote_words;   // cluster select: if set, every pick also adds one to its vote byte (four bytes per word)
   uint32_t* apply_bits;   // list mode, optional: the vote masks [apply_rows][W] to update in place instead of
                           // writing the picks to worker_bits
   int64_t d;
@@ -67,7 +75,7 @@ struct P {
   uint32_t* sample_done;  // [N] ticket counters (last CTA of a worker finishes the job)
   uint32_t* count_done;   // [N]
   uint32_t* votes_done;   // [1]
-  uint8_t* hot;           // [nc_pad] 1 if any worker kept a candidate in the chunk
+  uint8_t* hot;           // [nc_pad] general mode: 1 if any worker picked a coordinate of the chunk
   uint32_t* vote_hist;    // [256]
   uint32_t* tau;          // [N] candidate threshold of this call
   uint32_t* tau_next;     // [N] threshold proposed for the next call (threshold tracking), or null
@@ -102,6 +110,21 @@ __device__ __forceinline__ void pdl_enter() {
 }
 
 __device__ __forceinline__ uint32_t fkey(float x) { return __float_as_uint(x) & 0x7fffffffu; }
+
+// one more vote for coordinate j: the vote bytes are packed four to a word and start out zero
+__device__ __forceinline__ void add_vote(uint32_t* __restrict__ vote_words, uint32_t j) {
+  atomicAdd(vote_words + (j >> 2), 1u << (8u * (j & 3u)));
+}
+
+// this CTA's share of clearing `nwords` 32-bit words at a 16-byte aligned address
+__device__ __forceinline__ void zero_share(uint32_t* __restrict__ ptr, size_t nwords, size_t bid, size_t nblocks) {
+  const size_t nvec = nwords >> 2;
+  const size_t per = (nvec + nblocks - 1) / nblocks;
+  const size_t v0 = bid * per, v1 = v0 + per < nvec ? v0 + per : nvec;
+  uint4* q = reinterpret_cast<uint4*>(ptr);
+  for (size_t i = v0 + threadIdx.x; i < v1; i += blockDim.x) q[i] = make_uint4(0, 0, 0, 0);
+  if (bid == 0 && threadIdx.x < (nwords & 3)) ptr[(nvec << 2) + threadIdx.x] = 0u;
+}
 
 __device__ __forceinline__ uint32_t lanemask_lt() {
   uint32_t m;
@@ -151,10 +174,11 @@ __device__ __forceinline__ Geom chunk_geom(int n, int c, int64_t d) {
 
 // Thread (warp w, lane l) owns slots w*128 + i*32 + l, i = 0..3: a warp covers 512 consecutive
 // coordinates, in index order (i, l, element).  ACC: acc = err + grads is computed and stored to err.
+// t = the thread's position among the 256 that share the chunk.
 template <bool ACC>
 __device__ __forceinline__ void load_keys(const Geom& g, const float* __restrict__ grads, float* __restrict__ err,
-                                          uint32_t (&key)[4][4], uint32_t (&vm)[4]) {
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+                                          uint32_t (&key)[4][4], uint32_t (&vm)[4], int t = threadIdx.x) {
+  const int warp = t >> 5, lane = t & 31;
   float4 ev[4], gv[4];
   int kind[4];
 #pragma unroll
@@ -495,10 +519,6 @@ __global__ void __launch_bounds__(TPB, 4) k_acc_compact(P p, const float* __rest
   const uint32_t tau = p.tau[n];
   uint32_t key[4][4], vm[4], cm[4];
   load_keys<true>(g, grads, err, key, vm);
-  if (threadIdx.x < WPC) {  // the worker's mask starts out empty
-    const int64_t wi = (int64_t)c * WPC + threadIdx.x;
-    if (wi < p.W) p.worker_bits[(size_t)n * p.W + wi] = 0u;
-  }
   uint32_t xkey[4] = {0, 0, 0, 0}, xcm = 0;
   if (threadIdx.x == TPB - 1) {
     uint32_t xvm;
@@ -522,10 +542,7 @@ __global__ void __launch_bounds__(TPB, 4) k_acc_compact(P p, const float* __rest
   // issued now and consumed after the staging, so that its round trip overlaps with it
   uint32_t base_r = 0;
   if (threadIdx.x == 0) {
-    if (total) {
-      base_r = atomicAdd(&p.cand_cnt[n], total);
-      p.hot[c] = 1;  // same value from every worker: a plain store is enough
-    }
+    if (total) base_r = atomicAdd(&p.cand_cnt[n], total);
     p.chunk_cnt[(size_t)n * p.nchunks + c] = total;
     if (total == 0) p.chunk_base[(size_t)n * p.nchunks + c] = 0;
   }
@@ -847,48 +864,69 @@ __device__ void vote_scan(const P& p) {
   }
   __syncthreads();
   const uint32_t vstar = s_v[0], quota = s_v[3];
-  // each thread owns `per` consecutive chunks (a multiple of 8, so its counts are whole 16-byte loads)
-  const int per = (((p.nchunks + NT - 1) / NT) + 7) & ~7;
-  const int c0 = min(p.nc_pad, (int)threadIdx.x * per), c1 = min(p.nc_pad, c0 + per);
+  // Tiles of NT*8 chunks, a thread taking 8 neighbouring chunks of a tile (one 16-byte load per
+  // count array); the loads of TB tiles are issued together, then every tile costs two block scans.
+  // ecarry / scarry: v*-ties seen and outputs placed in the tiles before.
   const uint16_t* hge = p.chunk_vh + (size_t)vstar * p.nc_pad;                                   // votes >= v*
   const uint16_t* hgt = (int)vstar < p.N ? p.chunk_vh + (size_t)(vstar + 1) * p.nc_pad : nullptr;  // votes > v*
-  uint32_t esum = 0, gsum = 0;
-  for (int c = c0; c < c1; c += 8) {
-    const uint4 a = __ldcg(reinterpret_cast<const uint4*>(hge + c));
-    const uint4 g = hgt ? __ldcg(reinterpret_cast<const uint4*>(hgt + c)) : make_uint4(0, 0, 0, 0);
-    const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, gw[4] = {g.x, g.y, g.z, g.w};
+  constexpr int TB = 4;
+  uint32_t ecarry = 0, scarry = 0;
+  for (int c00 = 0; c00 < p.nc_pad; c00 += NT * 8 * TB) {  // uniform over the CTA
+    uint4 av[TB], gv[TB];
 #pragma unroll
-    for (int q = 0; q < 8; q++) {
-      if (c + q < p.nchunks) {
-        const uint32_t ge = (aw[q >> 1] >> (16 * (q & 1))) & 0xffffu, gt = (gw[q >> 1] >> (16 * (q & 1))) & 0xffffu;
-        esum += ge - gt;
-        gsum += gt;
+    for (int k = 0; k < TB; k++) {
+      const int c = c00 + (k * NT + (int)threadIdx.x) * 8;
+      av[k] = make_uint4(0, 0, 0, 0);
+      gv[k] = make_uint4(0, 0, 0, 0);
+      if (c < p.nc_pad) {
+        av[k] = __ldcg(reinterpret_cast<const uint4*>(hge + c));
+        if (hgt) gv[k] = __ldcg(reinterpret_cast<const uint4*>(hgt + c));
       }
     }
-  }
-  uint32_t tot;
-  const uint32_t epre = block_excl_scan<NT>(esum, s_w, tot);
-  const uint32_t taken_before = epre < quota ? epre : quota;              // ties kept in earlier chunks
-  const uint32_t taken_here = min(epre + esum, quota) - taken_before;     // ties kept in this thread's chunks
-  const uint32_t spre = block_excl_scan<NT>(gsum + taken_here, s_w, tot);
-  uint32_t run = epre, srun = spre;
-  for (int c = c0; c < c1; c += 8) {
-    const uint4 a = __ldcg(reinterpret_cast<const uint4*>(hge + c));
-    const uint4 g = hgt ? __ldcg(reinterpret_cast<const uint4*>(hgt + c)) : make_uint4(0, 0, 0, 0);
-    const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, gw[4] = {g.x, g.y, g.z, g.w};
 #pragma unroll
-    for (int q = 0; q < 8; q++) {
-      if (c + q < p.nchunks) {
+    for (int k = 0; k < TB; k++) {
+      if (c00 + k * NT * 8 >= p.nc_pad) break;  // uniform over the CTA
+      const int c = c00 + (k * NT + (int)threadIdx.x) * 8;
+      const uint32_t aw[4] = {av[k].x, av[k].y, av[k].z, av[k].w}, gw[4] = {gv[k].x, gv[k].y, gv[k].z, gv[k].w};
+      uint32_t eqv[8], gtv[8], esum = 0, gsum = 0;
+#pragma unroll
+      for (int q = 0; q < 8; q++) {
         const uint32_t ge = (aw[q >> 1] >> (16 * (q & 1))) & 0xffffu, gt = (gw[q >> 1] >> (16 * (q & 1))) & 0xffffu;
-        const uint32_t eq = ge - gt;
-        const uint32_t take = run >= quota ? 0u : min(eq, quota - run);
-        p.tie_take[c + q] = take;
-        p.out_base[c + q] = srun;
-        run += eq;
-        srun += gt + take;
+        const bool in = c + q < p.nchunks;
+        eqv[q] = in ? ge - gt : 0u;
+        gtv[q] = in ? gt : 0u;
+        esum += eqv[q];
+        gsum += gtv[q];
       }
+      uint32_t etot, stot;
+      const uint32_t epre = ecarry + block_excl_scan<NT>(esum, s_w, etot);
+      const uint32_t taken_before = epre < quota ? epre : quota;           // ties kept in earlier chunks
+      const uint32_t taken_here = min(epre + esum, quota) - taken_before;  // ties kept in this thread's chunks
+      const uint32_t spre = scarry + block_excl_scan<NT>(gsum + taken_here, s_w, stot);
+      // eight neighbouring chunks per thread: their results go out as 16-byte stores (the arrays are
+      // padded to whole groups of eight; the slot after the last chunk holds K, the end of the output)
+      uint32_t run = epre, srun = spre, tk[8], ob[8];
+#pragma unroll
+      for (int q = 0; q < 8; q++) {
+        const uint32_t take = run >= quota ? 0u : min(eqv[q], quota - run);
+        tk[q] = take;
+        ob[q] = c + q == p.nchunks ? (uint32_t)p.K : srun;
+        run += eqv[q];
+        srun += gtv[q] + take;
+      }
+      if (c < p.nc_pad) {
+        uint4* tt = reinterpret_cast<uint4*>(p.tie_take + c);
+        uint4* oo = reinterpret_cast<uint4*>(p.out_base + c);
+        tt[0] = make_uint4(tk[0], tk[1], tk[2], tk[3]);
+        tt[1] = make_uint4(tk[4], tk[5], tk[6], tk[7]);
+        oo[0] = make_uint4(ob[0], ob[1], ob[2], ob[3]);
+        oo[1] = make_uint4(ob[4], ob[5], ob[6], ob[7]);
+      }
+      ecarry += etot;
+      scarry += stot;
     }
   }
+  __syncthreads();
   if (threadIdx.x == 0) p.out_base[p.nchunks] = (uint32_t)p.K;  // sentinel: end of the last chunk
 }
 
@@ -1013,7 +1051,10 @@ __global__ void __launch_bounds__(TPB) k_set_bits(P p, float* __restrict__ err) 
           const int jf = g.j0 - g.h + 4 * (warp * 128 + i * 32 + lane);
 #pragma unroll
           for (int e = 0; e < 4; e++)
-            if (sm[i] & (1u << e)) atomicOr(bits_row + ((uint32_t)(jf + e) >> 5), 1u << ((uint32_t)(jf + e) & 31u));
+            if (sm[i] & (1u << e)) {
+            atomicOr(bits_row + ((uint32_t)(jf + e) >> 5), 1u << ((uint32_t)(jf + e) & 31u));
+            if (p.vote_words) add_vote(p.vote_words, (uint32_t)(jf + e));
+          }
         }
       }
       if (xsm) {
@@ -1021,7 +1062,10 @@ __global__ void __launch_bounds__(TPB) k_set_bits(P p, float* __restrict__ err) 
         const int jf = g.j0 - g.h + 4096;
 #pragma unroll
         for (int e = 0; e < 4; e++)
-          if (xsm & (1u << e)) atomicOr(bits_row + ((uint32_t)(jf + e) >> 5), 1u << ((uint32_t)(jf + e) & 31u));
+          if (xsm & (1u << e)) {
+            atomicOr(bits_row + ((uint32_t)(jf + e) >> 5), 1u << ((uint32_t)(jf + e) & 31u));
+            if (p.vote_words) add_vote(p.vote_words, (uint32_t)(jf + e));
+          }
       }
       if (any) p.hot[c] = 1;  // same value from every thread
     }
@@ -1047,6 +1091,7 @@ __global__ void __launch_bounds__(TPB) k_set_bits(P p, float* __restrict__ err) 
           acc = 0;
         }
         acc |= 1u << (j & 31u);
+        if (p.vote_words) add_vote(p.vote_words, j);
       }
     }
     if (acc) put_bits(p, n, curw, acc);
@@ -1070,10 +1115,417 @@ __global__ void __launch_bounds__(TPB) k_set_bits(P p, float* __restrict__ err) 
         eq = kv.x == T;
       }
       const uint32_t eb = __ballot_sync(FULL, eq);
-      if (eq && run + __popc(eb & lt) < need && (int64_t)kv.y < p.d) put_bits(p, n, kv.y >> 5, 1u << (kv.y & 31u));
+      if (eq && run + __popc(eb & lt) < need && (int64_t)kv.y < p.d) {
+        put_bits(p, n, kv.y >> 5, 1u << (kv.y & 31u));
+        if (p.vote_words) add_vote(p.vote_words, kv.y);
+      }
       run += __popc(eb);
     }
   }
+}
+
+// ---------------------------------------------------------------------------------------------
+// select + vote bits in one kernel: a thread-block cluster per worker.  The cluster's CTAs split the
+// worker's candidate buffer, keep their keys in shared memory, count each radix digit (11 + 10 + 10
+// bits) into a local shared-memory histogram and, after a cluster barrier, read one another's
+// histograms through distributed shared memory; every CTA thus resolves the digit by itself and no
+// histogram leaves the SMs.  With T_n known the same CTAs set the worker's mask bits.  A worker whose
+// candidate count missed [K, cap] is counted over its full row by the same cluster, and a worker that
+// keeps only part of its threshold ties orders them per chunk as k_count / k_set_bits do.
+// Every condition under which a cluster barrier is reached depends only on values that all CTAs of
+// the cluster compute alike (the candidate count and the merged histograms).
+// ---------------------------------------------------------------------------------------------
+namespace cg = cooperative_groups;
+
+constexpr int CL = 8;           // CTAs of the cluster that serves one worker (portable cluster size)
+constexpr int ST = 1024;        // threads per CTA
+constexpr int SK_KEYS = 32768;  // candidate keys a CTA keeps in shared memory between the digit passes
+
+// block_pick2 over a histogram in shared memory, ST threads; rank 0 = not asked (bin = rem = 0)
+template <int NB>
+__device__ void smem_pick2(const uint32_t* s_hist, uint32_t rank_a, uint32_t rank_b, uint32_t& bin_a, uint32_t& rem_a,
+                           uint32_t& bin_b, uint32_t& rem_b) {
+  constexpr int PER = NB / ST;
+  __shared__ uint32_t s_wsum[ST / 32];
+  __shared__ uint32_t s_res[4];
+  const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+  uint32_t loc[PER];
+  uint32_t sum = 0;
+#pragma unroll
+  for (int k = 0; k < PER; k++) {
+    loc[k] = s_hist[t * PER + k];
+    sum += loc[k];
+  }
+  if (t < 4) s_res[t] = 0;
+  uint32_t x = sum;  // inclusive suffix sum within the warp
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const uint32_t y = __shfl_down_sync(FULL, x, off);
+    if (lane + off < 32) x += y;
+  }
+  if (lane == 0) s_wsum[warp] = x;
+  __syncthreads();
+  uint32_t above0 = x - sum;
+  for (int w = warp + 1; w < ST / 32; w++) above0 += s_wsum[w];
+#pragma unroll
+  for (int which = 0; which < 2; which++) {
+    const uint32_t rank = which ? rank_b : rank_a;
+    uint32_t above = above0;
+    if (above < rank && rank <= above + sum) {
+      bool done = false;
+#pragma unroll
+      for (int k = PER - 1; k >= 0; k--) {
+        if (!done) {
+          if (above + loc[k] >= rank) {
+            s_res[2 * which] = (uint32_t)(t * PER + k);
+            s_res[2 * which + 1] = rank - above;
+            done = true;
+          } else {
+            above += loc[k];
+          }
+        }
+      }
+    }
+  }
+  __syncthreads();
+  bin_a = s_res[0];
+  rem_a = s_res[1];
+  bin_b = s_res[2];
+  rem_b = s_res[3];
+  __syncthreads();
+}
+
+// s_out[b] = sum over the cluster's CTAs of their s_local[b]
+template <int NB>
+__device__ __forceinline__ void cluster_merge(cg::cluster_group& cluster, uint32_t* s_local, uint32_t* s_out) {
+  const uint32_t* peer[CL];
+#pragma unroll
+  for (int r = 0; r < CL; r++) peer[r] = cluster.map_shared_rank(s_local, r);
+  for (int b = threadIdx.x; b < NB; b += ST) {
+    uint32_t v[CL];
+#pragma unroll
+    for (int r = 0; r < CL; r++) v[r] = peer[r][b];
+    uint32_t sum = 0;
+#pragma unroll
+    for (int r = 0; r < CL; r++) sum += v[r];
+    s_out[b] = sum;
+  }
+  __syncthreads();
+}
+
+// f(key) for every element of the chunks of row n that fall to CTA `rank` of the cluster: four
+// chunks at a time, 256 threads each
+template <typename F>
+__device__ __forceinline__ void cluster_row_keys(const P& p, int n, float* __restrict__ err, uint32_t rank, F f) {
+  const int sub = threadIdx.x >> 8, t = threadIdx.x & 255;
+  for (int c = (int)rank * 4 + sub; c < p.nchunks; c += CL * 4) {
+    const Geom g = chunk_geom(n, c, p.d);
+    uint32_t key[4][4], vm[4];
+    load_keys<false>(g, nullptr, err, key, vm, t);
+#pragma unroll
+    for (int i = 0; i < 4; i++)
+#pragma unroll
+      for (int e = 0; e < 4; e++)
+        if (vm[i] & (1u << e)) f(key[i][e]);
+    if (t == TPB - 1) {
+      uint32_t xkey[4], xvm;
+      load_extra<false>(g, nullptr, err, xkey, xvm);
+#pragma unroll
+      for (int e = 0; e < 4; e++)
+        if (xvm & (1u << e)) f(xkey[e]);
+    }
+  }
+}
+
+__global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(ST, 1) k_select_cluster(P p, float* __restrict__ err) {
+  pdl_enter();
+  cg::cluster_group cluster = cg::this_cluster();
+  extern __shared__ uint32_t s_keys[];       // [SK_KEYS]
+  __shared__ uint32_t s_h[3][H1_BINS];       // this CTA's digit counts; pass 2: [0,1024) K-th key's bin, [1024,2048) tracked bin
+  __shared__ uint32_t s_m[H1_BINS];          // the same counts summed over the cluster
+  __shared__ uint32_t s_te[4][9];
+  __shared__ uint32_t s_ws[ST / 32];
+  __shared__ uint32_t s_res3[3];
+  __shared__ uint32_t s_hw[H1_BINS];         // window counts of this CTA's slice
+  {
+    // The workers' bit masks and the vote count start out empty.  They are cleared here, by all CTAs
+    // of the grid together, and not in the streaming pass: what is written now is still in L2 when
+    // the picks arrive as atomics (k_set_bits), whereas lines cleared before the row streamed through
+    // would each have to come back from DRAM.  Clusters beyond the workers' only clear.
+    const size_t nblocks = (size_t)gridDim.x * gridDim.y, bid = (size_t)blockIdx.y * gridDim.x + blockIdx.x;
+    zero_share(p.worker_bits, (size_t)p.N * (size_t)p.W, bid, nblocks);
+    if (p.vote_words != nullptr) zero_share(p.vote_words, (size_t)p.nchunks * (CH / 4), bid, nblocks);
+  }
+  if ((int)blockIdx.y >= p.N) return;  // alike in every CTA of the cluster
+  const int n = blockIdx.y;
+  const uint32_t rank = cluster.block_rank();
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  for (int b = tid; b < 3 * H1_BINS; b += ST) (&s_h[0][0])[b] = 0;
+  __syncthreads();
+  const uint32_t K = (uint32_t)p.K;
+  const uint32_t cnt = p.cand_cnt[n];
+  const bool fast = cnt >= K && cnt <= p.cap;  // alike in every CTA of the cluster
+  const bool tracking = p.tau_next != nullptr;
+  const uint2* cd = p.cand + (size_t)n * p.cap;
+  // this CTA's slice of the candidate buffer
+  const uint32_t per = (cnt + CL - 1) / CL;
+  const uint32_t s0 = min(cnt, rank * per);
+  const uint32_t len = fast ? min(cnt, s0 + per) - s0 : 0u;
+
+  // ---- the usual case: the K-th key lies in a window of 2^22 keys above tau_n ----
+  uint32_t T = 0, need = 0, cnt_eq = 0;
+  bool resolved = false;  // alike in every CTA of the cluster
+  if (fast) {
+    const uint32_t tau = p.tau[n];
+    uint32_t wsum = 0;
+    for (int b = tid; b < H1_BINS; b += ST) s_hw[b] = 0;
+    __syncthreads();
+    for (uint32_t l0 = 0; l0 < len; l0 += ST * 8) {  // uniform over the CTA
+      uint32_t k[8];
+#pragma unroll
+      for (int q = 0; q < 8; q++) {
+        const uint32_t li = l0 + q * ST + tid;
+        k[q] = li < len ? __ldcg(&cd[s0 + li].x) : 0u;
+      }
+#pragma unroll
+      for (int q = 0; q < 8; q++) {
+        const uint32_t li = l0 + q * ST + tid;
+        if (li < len) {
+          if (li < SK_KEYS) s_keys[li] = k[q];
+          const uint32_t wb = (k[q] - tau) >> WIN_SHIFT;
+          if (wb < (uint32_t)H1_BINS) atomicAdd(&s_hw[wb], 1u);
+        }
+      }
+    }
+    cluster.sync();
+    {
+      const uint32_t* peer[CL];
+#pragma unroll
+      for (int r = 0; r < CL; r++) peer[r] = cluster.map_shared_rank(s_hw, r);
+      for (int b = tid; b < H1_BINS; b += ST) {
+        uint32_t v = 0;
+#pragma unroll
+        for (int r = 0; r < CL; r++) v += peer[r][b];
+        s_m[b] = v;
+        wsum += v;
+      }
+    }
+    wsum = __reduce_add_sync(FULL, wsum);
+    if (lane == 0) s_ws[warp] = wsum;
+    __syncthreads();
+    uint32_t win_total = 0;
+    for (int w = 0; w < ST / 32; w++) win_total += s_ws[w];
+    const uint32_t above = cnt - win_total;  // candidates beyond the window
+    if (K > above) {
+      uint32_t bw, rem, bt, trem_w;
+      const uint32_t rt = (tracking && p.track_rank > above && p.track_rank <= cnt) ? p.track_rank - above : 0u;
+      smem_pick2<H1_BINS>(s_m, K - above, rt, bw, rem, bt, trem_w);
+      // the keys of that bin go to a short list
+      uint32_t* lcnt = p.hist3 + (size_t)n * H3_BINS;
+      uint32_t* list = p.hist2 + (size_t)n * H2_BINS;
+      for (uint32_t li = tid; li < len; li += ST) {
+        const uint32_t kk = li < SK_KEYS ? s_keys[li] : __ldcg(&cd[s0 + li].x);
+        if (((kk - tau) >> WIN_SHIFT) == bw) {
+          const uint32_t at = atomicAdd(lcnt, 1u);
+          if (at < (uint32_t)WIN_LIST) list[at] = kk;
+        }
+      }
+      __threadfence();
+      cluster.sync();
+      const uint32_t m = __ldcg(lcnt);
+      if (m <= (uint32_t)WIN_LIST) {
+        resolved = true;
+        // rank the list: T_n is its rem-th largest key
+        uint32_t mine = 0;
+        if ((uint32_t)tid < m) {
+          mine = __ldcg(list + tid);
+          s_m[tid] = mine;
+        }
+        __syncthreads();
+        if ((uint32_t)tid < m) {
+          uint32_t gt = 0, eq = 0;
+          for (uint32_t i = 0; i < m; i++) {
+            const uint32_t o = s_m[i];
+            gt += o > mine;
+            eq += o == mine;
+          }
+          if (gt < rem && rem <= gt + eq) {  // every thread that holds T_n writes the same values
+            s_res3[0] = mine;
+            s_res3[1] = rem - gt;
+            s_res3[2] = eq;
+          }
+        }
+        __syncthreads();
+        T = s_res3[0];
+        need = s_res3[1];
+        cnt_eq = s_res3[2];
+        if (tracking && rank == 0 && tid == 0) {
+          uint32_t next = tau + (bt << WIN_SHIFT);
+          if (trem_w == 0) {
+            // the candidates do not reach the tracked rank: go below tau by linear extrapolation in
+            // key space from (K, T_n) and (cnt, tau), a quarter to spare, between 2^10 and 2^19 per call
+            const float slope = T > tau ? (float)(T - tau) / (float)(cnt - K + 1u) : 0.f;
+            float drop = 1.25f * slope * (float)(p.track_rank > cnt ? p.track_rank - cnt : 1u);
+            drop = fminf(fmaxf(drop, 1024.f), 524288.f);
+            next = tau > (uint32_t)drop ? tau - (uint32_t)drop : 0u;
+          }
+          p.tau_next[n] = next;
+        }
+      }
+    }
+  }
+  if (!resolved) {
+  // ---- digit 1 ----
+  if (fast) {
+    for (uint32_t l0 = 0; l0 < len; l0 += ST * 8) {  // uniform over the CTA
+      uint32_t k[8];
+#pragma unroll
+      for (int q = 0; q < 8; q++) {
+        const uint32_t li = l0 + q * ST + tid;
+        k[q] = li < len ? __ldcg(&cd[s0 + li].x) : 0u;
+      }
+#pragma unroll
+      for (int q = 0; q < 8; q++) {
+        const uint32_t li = l0 + q * ST + tid;
+        const bool ok = li < len;
+        const uint32_t act = __ballot_sync(FULL, ok);
+        if (ok) {
+          if (li < SK_KEYS) s_keys[li] = k[q];
+          // keys just above a threshold share a few leading digits: one shared-memory atomic per
+          // distinct digit of the warp instead of one per lane
+          const uint32_t bin = k[q] >> 20;
+          const uint32_t same = __match_any_sync(act, bin);
+          if (lane == __ffs(same) - 1) atomicAdd(&s_h[0][bin], (uint32_t)__popc(same));
+        }
+      }
+    }
+  } else {
+    cluster_row_keys(p, n, err, rank, [&](uint32_t key) { atomicAdd(&s_h[0][key >> 20], 1u); });
+  }
+  cluster.sync();
+  cluster_merge<H1_BINS>(cluster, s_h[0], s_m);
+  uint32_t b1, rem1, tb, trem;
+  smem_pick2<H1_BINS>(s_m, K, tracking ? p.track_rank : 0u, b1, rem1, tb, trem);
+  const uint32_t track_bin = (tracking && trem != 0 && tb != b1) ? tb : 0xffffffffu;
+
+  // ---- digit 2 (and, with threshold tracking, the second digit of the tracked rank) ----
+  auto add2 = [&](uint32_t key) {
+    const uint32_t d1 = key >> 20;
+    if (d1 == b1) atomicAdd(&s_h[1][(key >> 10) & 1023u], 1u);
+    else if (d1 == track_bin) atomicAdd(&s_h[1][1024u + ((key >> 10) & 1023u)], 1u);
+  };
+  if (fast) {
+    for (uint32_t li = tid; li < len; li += ST) add2(li < SK_KEYS ? s_keys[li] : __ldcg(&cd[s0 + li].x));
+  } else {
+    cluster_row_keys(p, n, err, rank, add2);
+  }
+  cluster.sync();
+  cluster_merge<H1_BINS>(cluster, s_h[1], s_m);
+  uint32_t b2, rem2, tb2 = 0, trem2 = 0;
+  if (tracking && trem != 0 && tb == b1) {  // the usual case: both ranks in the same first-digit bin
+    smem_pick2<H2_BINS>(s_m, rem1, trem, b2, rem2, tb2, trem2);
+  } else {
+    uint32_t u0, u1;
+    smem_pick2<H2_BINS>(s_m, rem1, 0u, b2, rem2, u0, u1);
+    if (tracking && trem != 0) smem_pick2<H2_BINS>(s_m + 1024, trem, 0u, tb2, trem2, u0, u1);
+  }
+  if (tracking && rank == 0 && tid == 0) {
+    uint32_t next = (tb << 20) | (tb2 << 10);
+    if (trem == 0) {
+      // the counted keys do not reach the tracked rank: go below tau by linear extrapolation in key
+      // space from (K, K-th key) and (cnt, tau), a quarter to spare, between 2^10 and 2^19 per call
+      const uint32_t tau = p.tau[n];
+      const uint32_t t21 = (b1 << 20) | (b2 << 10);
+      const float slope = (t21 > tau && cnt >= K) ? (float)(t21 - tau) / (float)(cnt - K + 1u) : 0.f;
+      float drop = 1.25f * slope * (float)(p.track_rank > cnt ? p.track_rank - cnt : 1u);
+      drop = fminf(fmaxf(drop, 1024.f), 524288.f);
+      next = tau > (uint32_t)drop ? tau - (uint32_t)drop : 0u;
+    }
+    p.tau_next[n] = next;
+  }
+
+  // ---- digit 3 ----
+  const uint32_t prefix = (b1 << 10) | b2;
+  auto add3 = [&](uint32_t key) {
+    if ((key >> 10) == prefix) atomicAdd(&s_h[2][key & 1023u], 1u);
+  };
+  if (fast) {
+    for (uint32_t li = tid; li < len; li += ST) add3(li < SK_KEYS ? s_keys[li] : __ldcg(&cd[s0 + li].x));
+  } else {
+    cluster_row_keys(p, n, err, rank, add3);
+  }
+  cluster.sync();
+  cluster_merge<H3_BINS>(cluster, s_h[2], s_m);
+  uint32_t b3, u0, u1;
+  smem_pick2<H3_BINS>(s_m, rem2, 0u, b3, need, u0, u1);
+  cnt_eq = s_m[b3];
+  T = (b1 << 20) | (b2 << 10) | b3;
+  cluster.sync();  // from here on no CTA reads a peer's shared memory
+  }
+  if (rank == 0 && tid == 0) {
+    uint32_t* ws = p.wstate + (size_t)n * 8;
+    ws[4] = T;
+    ws[5] = K - need;
+    ws[6] = cnt_eq;
+    ws[7] = need;
+    p.thresh[n * 3 + 0] = T;
+    p.thresh[n * 3 + 1] = K - need;
+    p.thresh[n * 3 + 2] = cnt_eq;
+    p.diag_cnt[n] = cnt;
+  }
+  const bool all_ties = need >= cnt_eq;  // alike in every CTA of the cluster
+
+  if (fast) {
+    // the picks themselves are made by k_set_bits, which follows; a worker that keeps only part of its
+    // threshold ties (lowest index first) needs the ties per chunk and their running offsets for that
+    if (all_ties) return;
+    for (int c = (int)rank * (ST / 32) + warp; c < p.nchunks; c += CL * (ST / 32)) {
+      const size_t ci = (size_t)n * p.nchunks + c;
+      const uint32_t ccnt = p.chunk_cnt[ci], base = p.chunk_base[ci];
+      uint32_t eq = 0;
+      for (uint32_t i = lane; i < ccnt; i += 32) eq += __ldcg(&cd[base + i].x) == T;
+      eq = __reduce_add_sync(FULL, eq);
+      if (lane == 0) p.chunk_eq[ci] = eq;
+    }
+    __threadfence();
+    cluster.sync();
+    if (rank == 0) chunk_scan<ST>(p, n);
+    return;
+  }
+
+  // ---- full-row worker: its picks are read off the row itself by k_set_bits; partly kept ties need
+  // the ties per chunk and their running offsets ----
+  if (all_ties) return;
+  const int sub = tid >> 8, t = tid & 255, w8 = t >> 5;
+  for (int c0 = (int)rank * 4; c0 < p.nchunks; c0 += CL * 4) {  // uniform over the CTA
+    const int c = c0 + sub;
+    const bool valid = c < p.nchunks;
+    uint32_t eq = 0;
+    if (valid) {
+      const Geom g = chunk_geom(n, c, p.d);
+      uint32_t key[4][4], vm[4];
+      load_keys<false>(g, nullptr, err, key, vm, t);
+#pragma unroll
+      for (int i = 0; i < 4; i++) eq += __popc(vm[i] & eq_mask(key[i], T));
+      if (t == TPB - 1) {
+        uint32_t xkey[4], xvm;
+        load_extra<false>(g, nullptr, err, xkey, xvm);
+        eq += __popc(xvm & eq_mask(xkey, T));
+      }
+    }
+    eq = __reduce_add_sync(FULL, eq);
+    if (lane == 0) s_te[sub][w8] = eq;
+    __syncthreads();
+    if (valid && t == 0) {
+      uint32_t te = 0;
+      for (int w = 0; w < 8; w++) te += s_te[sub][w];
+      p.chunk_eq[(size_t)n * p.nchunks + c] = te;
+    }
+    __syncthreads();
+  }
+  __threadfence();
+  cluster.sync();
+  if (rank == 0) chunk_scan<ST>(p, n);
 }
 
 constexpr int VT = 128;  // threads of k_votes: one per mask word of the chunk
@@ -1232,31 +1684,83 @@ __global__ void __launch_bounds__(TPB) k_lists(P p) {
 // mask: counting select over the vote values 0..N
 // ---------------------------------------------------------------------------------------------
 // per-chunk and global histogram of vote values, from a vote vector (stand-alone mv_select)
-__global__ void __launch_bounds__(TPB) k_vote_hist(P p, const uint8_t* __restrict__ votes) {
+// `copy` (optional): the votes are also written there (the caller's array, when the count was kept elsewhere).
+// A warp per chunk: its 4096 vote bytes are eight 16-byte loads per lane, all in flight together, and
+// nothing in a chunk's path waits for another warp; the CTA's eight chunks share one flush of the
+// global counts and one ticket.
+constexpr int VH_WARPS = TPB / 32;
+
+__global__ void __launch_bounds__(TPB) k_vote_hist(P p, const uint8_t* __restrict__ votes, uint8_t* __restrict__ copy) {
   pdl_enter();
-  __shared__ uint32_t s_vh[256];
-  const int c = blockIdx.x, tid = threadIdx.x;
-  s_vh[tid] = 0;
-  __syncthreads();
-  const int64_t jb = (int64_t)c * CH + (int64_t)tid * 16;
-  if (jb < p.d) {
-    if (jb + 16 <= p.d) {
-      const uint4 q = *reinterpret_cast<const uint4*>(votes + jb);
-      const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+  __shared__ uint32_t s_vh[VH_WARPS][256];  // exact counts per vote value, one row per warp
+  __shared__ uint32_t s_tot[256];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int c = blockIdx.x * VH_WARPS + warp;
+  s_tot[tid] = 0;
 #pragma unroll
-      for (int b = 0; b < 16; b++) {
-        const uint32_t v = (w[b >> 2] >> (8 * (b & 3))) & 0xffu;
-        if (v) atomicAdd(&s_vh[v], 1u);
+  for (int k = 0; k < 8; k++) s_vh[warp][k * 32 + lane] = 0;
+  __syncthreads();
+  if (c < p.nchunks) {
+    uint4 q[8];
+#pragma unroll
+    for (int u = 0; u < 8; u++) {
+      const int64_t jb = (int64_t)c * CH + (int64_t)(u * 32 + lane) * 16;
+      q[u] = make_uint4(0, 0, 0, 0);
+      if (jb + 16 <= p.d) {
+        q[u] = __ldcg(reinterpret_cast<const uint4*>(votes + jb));
+      } else if (jb < p.d) {  // the row's last, partial 16 bytes
+        uint32_t w[4] = {0, 0, 0, 0};
+        for (int b = 0; b < 16 && jb + b < p.d; b++) w[b >> 2] |= (uint32_t)__ldcg(votes + jb + b) << (8 * (b & 3));
+        q[u] = make_uint4(w[0], w[1], w[2], w[3]);
       }
-    } else {
-      for (int b = 0; b < 16 && jb + b < p.d; b++) {
-        const uint32_t v = votes[jb + b];
-        if (v) atomicAdd(&s_vh[v], 1u);
+    }
+#pragma unroll
+    for (int u = 0; u < 8; u++) {
+      const int64_t jb = (int64_t)c * CH + (int64_t)(u * 32 + lane) * 16;
+      const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+      if (copy != nullptr) {
+        if (jb + 16 <= p.d) {
+          *reinterpret_cast<uint4*>(copy + jb) = q[u];
+        } else {
+          for (int b = 0; b < 16 && jb + b < p.d; b++) copy[jb + b] = (uint8_t)((w[b >> 2] >> (8 * (b & 3))) & 0xffu);
+        }
       }
+      if (w[0] | w[1] | w[2] | w[3]) {
+#pragma unroll
+        for (int b = 0; b < 16; b++) {
+          const uint32_t v = (w[b >> 2] >> (8 * (b & 3))) & 0xffu;
+          if (v) atomicAdd(&s_vh[warp][v], 1u);
+        }
+      }
+    }
+    __syncwarp();
+    // cum[v] = #{votes >= v}: lane l owns the values 8l .. 8l+7
+    uint32_t ex[8], lsum = 0;
+#pragma unroll
+    for (int k = 0; k < 8; k++) {
+      const int v = lane * 8 + k;
+      ex[k] = (v >= 1 && v <= p.N) ? s_vh[warp][v] : 0u;
+      lsum += ex[k];
+    }
+    uint32_t x = lsum;  // inclusive suffix sum over the lanes
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const uint32_t y = __shfl_down_sync(FULL, x, off);
+      if (lane + off < 32) x += y;
+    }
+    uint32_t run = x - lsum;  // counts of the values owned by higher lanes
+    const int64_t rem = p.d - (int64_t)c * CH;
+    const uint32_t valid = (uint32_t)(rem < CH ? rem : CH);
+#pragma unroll
+    for (int k = 7; k >= 0; k--) {
+      const int v = lane * 8 + k;
+      run += ex[k];
+      if (v <= p.N) p.chunk_vh[(size_t)v * p.nc_pad + c] = (uint16_t)(v == 0 ? valid : run);
+      if (ex[k]) atomicAdd(&s_tot[v], ex[k]);
     }
   }
   __syncthreads();
-  store_vote_hist_impl(p, c, s_vh);
+  if (tid >= 1 && tid <= p.N && s_tot[tid]) atomicAdd(&p.vote_hist[tid], s_tot[tid]);  // the zero-vote count is derived later
   if (last_cta(p.votes_done, gridDim.x)) vote_scan<TPB>(p);
 }
 
@@ -1580,12 +2084,14 @@ __global__ void __launch_bounds__(TPB) k_rs_fill(P p, P a, const uint8_t* __rest
   }
 }
 
-// selected coordinates per chunk of one bit-mask row (a warp per chunk)
+// selected coordinates per chunk of bit-mask row blockIdx.y (a warp per chunk)
 __global__ void __launch_bounds__(TPB) k_chunk_popc(const uint32_t* __restrict__ bits, int64_t W, int nchunks,
                                                     uint32_t* __restrict__ chunk_sel) {
   pdl_enter();
   const int c = blockIdx.x * (TPB / 32) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
   if (c >= nchunks) return;
+  bits += (size_t)blockIdx.y * (size_t)W;
+  chunk_sel += (size_t)blockIdx.y * (size_t)nchunks;
   uint32_t s = 0;
 #pragma unroll
   for (int q = 0; q < 4; q++) {
@@ -1752,6 +2258,7 @@ P make_params(const mv_ctx* ctx, const Layout& L, int N, int64_t d, int64_t K) {
   p.force_general = ctx->mode == MV_MODE_GENERAL ? 1 : 0;
   p.list_mode = 0;
   p.apply_rows = 0;
+  p.vote_words = nullptr;
   p.apply_bits = nullptr;
   p.d = d;
   p.K = K;
@@ -1791,11 +2298,11 @@ P make_params(const mv_ctx* ctx, const Layout& L, int N, int64_t d, int64_t K) {
 }
 
 template <typename... KArgs, typename... Args>
-cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args) {
+cudaError_t launch_smem(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
-  cfg.dynamicSmemBytes = 0;
+  cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -1803,6 +2310,27 @@ cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args) {
+  return launch_smem(kernel, grid, block, 0, st, args...);
+}
+
+// k_select_cluster keeps SK_KEYS keys in dynamic shared memory: above the default limit, so the
+// kernel is told once per device
+bool cluster_select_ready() {
+  static bool done[64] = {false};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+  if (!done[dev]) {
+    if (cudaFuncSetAttribute(k_select_cluster, cudaFuncAttributeMaxDynamicSharedMemorySize, SK_KEYS * 4) != cudaSuccess) {
+      cudaGetLastError();
+      return false;
+    }
+    done[dev] = true;
+  }
+  return true;
 }
 
 int per_row_ctas(int N, int want, int budget) {
@@ -1884,13 +2412,13 @@ int vote_impl(mv_ctx* ctx, P p, const Layout& L, const float* grads, float* err,
   if (ctx->clean_bytes < L.zero_bytes && cudaMemsetAsync(ctx->ws, 0, L.zero_bytes, st) != cudaSuccess)
     return MV_ERR_CUDA;
   ctx->clean_bytes = 0;  // dirty from here on, until a whole step's last kernel has cleared it again
-  // per-chunk outputs of the vote count start out cleared (only chunks with candidates are
-  // visited later); cleared on the side stream, concurrently with the sampling and streaming pass
+  // general mode: per-chunk outputs of the vote count start out cleared (only chunks with picks are
+  // visited later); cleared on the side stream, concurrently with the first pass
   cudaStream_t zs = st;
-  if (!topk_only && ctx->phase_timing != 1 && side_ready(ctx) && cudaEventRecord(ctx->ev_fork, st) == cudaSuccess &&
-      cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) == cudaSuccess)
+  if (p.force_general && !topk_only && ctx->phase_timing != 1 && side_ready(ctx) &&
+      cudaEventRecord(ctx->ev_fork, st) == cudaSuccess && cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) == cudaSuccess)
     zs = ctx->side;
-  {
+  if (p.force_general && !topk_only) {
     const size_t nc = (size_t)p.nchunks;
     cudaError_t e = cudaMemsetAsync(p.votes, 0, (size_t)p.d, zs);
     if (e == cudaSuccess) e = cudaMemsetAsync(p.chunk_sel, 0, (size_t)N * nc * 4, zs);
@@ -1926,11 +2454,27 @@ int vote_impl(mv_ctx* ctx, P p, const Layout& L, const float* grads, float* err,
       launch_k(k_sample_hist, dim3(dim3(gs, N)), dim3(512), st, p, grads, err, U, Ls, all, rank);
       MV_LAUNCH_CHECK();
     }
+    // the votes are counted while the picks are made, in the workspace's vote array (whole chunks long)
+    uint8_t* const ws_votes = (uint8_t*)(ctx->ws + L.votes);
+    p.vote_words = topk_only ? nullptr : (uint32_t*)ws_votes;
     if (ctx->timing_now) cudaEventRecord(ctx->ev[2 * (ctx->timed % 64)], st);
     launch_k(k_acc_compact, dim3(dim3(p.nchunks, N)), dim3(TPB), st, p, grads, err);
     MV_LAUNCH_CHECK();
     if (ctx->timing_now) cudaEventRecord(ctx->ev[2 * (ctx->timed++ % 64) + 1], st);
-    launch_k(k_hist<1, false>, dim3(dim3(gh, N)), dim3(TPB), st, p, nullptr, err);
+    if (!cluster_select_ready()) return MV_ERR_CUDA;
+    // a cluster per worker resolves T_n, sets the worker's mask bits and adds its votes
+    // (with few workers, extra clusters that only help clearing fill the GPU)
+    const int zc = N * CL < 144 ? (144 - N * CL) / CL : 0;
+    launch_smem(k_select_cluster, dim3(dim3(CL, N + zc)), dim3(ST), SK_KEYS * 4, st, p, err);
+    MV_LAUNCH_CHECK();
+    // the picks: mask bits and votes, from the candidates (or the row), by the whole GPU
+    launch_k(k_set_bits, dim3(dim3(per_row_ctas(N, (int)((p.cap + TPB * 16 - 1) / (TPB * 16)), 148 * 4), N)), dim3(TPB), st, p,
+             err);
+    MV_LAUNCH_CHECK();
+    if (topk_only) return MV_OK;
+    // vote histograms per chunk, v* and the output offsets (the caller's vote array gets its copy here)
+    launch_k(k_vote_hist, dim3((p.nchunks + VH_WARPS - 1) / VH_WARPS), dim3(TPB), st, p, (const uint8_t*)ws_votes,
+             p.votes != ws_votes ? p.votes : (uint8_t*)nullptr);
     MV_LAUNCH_CHECK();
   } else {
     if (ctx->timing_now) cudaEventRecord(ctx->ev[2 * (ctx->timed % 64)], st);
@@ -1938,30 +2482,36 @@ int vote_impl(mv_ctx* ctx, P p, const Layout& L, const float* grads, float* err,
     MV_LAUNCH_CHECK();
     if (ctx->timing_now) cudaEventRecord(ctx->ev[2 * (ctx->timed++ % 64) + 1], st);
   }
-  launch_k(k_hist<2, false>, dim3(dim3(gh, N)), dim3(TPB), st, p, nullptr, err);
-  MV_LAUNCH_CHECK();
-  launch_k(k_hist<3, false>, dim3(dim3(gh, N)), dim3(TPB), st, p, nullptr, err);
-  MV_LAUNCH_CHECK();
-  launch_k(k_count, dim3(dim3(gh, N)), dim3(TPB), st, p, err);
-  MV_LAUNCH_CHECK();
-  const int gb = p.force_general ? gh : per_row_ctas(N, (int)((p.cap + TPB * 16 - 1) / (TPB * 16)), 148 * 4);
-  launch_k(k_set_bits, dim3(dim3(gb, N)), dim3(TPB), st, p, err);
-  MV_LAUNCH_CHECK();
+  if (p.force_general) {
+    launch_k(k_hist<2, false>, dim3(dim3(gh, N)), dim3(TPB), st, p, nullptr, err);
+    MV_LAUNCH_CHECK();
+    launch_k(k_hist<3, false>, dim3(dim3(gh, N)), dim3(TPB), st, p, nullptr, err);
+    MV_LAUNCH_CHECK();
+    launch_k(k_count, dim3(dim3(gh, N)), dim3(TPB), st, p, err);
+    MV_LAUNCH_CHECK();
+    launch_k(k_set_bits, dim3(dim3(gh, N)), dim3(TPB), st, p, err);
+    MV_LAUNCH_CHECK();
+  }
   if (topk_only) return MV_OK;
-  if (zs != st && cudaStreamWaitEvent(st, ctx->ev_zero, 0) != cudaSuccess) return MV_ERR_CUDA;
-  {
+  if (p.force_general) {
+    if (zs != st && cudaStreamWaitEvent(st, ctx->ev_zero, 0) != cudaSuccess) return MV_ERR_CUDA;
     const dim3 gv(p.nchunks < 148 * 8 ? p.nchunks : 148 * 8);
     if (N < 4) launch_k(k_votes<2>, gv, dim3(VT), st, p);
     else if (N < 16) launch_k(k_votes<4>, gv, dim3(VT), st, p);
     else if (N < 64) launch_k(k_votes<6>, gv, dim3(VT), st, p);
     else launch_k(k_votes<8>, gv, dim3(VT), st, p);
+    MV_LAUNCH_CHECK();
   }
-  MV_LAUNCH_CHECK();
   // the index lists feed nothing later in the step: write them on the side stream
   cudaStream_t ls = st;
   if (ctx->phase_timing != 1 && side_ready(ctx) && cudaEventRecord(ctx->ev_fork, st) == cudaSuccess &&
       cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) == cudaSuccess)
     ls = ctx->side;
+  if (!p.force_general) {  // selected coordinates per (worker, chunk), which the general vote count leaves behind
+    launch_k(k_chunk_popc, dim3(dim3((p.nchunks + TPB / 32 - 1) / (TPB / 32), N)), dim3(TPB), ls,
+             (const uint32_t*)p.worker_bits, p.W, p.nchunks, p.chunk_sel);
+    MV_LAUNCH_CHECK();
+  }
   launch_k(k_scan_sel, dim3(N), dim3(1024), ls, p);
   MV_LAUNCH_CHECK();
   launch_k(k_lists, dim3(dim3((p.nchunks + TPB / 32 - 1) / (TPB / 32), N)), dim3(TPB), ls, p);
@@ -1980,7 +2530,7 @@ int select_impl(mv_ctx* ctx, P p, const Layout& L, const uint8_t* votes, bool ha
   if (!have_hist) {
     ctx->clean_bytes = 0;
     if (cudaMemsetAsync(ctx->ws + L.votes_done, 0, L.zero_bytes - L.votes_done, st) != cudaSuccess) return MV_ERR_CUDA;
-    launch_k(k_vote_hist, dim3(p.nchunks), dim3(TPB), st, p, votes);
+    launch_k(k_vote_hist, dim3((p.nchunks + VH_WARPS - 1) / VH_WARPS), dim3(TPB), st, p, votes, (uint8_t*)nullptr);
     MV_LAUNCH_CHECK();
   }
   launch_k(k_vote_write, dim3(p.nchunks), dim3(TPB), st, p, votes, out_idx, mask_bits);
@@ -2549,7 +3099,8 @@ int mv_select_static(void* stream, const uint8_t* votes, int N, int64_t d, int64
   p.chunk_vh = (uint16_t*)(base + ST_CHUNK_VH);
   // the array keeps whatever the last call left: the ticket and the vote histogram start at zero
   if (cudaMemsetAsync(base, 0, ST_VSTATE, st) != cudaSuccess) return MV_ERR_CUDA;
-  if (launch_k(k_vote_hist, dim3(p.nchunks), dim3(TPB), st, p, votes) != cudaSuccess) return MV_ERR_CUDA;
+  if (launch_k(k_vote_hist, dim3((p.nchunks + VH_WARPS - 1) / VH_WARPS), dim3(TPB), st, p, votes, (uint8_t*)nullptr) != cudaSuccess)
+    return MV_ERR_CUDA;
   if (launch_k(k_vote_write, dim3(p.nchunks), dim3(TPB), st, p, votes, out_idx, mask_bits) != cudaSuccess)
     return MV_ERR_CUDA;
   if (cudaGetLastError() != cudaSuccess) return MV_ERR_CUDA;
