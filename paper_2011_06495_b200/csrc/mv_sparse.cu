@@ -61,6 +61,7 @@ struct P {
   int force_general;
   int list_mode;          // 1: the rows are plain (key, index) lists to select min(K, length) from (add-drop)
   int apply_rows;         // list mode: rows < apply_rows are "add" lists, the others "drop" lists
+  const float* prefetch_acc;  // k_vote_write: if set, the rows whose elements at supp(M) the gather is about to read
   uint32_t* vote_words;   // cluster select: if set, every pick also adds one to its vote byte (four bytes per word)
   uint32_t* apply_bits;   // list mode, optional: the vote masks [apply_rows][W] to update in place instead of
                           // writing the picks to worker_bits
@@ -1137,7 +1138,8 @@ __global__ void __launch_bounds__(TPB) k_set_bits(P p, float* __restrict__ err) 
 // ---------------------------------------------------------------------------------------------
 namespace cg = cooperative_groups;
 
-constexpr int CL = 8;           // CTAs of the cluster that serves one worker (portable cluster size)
+// CL = CTAs of the cluster that serves one worker: 8 (the portable maximum), or 4 when there are so many
+// workers that clusters of 8 would not all be resident at once
 constexpr int ST = 1024;        // threads per CTA
 constexpr int SK_KEYS = 32768;  // candidate keys a CTA keeps in shared memory between the digit passes
 
@@ -1196,7 +1198,7 @@ __device__ void smem_pick2(const uint32_t* s_hist, uint32_t rank_a, uint32_t ran
 }
 
 // s_out[b] = sum over the cluster's CTAs of their s_local[b]
-template <int NB>
+template <int NB, int CL>
 __device__ __forceinline__ void cluster_merge(cg::cluster_group& cluster, uint32_t* s_local, uint32_t* s_out) {
   const uint32_t* peer[CL];
 #pragma unroll
@@ -1215,7 +1217,7 @@ __device__ __forceinline__ void cluster_merge(cg::cluster_group& cluster, uint32
 
 // f(key) for every element of the chunks of row n that fall to CTA `rank` of the cluster: four
 // chunks at a time, 256 threads each
-template <typename F>
+template <int CL, typename F>
 __device__ __forceinline__ void cluster_row_keys(const P& p, int n, float* __restrict__ err, uint32_t rank, F f) {
   const int sub = threadIdx.x >> 8, t = threadIdx.x & 255;
   for (int c = (int)rank * 4 + sub; c < p.nchunks; c += CL * 4) {
@@ -1237,7 +1239,8 @@ __device__ __forceinline__ void cluster_row_keys(const P& p, int n, float* __res
   }
 }
 
-__global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(ST, 1) k_select_cluster(P p, float* __restrict__ err) {
+template <int CL>
+__global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(ST, 1) k_select_cluster(P p, float* __restrict__ err, int zero_first) {
   pdl_enter();
   cg::cluster_group cluster = cg::this_cluster();
   extern __shared__ uint32_t s_keys[];       // [SK_KEYS]
@@ -1252,9 +1255,13 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(ST, 1) k_select_clu
     // of the grid together, and not in the streaming pass: what is written now is still in L2 when
     // the picks arrive as atomics (k_set_bits), whereas lines cleared before the row streamed through
     // would each have to come back from DRAM.  Clusters beyond the workers' only clear.
-    const size_t nblocks = (size_t)gridDim.x * gridDim.y, bid = (size_t)blockIdx.y * gridDim.x + blockIdx.x;
-    zero_share(p.worker_bits, (size_t)p.N * (size_t)p.W, bid, nblocks);
-    if (p.vote_words != nullptr) zero_share(p.vote_words, (size_t)p.nchunks * (CH / 4), bid, nblocks);
+    // Clusters zero_first and up take part: all of them, or only the extra ones when those are many.
+    if ((int)blockIdx.y >= zero_first) {
+      const size_t nblocks = (size_t)gridDim.x * (gridDim.y - zero_first);
+      const size_t bid = (size_t)(blockIdx.y - zero_first) * gridDim.x + blockIdx.x;
+      zero_share(p.worker_bits, (size_t)p.N * (size_t)p.W, bid, nblocks);
+      if (p.vote_words != nullptr) zero_share(p.vote_words, (size_t)p.nchunks * (CH / 4), bid, nblocks);
+    }
   }
   if ((int)blockIdx.y >= p.N) return;  // alike in every CTA of the cluster
   const int n = blockIdx.y;
@@ -1400,10 +1407,10 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(ST, 1) k_select_clu
       }
     }
   } else {
-    cluster_row_keys(p, n, err, rank, [&](uint32_t key) { atomicAdd(&s_h[0][key >> 20], 1u); });
+    cluster_row_keys<CL>(p, n, err, rank, [&](uint32_t key) { atomicAdd(&s_h[0][key >> 20], 1u); });
   }
   cluster.sync();
-  cluster_merge<H1_BINS>(cluster, s_h[0], s_m);
+  cluster_merge<H1_BINS, CL>(cluster, s_h[0], s_m);
   uint32_t b1, rem1, tb, trem;
   smem_pick2<H1_BINS>(s_m, K, tracking ? p.track_rank : 0u, b1, rem1, tb, trem);
   const uint32_t track_bin = (tracking && trem != 0 && tb != b1) ? tb : 0xffffffffu;
@@ -1417,10 +1424,10 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(ST, 1) k_select_clu
   if (fast) {
     for (uint32_t li = tid; li < len; li += ST) add2(li < SK_KEYS ? s_keys[li] : __ldcg(&cd[s0 + li].x));
   } else {
-    cluster_row_keys(p, n, err, rank, add2);
+    cluster_row_keys<CL>(p, n, err, rank, add2);
   }
   cluster.sync();
-  cluster_merge<H1_BINS>(cluster, s_h[1], s_m);
+  cluster_merge<H1_BINS, CL>(cluster, s_h[1], s_m);
   uint32_t b2, rem2, tb2 = 0, trem2 = 0;
   if (tracking && trem != 0 && tb == b1) {  // the usual case: both ranks in the same first-digit bin
     smem_pick2<H2_BINS>(s_m, rem1, trem, b2, rem2, tb2, trem2);
@@ -1452,10 +1459,10 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(ST, 1) k_select_clu
   if (fast) {
     for (uint32_t li = tid; li < len; li += ST) add3(li < SK_KEYS ? s_keys[li] : __ldcg(&cd[s0 + li].x));
   } else {
-    cluster_row_keys(p, n, err, rank, add3);
+    cluster_row_keys<CL>(p, n, err, rank, add3);
   }
   cluster.sync();
-  cluster_merge<H3_BINS>(cluster, s_h[2], s_m);
+  cluster_merge<H3_BINS, CL>(cluster, s_h[2], s_m);
   uint32_t b3, u0, u1;
   smem_pick2<H3_BINS>(s_m, rem2, 0u, b3, need, u0, u1);
   cnt_eq = s_m[b3];
@@ -1822,7 +1829,15 @@ __global__ void __launch_bounds__(TPB) k_vote_write(P p, const uint8_t* __restri
   while (s2) {
     const int b = __ffs(s2) - 1;
     s2 &= s2 - 1;
-    if (pos < (uint32_t)p.K) out_idx[pos] = (int32_t)(jb + b);
+    if (pos < (uint32_t)p.K) {
+      out_idx[pos] = (int32_t)(jb + b);
+      // the gather that follows reads this coordinate of every row, scattered over DRAM: ask for
+      // those sectors now, so that they are on their way while this kernel drains and the next starts
+      if (p.prefetch_acc != nullptr) {
+        const float* a = p.prefetch_acc + (jb + b);
+        for (int n = 0; n < p.N; n++) asm volatile("prefetch.global.L2 [%0];" ::"l"(a + (size_t)n * (size_t)p.d));
+      }
+    }
     pos++;
   }
   if (mask_bits != nullptr) {
@@ -2259,6 +2274,7 @@ P make_params(const mv_ctx* ctx, const Layout& L, int N, int64_t d, int64_t K) {
   p.list_mode = 0;
   p.apply_rows = 0;
   p.vote_words = nullptr;
+  p.prefetch_acc = nullptr;
   p.apply_bits = nullptr;
   p.d = d;
   p.K = K;
@@ -2324,7 +2340,8 @@ bool cluster_select_ready() {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
   if (!done[dev]) {
-    if (cudaFuncSetAttribute(k_select_cluster, cudaFuncAttributeMaxDynamicSharedMemorySize, SK_KEYS * 4) != cudaSuccess) {
+    if (cudaFuncSetAttribute(k_select_cluster<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, SK_KEYS * 4) != cudaSuccess ||
+        cudaFuncSetAttribute(k_select_cluster<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, SK_KEYS * 4) != cudaSuccess) {
       cudaGetLastError();
       return false;
     }
@@ -2464,8 +2481,14 @@ int vote_impl(mv_ctx* ctx, P p, const Layout& L, const float* grads, float* err,
     if (!cluster_select_ready()) return MV_ERR_CUDA;
     // a cluster per worker resolves T_n, sets the worker's mask bits and adds its votes
     // (with few workers, extra clusters that only help clearing fill the GPU)
-    const int zc = N * CL < 144 ? (144 - N * CL) / CL : 0;
-    launch_smem(k_select_cluster, dim3(dim3(CL, N + zc)), dim3(ST), SK_KEYS * 4, st, p, err);
+    const int cl = N * 8 <= 144 ? 8 : 4;                    // one CTA per SM: keep all clusters resident if possible
+    const int zc = N * cl < 144 ? (144 - N * cl) / cl : 0;  // clusters that only clear
+    // the extra clusters clear alone if that does not take them longer than the select takes (measured:
+    // about 450 KB per CTA); otherwise every CTA of the grid clears a share first
+    const size_t clear_bytes = (size_t)N * (size_t)p.W * 4 + (topk_only ? 0 : (size_t)p.nchunks * CH);
+    const int zero_first = (zc * cl >= 32 && clear_bytes / (size_t)(zc * cl) <= 450 * 1024) ? N : 0;
+    if (cl == 8) launch_smem(k_select_cluster<8>, dim3(dim3(8, N + zc)), dim3(ST), SK_KEYS * 4, st, p, err, zero_first);
+    else launch_smem(k_select_cluster<4>, dim3(dim3(4, N + zc)), dim3(ST), SK_KEYS * 4, st, p, err, zero_first);
     MV_LAUNCH_CHECK();
     // the picks: mask bits and votes, from the candidates (or the row), by the whole GPU
     launch_k(k_set_bits, dim3(dim3(per_row_ctas(N, (int)((p.cap + TPB * 16 - 1) / (TPB * 16)), 148 * 4), N)), dim3(TPB), st, p,
@@ -2767,6 +2790,7 @@ int mv_sparse_step(mv_ctx* ctx, const float* grads, float* err, int N, int64_t d
   ctx->last_d = d;
   ctx->last_K = K;
   rc = vote_impl(ctx, p, L, grads, err);
+  p.prefetch_acc = err;
   if (rc == MV_OK) rc = select_impl(ctx, p, L, p.votes, true, out_idx, nullptr);
   if (rc == MV_OK) rc = aggregate_impl(ctx, err, N, d, K, out_idx, out_val, L.zero_bytes);
   const int rcj = join_side(ctx);

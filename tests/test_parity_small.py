@@ -287,6 +287,32 @@ def test_threshold_tracking_over_steps(N, d, K):
     assert launches[0] == launches[1] + 1 and len(set(launches[1:])) == 1      # the sampling kernel runs once
 
 
+@pytest.mark.parametrize("mode", [B.MV_MODE_AUTO, B.MV_MODE_TRACK], ids=["auto", "track"])
+def test_magnitudes_spread_over_many_binades(mode):
+    """Magnitudes log-uniform over sixty binades: the candidates above the threshold bound span many
+    powers of two, so the K-th key lies far outside the narrow window of keys that the select looks
+    at first and the three-digit radix select over the candidates has to find it; with ties (every
+    magnitude is a power of 2^(1/8), so there are only a few hundred distinct keys) on top."""
+    N, d, K = 3, 300_007, 2000
+    g = torch.Generator().manual_seed(4242)
+    ctx = B.MvContext(N, d, K, device=DEV, mode=mode)
+    err_gpu = torch.zeros(N, d, device=DEV)
+    err_ref = np.zeros((N, d), dtype=np.float32)
+    out_idx = torch.empty(K, dtype=torch.int32, device=DEV)
+    out_val = torch.empty(K, dtype=torch.float32, device=DEV)
+    for step in range(3):
+        expo = torch.randint(-240, 240, (N, d), generator=g).float() / 8.0
+        sign = torch.randint(0, 2, (N, d), generator=g).float() * 2 - 1
+        grads = (sign * torch.exp2(expo)).float().contiguous()
+        ref = O.mv_sparse_step(grads.numpy(), err_ref, K)
+        ctx.mv_sparse_step(grads.to(DEV), err_gpu, out_idx, out_val)
+        torch.cuda.synchronize()
+        PT.first_diff(PT.npy(out_idx), ref["out_idx"], f"step {step} out_idx")
+        PT.check_out_val(PT.npy(out_val), ref, ref["acc"], ref["out_idx"].astype(np.int64), f"step {step} out_val")
+        PT.first_diff(PT.bits(PT.npy(err_gpu)), PT.bits(ref["err"]), f"step {step} err")
+        err_ref = ref["err"]
+
+
 @pytest.mark.parametrize("name,N,d,K", [("c3", 8, 400_009, 400), ("c2", 6, 300_007, 3000), ("c4", 4, 500_003, 125)])
 def test_threshold_tracking_long_run(name, N, d, K):
     """Hundreds of consecutive steps: the tracked threshold neither drifts out of the usable range
