@@ -386,6 +386,49 @@ def test_threshold_tracking_survives_a_change_of_scale():
     assert ctx.last_launches() == before - 1
 
 
+@pytest.mark.parametrize("mode", [B.MV_MODE_AUTO, B.MV_MODE_TRACK], ids=["auto", "track"])
+def test_one_context_changing_K_and_entry_points(mode):
+    """One context serves steps whose K changes from call to call, with other entry points (the
+    three phases, with buffers of their own) called in between: every call starts from clean
+    scratch counters, masks and votes whatever the call before it left, and a tracked threshold
+    of another K is not reused."""
+    N, d = 5, 200_003
+    Ks = [2000, 150, 2000, 2000, 7000, 150, 2000]
+    g = torch.Generator().manual_seed(9001)
+    ctx = B.MvContext(N, d, max(Ks), device=DEV, mode=mode)
+    err_gpu = torch.zeros(N, d, device=DEV)
+    err_ref = np.zeros((N, d), dtype=np.float32)
+    W = (d + 31) // 32
+    for step, K in enumerate(Ks):
+        grads = torch.randn(N, d, generator=g) * (1.0 + 0.1 * step)
+        ref = O.mv_sparse_step(grads.numpy(), err_ref, K)
+        out_idx = torch.full((K,), -7, dtype=torch.int32, device=DEV)
+        out_val = torch.full((K,), float("nan"), dtype=torch.float32, device=DEV)
+        ctx.mv_sparse_step(grads.to(DEV), err_gpu, out_idx, out_val, K=K)
+        torch.cuda.synchronize()
+        PT.first_diff(PT.npy(out_idx), ref["out_idx"], f"step {step} K={K} out_idx")
+        PT.check_out_val(PT.npy(out_val), ref, ref["acc"], ref["out_idx"].astype(np.int64), f"step {step} out_val")
+        PT.first_diff(PT.bits(PT.npy(err_gpu)), PT.bits(ref["err"]), f"step {step} err")
+        err_ref = ref["err"]
+        if step % 2 == 0:
+            # the phases on other data, another K, outputs in caller buffers: must not disturb the next step
+            K2 = 333
+            g2 = torch.randn(N, d, generator=g)
+            acc2 = torch.zeros(N, d, device=DEV)
+            votes = torch.full((d,), 9, dtype=torch.uint8, device=DEV)
+            bits_ = torch.full((N, W), -1, dtype=torch.int32, device=DEV)
+            idx2 = torch.empty(K2, dtype=torch.int32, device=DEV)
+            val2 = torch.empty(K2, dtype=torch.float32, device=DEV)
+            ref2 = O.mv_sparse_step(g2.numpy(), np.zeros((N, d), dtype=np.float32), K2)
+            ctx.mv_vote(g2.to(DEV), acc2, None, bits_, votes, None, K=K2)
+            ctx.mv_select(votes, N, idx2, None, K=K2)
+            ctx.mv_aggregate(acc2, idx2, val2)
+            torch.cuda.synchronize()
+            PT.first_diff(PT.npy(votes), ref2["votes"], f"step {step} phases votes")
+            PT.first_diff(PT.npy(idx2), ref2["out_idx"], f"step {step} phases out_idx")
+            PT.first_diff(PT.bits(PT.npy(acc2)), PT.bits(ref2["err"]), f"step {step} phases err")
+
+
 def test_checkpoint_resume():
     """The residual is the only state: saving and restoring it mid-run changes nothing."""
     w = WL.scaled(WL.resnet_like("c3"), d=50021, N=5, steps=6)
