@@ -229,6 +229,49 @@ def run_reference(args, w: WL.Workload):
     print(json.dumps(line), flush=True)
 
 
+def run_sweep(args):
+    """The sweep of the configuration list: N in {4,16,64} x d in {2^20,2^24,2^27} x K/d in {1e-2,1e-3,2.5e-4},
+    gradients with cross-worker correlation 0.3, residuals ~ N(0, 0.01^2).  Per cell: 3 warm-up steps, then
+    `reps` single steps, each from the same saved residual (the restore is outside the timed region), the
+    threshold sampled in every step (stateless mode); the median is reported.  One GPU."""
+    from paper_2011_06495_b200 import binding as B
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    peak, peak_kind = measured_peak()
+    reps = 10
+    for w in WL.sweep_cells():
+        grads = WL.gradients(w, 0, device=dev)
+        err0 = WL.initial_err(w, device=dev)
+        err = torch.empty_like(err0)
+        out_idx = torch.empty(w.K, dtype=torch.int32, device=dev)
+        out_val = torch.empty(w.K, dtype=torch.float32, device=dev)
+        ctx = B.MvContext(w.N, w.d, w.K, device=dev, mode=B.MV_MODE_AUTO)
+        times = []
+        for it in range(3 + reps):
+            err.copy_(err0)
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ev0.record()
+            ctx.mv_sparse_step(grads, err, out_idx, out_val)
+            ev1.record()
+            torch.cuda.synchronize()
+            if it >= 3:
+                times.append(ev0.elapsed_time(ev1))
+        ms = float(np.median(times))
+        nbytes = w.N * w.d * 4
+        line = {"metric": METRIC, "value": 1000.0 / ms, "unit": UNIT, "ms_per_step": ms, "ms_min": float(min(times)),
+                "config": {"workload": f"sweep cell N={w.N} d={w.d} K={w.K}", "N": w.N, "d": w.d, "K": w.K,
+                           "l2": "inputs larger than L2" if 2 * nbytes > L2_BYTES else "inputs fit in L2"},
+                "effective_gradient_gbs": nbytes / ms / 1e6, "step_roofline_frac": 3 * nbytes / ms / 1e6 / peak,
+                "peak": peak, "peak_kind": "of " + peak_kind, "launches_per_step": ctx.last_launches(),
+                "fallback_workers": int((ctx.read_diag(w.N)[:, 2] != 0).sum()), "repeats": reps, "dtype": "f32", "data": "synthetic"}
+        print(json.dumps(line), flush=True)
+        ctx.close()
+        del grads, err0, err, out_idx, out_val, ctx
+        torch.cuda.empty_cache()
+
+
 def max_over_ranks(value: float, dist, device) -> float:
     """Largest value over all ranks (the job is as slow as its slowest replica)."""
     t = torch.tensor([value], dtype=torch.float64, device=device)
@@ -264,7 +307,13 @@ def main():
                          "rs: random selection proportional to the votes (Algorithm 1, second variant)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--sweep", action="store_true",
+                    help="instead of the one bench line: time the 27 cells of the sweep (N x d x K/d), one JSON line per "
+                         "cell, a single step timed after warm-up with the residual restored before every repeat")
     args = ap.parse_args()
+    if args.sweep:
+        run_sweep(args)
+        return
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     w = WL.resnet_like(args.workload)

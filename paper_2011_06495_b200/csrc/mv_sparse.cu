@@ -1240,7 +1240,7 @@ __device__ __forceinline__ void cluster_row_keys(const P& p, int n, float* __res
 }
 
 template <int CL>
-__global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(ST, 1) k_select_cluster(P p, float* __restrict__ err, int zero_first) {
+__global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(ST, 1) k_select_cluster(P p, float* __restrict__ err, int zero_first, int n_select) {
   pdl_enter();
   cg::cluster_group cluster = cg::this_cluster();
   extern __shared__ uint32_t s_keys[];       // [SK_KEYS]
@@ -1263,7 +1263,7 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(ST, 1) k_select_clu
       if (p.vote_words != nullptr) zero_share(p.vote_words, (size_t)p.nchunks * (CH / 4), bid, nblocks);
     }
   }
-  if ((int)blockIdx.y >= p.N) return;  // alike in every CTA of the cluster
+  if ((int)blockIdx.y >= n_select) return;  // alike in every CTA of the cluster (n_select: workers selected here)
   const int n = blockIdx.y;
   const uint32_t rank = cluster.block_rank();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -2481,15 +2481,30 @@ int vote_impl(mv_ctx* ctx, P p, const Layout& L, const float* grads, float* err,
     if (!cluster_select_ready()) return MV_ERR_CUDA;
     // a cluster per worker resolves T_n, sets the worker's mask bits and adds its votes
     // (with few workers, extra clusters that only help clearing fill the GPU)
-    const int cl = N * 8 <= 144 ? 8 : 4;                    // one CTA per SM: keep all clusters resident if possible
-    const int zc = N * cl < 144 ? (144 - N * cl) / cl : 0;  // clusters that only clear
+    // (candidate buffers of more than 2^20 entries per worker are more than a cluster's 4 or 8 SMs
+    // should walk, above all when the workers are few: those go through the grid-wide select kernels
+    // and the clusters only clear)
+    const bool wide = p.cap > (1u << 20);
+    const int nsel = wide ? 0 : N;
+    const int cl = nsel * 8 <= 144 ? 8 : 4;                       // one CTA per SM: keep all clusters resident if possible
+    const int zc = nsel * cl < 144 ? (144 - nsel * cl) / cl : 0;  // clusters that only clear
     // the extra clusters clear alone if that does not take them longer than the select takes (measured:
     // about 450 KB per CTA); otherwise every CTA of the grid clears a share first
     const size_t clear_bytes = (size_t)N * (size_t)p.W * 4 + (topk_only ? 0 : (size_t)p.nchunks * CH);
-    const int zero_first = (zc * cl >= 32 && clear_bytes / (size_t)(zc * cl) <= 450 * 1024) ? N : 0;
-    if (cl == 8) launch_smem(k_select_cluster<8>, dim3(dim3(8, N + zc)), dim3(ST), SK_KEYS * 4, st, p, err, zero_first);
-    else launch_smem(k_select_cluster<4>, dim3(dim3(4, N + zc)), dim3(ST), SK_KEYS * 4, st, p, err, zero_first);
+    const int zero_first = (nsel > 0 && zc * cl >= 32 && clear_bytes / (size_t)(zc * cl) <= 450 * 1024) ? nsel : 0;
+    if (cl == 8) launch_smem(k_select_cluster<8>, dim3(dim3(8, nsel + zc)), dim3(ST), SK_KEYS * 4, st, p, err, zero_first, nsel);
+    else launch_smem(k_select_cluster<4>, dim3(dim3(4, nsel + zc)), dim3(ST), SK_KEYS * 4, st, p, err, zero_first, nsel);
     MV_LAUNCH_CHECK();
+    if (wide) {
+      launch_k(k_hist<1, false>, dim3(dim3(gh, N)), dim3(TPB), st, p, nullptr, err);
+      MV_LAUNCH_CHECK();
+      launch_k(k_hist<2, false>, dim3(dim3(gh, N)), dim3(TPB), st, p, nullptr, err);
+      MV_LAUNCH_CHECK();
+      launch_k(k_hist<3, false>, dim3(dim3(gh, N)), dim3(TPB), st, p, nullptr, err);
+      MV_LAUNCH_CHECK();
+      launch_k(k_count, dim3(dim3(gh, N)), dim3(TPB), st, p, err);
+      MV_LAUNCH_CHECK();
+    }
     // the picks: mask bits and votes, from the candidates (or the row), by the whole GPU
     launch_k(k_set_bits, dim3(dim3(per_row_ctas(N, (int)((p.cap + TPB * 16 - 1) / (TPB * 16)), 148 * 4), N)), dim3(TPB), st, p,
              err);

@@ -259,7 +259,8 @@ def test_error_feedback_over_steps():
         err_ref = ref["err"]
 
 
-@pytest.mark.parametrize("N,d,K", [(6, 200003, 2000), (3, 1000003, 250), (4, 50000, 5000), (2, 4097, 7)])
+@pytest.mark.parametrize("N,d,K", [(6, 200003, 2000), (3, 1000003, 250), (4, 50000, 5000), (2, 4097, 7),
+                                   (2, (1 << 21) + 3, 300_000)])   # the last: candidate buffers beyond 2^20 entries
 def test_threshold_tracking_over_steps(N, d, K):
     """MV_MODE_TRACK: after the first call the candidate threshold comes from the previous call's key
     histogram (one kernel fewer); every step stays bit-identical to the oracle, and on slowly
