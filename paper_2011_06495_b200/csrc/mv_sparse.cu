@@ -23,10 +23,10 @@
 // With threshold tracking the sample is skipped after the first call: while a call resolves its
 // K-th key, the same counts locate a slightly larger rank, and that key is the next call's tau_n.
 // MV_MODE_GENERAL (no sampling) fuses a full radix histogram into the first pass instead and uses the
-// grid-wide select kernels k_hist<1..3>, k_count, k_set_bits and the bit-sliced vote count k_votes;
-// the same select kernels serve the variants in "list mode" over explicit (key, index) lists:
-// add-drop voting (k_ad_fill, k_ad_apply; Algorithm 2) and random selection proportional to the
-// votes (k_rs_fill; Algorithm 1, second variant).  A rank that holds only some of the workers gets
+// grid-wide select kernels k_hist<1..3>, k_count, k_set_bits and the bit-sliced vote count k_votes.
+// The variants select in "list mode" over explicit (key, index) lists: add-drop voting (k_ad_fill,
+// a cluster per list, k_ad_apply; Algorithm 2) and random selection proportional to the votes
+// (k_rs_fill, the grid-wide select kernels over its one long list; Algorithm 1, second variant).  A rank that holds only some of the workers gets
 // binary64 partial sums from k_gather and finishes with k_finish_mean.
 //
 // The magnitude order is the order of key(x) = bits(x) & 0x7fffffff; ties go to the lowest index.
@@ -1269,9 +1269,10 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(ST, 1) k_select_clu
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   for (int b = tid; b < 3 * H1_BINS; b += ST) (&s_h[0][0])[b] = 0;
   __syncthreads();
-  const uint32_t K = (uint32_t)p.K;
   const uint32_t cnt = p.cand_cnt[n];
-  const bool fast = cnt >= K && cnt <= p.cap;  // alike in every CTA of the cluster
+  const bool fast = worker_fast(p, n);  // alike in every CTA of the cluster
+  if (p.list_mode && !fast) return;     // an empty list (or one that overflowed its room) selects nothing
+  const uint32_t K = worker_K(p, n);    // list mode: min(K, length of the list)
   const bool tracking = p.tau_next != nullptr;
   const uint2* cd = p.cand + (size_t)n * p.cap;
   // this CTA's slice of the candidate buffer
@@ -1282,7 +1283,7 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(ST, 1) k_select_clu
   // ---- the usual case: the K-th key lies in a window of 2^22 keys above tau_n ----
   uint32_t T = 0, need = 0, cnt_eq = 0;
   bool resolved = false;  // alike in every CTA of the cluster
-  if (fast) {
+  if (fast && !p.list_mode) {  // (a list has no threshold bound: its keys go straight to the three digits)
     const uint32_t tau = p.tau[n];
     uint32_t wsum = 0;
     for (int b = tid; b < H1_BINS; b += ST) s_hw[b] = 0;
@@ -2869,14 +2870,22 @@ int mv_ad_step(mv_ctx* ctx, const float* grads, float* err, uint32_t* prev_bits,
            (const uint32_t*)prev_bits, (const float*)err);
   MV_LAUNCH_CHECK();
   const int ga = per_row_ctas(2 * N, (int)((a.cap + TPB * 8 - 1) / (TPB * 8)), 148 * 2);
-  launch_k(k_hist<1, false>, dim3(dim3(ga, 2 * N)), dim3(TPB), st, a, nullptr, err);
-  MV_LAUNCH_CHECK();
-  launch_k(k_hist<2, false>, dim3(dim3(ga, 2 * N)), dim3(TPB), st, a, nullptr, err);
-  MV_LAUNCH_CHECK();
-  launch_k(k_hist<3, false>, dim3(dim3(ga, 2 * N)), dim3(TPB), st, a, nullptr, err);
-  MV_LAUNCH_CHECK();
-  launch_k(k_count, dim3(dim3(ga, 2 * N)), dim3(TPB), st, a, err);
-  MV_LAUNCH_CHECK();
+  if (a.cap <= (1u << 20) && cluster_select_ready()) {
+    // a cluster per list finds the key of its K_ad-th entry (three radix digits; nothing is cleared here)
+    const int rows = 2 * N;
+    if (rows * 8 <= 144) launch_smem(k_select_cluster<8>, dim3(dim3(8, rows)), dim3(ST), SK_KEYS * 4, st, a, err, rows, rows);
+    else launch_smem(k_select_cluster<4>, dim3(dim3(4, rows)), dim3(ST), SK_KEYS * 4, st, a, err, rows, rows);
+    MV_LAUNCH_CHECK();
+  } else {
+    launch_k(k_hist<1, false>, dim3(dim3(ga, 2 * N)), dim3(TPB), st, a, nullptr, err);
+    MV_LAUNCH_CHECK();
+    launch_k(k_hist<2, false>, dim3(dim3(ga, 2 * N)), dim3(TPB), st, a, nullptr, err);
+    MV_LAUNCH_CHECK();
+    launch_k(k_hist<3, false>, dim3(dim3(ga, 2 * N)), dim3(TPB), st, a, nullptr, err);
+    MV_LAUNCH_CHECK();
+    launch_k(k_count, dim3(dim3(ga, 2 * N)), dim3(TPB), st, a, err);
+    MV_LAUNCH_CHECK();
+  }
   launch_k(k_set_bits, dim3(dim3(ga, 2 * N)), dim3(TPB), st, a, err);
   MV_LAUNCH_CHECK();
   if (!direct) {
