@@ -2423,7 +2423,9 @@ int join_side(mv_ctx* ctx) {
 // steps a1-a3: accumulate, per-worker top-K, votes
 // `topk_only`: stop once the workers' bit masks are set (no vote count, no index lists); everything
 // then stays on the caller's stream
-int vote_impl(mv_ctx* ctx, P p, const Layout& L, const float* grads, float* err, bool topk_only = false) {
+// `need_hist` = false: the per-chunk vote histograms and offsets are not wanted (the caller selects by other means)
+int vote_impl(mv_ctx* ctx, P p, const Layout& L, const float* grads, float* err, bool topk_only = false,
+              bool need_hist = true) {
   cudaStream_t st = ctx->stream;
   const int N = p.N;
   ctx->timing_now = ctx->timing > 0 && (ctx->timing_calls++ % ctx->timing) == 0;
@@ -2512,9 +2514,11 @@ int vote_impl(mv_ctx* ctx, P p, const Layout& L, const float* grads, float* err,
     MV_LAUNCH_CHECK();
     if (topk_only) return MV_OK;
     // vote histograms per chunk, v* and the output offsets (the caller's vote array gets its copy here)
-    launch_k(k_vote_hist, dim3((p.nchunks + VH_WARPS - 1) / VH_WARPS), dim3(TPB), st, p, (const uint8_t*)ws_votes,
-             p.votes != ws_votes ? p.votes : (uint8_t*)nullptr);
-    MV_LAUNCH_CHECK();
+    if (need_hist || p.votes != ws_votes) {
+      launch_k(k_vote_hist, dim3((p.nchunks + VH_WARPS - 1) / VH_WARPS), dim3(TPB), st, p, (const uint8_t*)ws_votes,
+               p.votes != ws_votes ? p.votes : (uint8_t*)nullptr);
+      MV_LAUNCH_CHECK();
+    }
   } else {
     if (ctx->timing_now) cudaEventRecord(ctx->ev[2 * (ctx->timed % 64)], st);
     launch_k(k_hist<1, true>, dim3(dim3(gh, N)), dim3(TPB), st, p, grads, err);
@@ -3023,10 +3027,9 @@ int mv_rs_step(mv_ctx* ctx, const float* grads, float* err, int N, int64_t d, in
   ctx->last_N = N;
   ctx->last_d = d;
   ctx->last_K = K;
-  rc = vote_impl(ctx, p, L, grads, err);
+  rc = vote_impl(ctx, p, L, grads, err, false, false);  // the random selection reads the votes themselves
   // the union of N top-K sets holds at least K coordinates, so the mask is always full
   if (rc == MV_OK) rc = rs_select_impl(ctx, p, L, p.votes, seed, draw, out_idx, nullptr);
-  // the vote count's own scan is not consumed here: the gather clears its state with the rest
   if (rc == MV_OK) rc = aggregate_impl(ctx, err, N, d, K, out_idx, out_val, L.zero_bytes);
   const int rcj = join_side(ctx);
   return rc != MV_OK ? rc : rcj;
