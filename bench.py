@@ -6,7 +6,10 @@
 A step is one whole pass of the hot path (error feedback, per-worker top-K, vote count, shared
 mask, aggregate, residual) over one batch of synthetic gradients; the residual is carried from
 step to step and every step gets fresh gradients from a pool that was generated before the timed
-region.  One JSON line is printed by rank 0.  With --gpus N > 1 (launched through torchrun) every
+region.  Before the warm-up the residuals are carried through 300 untimed steps, so that the timed
+steps are those of a run in progress (every chunk of every worker holds candidates) and not of its
+first iterations.  One JSON line is printed by rank 0; with the default workload it also carries the
+other two ResNet-scale configurations under "also".  With --gpus N > 1 (launched through torchrun) every
 rank runs an independent replica of the same workload: the path does not shard across devices.
 """
 from __future__ import annotations
@@ -34,7 +37,6 @@ RS_SEED = 201106495
 METRIC = "majority-vote sparse steps/s"
 UNIT = "steps/s"
 FALLBACK_HBM_GBS = 6650.0
-L2_BYTES = 126 * 1024 * 1024
 
 
 def measured_peak():
@@ -84,7 +86,7 @@ def recorded_traffic(workload: str, n_units: int):
         rec = json.load(open(path))
         if rec.get("source_sha256_16") != kernel_source_hash():
             return None
-        if n_units * 4 <= L2_BYTES:          # an L2-resident case moves other bytes than a streaming one
+        if n_units * 4 <= l2_bytes():        # an L2-resident case moves other bytes than a streaming one
             return None
         # captured on c2; the streaming pass moves the same bytes per element on any input larger than L2
         return float(rec["dram_bytes_per_element"]) * n_units
@@ -175,54 +177,61 @@ def host_cores() -> int:
         return os.cpu_count() or 1
 
 
-def oracle_steps_per_s(w: WL.Workload, steps: int, sample_workers: int, warmup: int = 0, method: str = "mv"):
-    """Times the CPU oracle as it stands on a bounded sample: the first `sample_workers` rows of
-    the workload, full d and K (a majority-vote step among those workers).  Returns
-    (steps/s of the sample, seconds per step, description)."""
+def oracle_run(w: WL.Workload, steps: int, warmup: int, threads: int, method: str = "mv"):
+    """Times the CPU oracle as it stands on the whole workload (all N workers, full d and K): `warmup`
+    untimed steps, then `steps` timed ones, the residual carried.  `threads` host threads work on
+    different workers' rows at the same time (the oracle's own option; its arithmetic is the same).
+    Returns (seconds per step, steps timed)."""
     from oracle import mv_oracle as O
-    ws = WL.Workload(w.name, N=sample_workers, d=w.d, K=w.K, steps=w.steps, kind=w.kind, config_id=w.config_id,
-                     segments=w.segments, std_lo=w.std_lo, std_hi=w.std_hi, rho=w.rho, err0_std=w.err0_std,
-                     round_decimals=w.round_decimals)
-    err = WL.initial_err(ws).numpy()
-    prev = np.zeros((ws.N, ws.d), dtype=bool)
+    err = WL.initial_err(w).numpy()
+    prev = np.zeros((w.N, w.d), dtype=bool)
     times = []
     for s in range(warmup + steps):
-        g = WL.gradients(ws, s).numpy()
+        g = WL.gradients(w, s).numpy()
         t0 = time.perf_counter()
         if method == "ad":
-            r = O.mv_ad_step(g, err, prev, ws.K, max(1, ws.K // 10))
+            r = O.mv_ad_step(g, err, prev, w.K, max(1, w.K // 10))
             prev = r["prev"]
         elif method == "rs":
             from oracle import rs_oracle as R
-            r = R.mv_rs_step(g, err, ws.K, RS_SEED, s)
+            r = R.mv_rs_step(g, err, w.K, RS_SEED, s)
         else:
-            r = O.mv_sparse_step(g, err, ws.K)
+            r = O.mv_sparse_step(g, err, w.K, threads=threads)
         dt = time.perf_counter() - t0
         err = r["err"]
         if s >= warmup:
             times.append(dt)
-    per_step = float(np.mean(times))
-    # the oracle's cost is linear in the number of workers (each row is selected on its own)
-    full_step = per_step * (w.N / sample_workers)
-    desc = (f"{sample_workers} of {w.N} workers, full d={w.d} and K={w.K}, {steps} step(s); "
-            f"scaled by {w.N}/{sample_workers} to the whole step")
-    return 1.0 / full_step, full_step, desc
+    return float(np.mean(times)), len(times)
+
+
+def oracle_budget_steps(w: WL.Workload, asked: int, seconds: float) -> int:
+    """How many whole steps of the oracle fit a budget of `seconds`, by its cost of roughly 10 ns per
+    element and thread plus the generation of the inputs; at least 1, at most `asked`."""
+    per_step = 25e-9 * w.N * w.d + 0.05
+    return int(max(1, min(asked, seconds // per_step)))
 
 
 def run_reference(args, w: WL.Workload):
-    """The reference arm: the CPU oracle on the host cores (rank 0 only)."""
+    """The reference arm: the CPU oracle on the host cores (rank 0 only), whole steps of the whole
+    workload.  `steps` and `warmup` in the line are the ones that ran."""
     if int(os.environ.get("RANK", "0")) != 0:
         return
-    torch.set_num_threads(max(1, host_cores()))
-    sample_workers = min(w.N, 2 if w.d > 1_000_000 else w.N)
-    steps = max(1, min(args.steps, 3))
-    sps, sec, desc = oracle_steps_per_s(w, steps, sample_workers, warmup=min(args.warmup, 1), method=args.method)
+    cores = host_cores()
+    threads = max(1, min(cores, w.N)) if args.method == "mv" else 1
+    steps = oracle_budget_steps(w, args.steps, 90.0)
+    warmup = 1 if args.warmup >= 1 else 0
+    sec, ran = oracle_run(w, steps, warmup, threads, method=args.method)
+    sps = 1.0 / sec
+    sample = (f"whole workload: all {w.N} workers, d={w.d}, K={w.K}; {ran} consecutive step(s) timed after {warmup} "
+              f"untimed, residual carried; {threads} host thread(s) over the workers' rows")
     line = {
-        "impl": "reference", "metric": METRIC, "value": sps, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+        "impl": "reference", "metric": METRIC, "value": sps, "unit": UNIT, "n_gpus": args.gpus, "steps": ran,
+        "warmup": warmup, "steps_asked": args.steps, "warmup_asked": args.warmup,
+        "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": workload_config(w),
-        "cpu_baseline": {"value": sps, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
+        "cpu_baseline": {"value": sps, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample,
+                         "host_cores_available": cores},
         "e2e": {"value": sps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -262,7 +271,7 @@ def run_sweep(args):
         nbytes = w.N * w.d * 4
         line = {"metric": METRIC, "value": 1000.0 / ms, "unit": UNIT, "ms_per_step": ms, "ms_min": float(min(times)),
                 "config": {"workload": f"sweep cell N={w.N} d={w.d} K={w.K}", "N": w.N, "d": w.d, "K": w.K,
-                           "l2": "inputs larger than L2" if 2 * nbytes > L2_BYTES else "inputs fit in L2"},
+                           "l2": "inputs larger than L2" if 2 * nbytes > l2_bytes() else "inputs fit in L2"},
                 "effective_gradient_gbs": nbytes / ms / 1e6, "step_roofline_frac": 3 * nbytes / ms / 1e6 / peak,
                 "peak": peak, "peak_kind": "of " + peak_kind, "launches_per_step": ctx.last_launches(),
                 "fallback_workers": int((ctx.read_diag(w.N)[:, 2] != 0).sum()), "repeats": reps, "dtype": "f32", "data": "synthetic"}
@@ -285,11 +294,162 @@ def job_steps_per_s(ms_total_max: float, world: int, steps: int) -> float:
     return world * steps / (ms_total_max * 1e-3)
 
 
+def l2_bytes() -> int:
+    """L2 capacity of the current CUDA device (what decides whether a workload streams from HBM)."""
+    if torch.cuda.is_available():
+        return int(torch.cuda.get_device_properties(torch.cuda.current_device()).L2_cache_size)
+    return 126 * 1024 * 1024      # no device to ask (the reference arm on a host without one): B200's data-sheet size
+
+
 def workload_config(w: WL.Workload):
+    nbytes = w.N * w.d * 4
     return {"workload": f"{w.name}: N={w.N} workers, d={w.d} fp32, K={w.K} ({w.note}), error feedback carried, "
                         f"fresh gradients every step",
-            "N": w.N, "d": w.d, "K": w.K, "l2": "inputs larger than L2" if w.N * w.d * 4 > L2_BYTES else "L2-resident",
+            "N": w.N, "d": w.d, "K": w.K,
+            "l2": "inputs larger than L2" if nbytes > l2_bytes() else "L2-resident",
             "parallelism": "replicas only"}
+
+
+PREHEAT_STEPS = 300      # untimed steps that carry the residuals into the error-feedback steady state
+POOL_BYTES = 32e9        # gradient tensors generated before the timed region (cycled if the run is longer)
+NOMINAL_HBM_GBS = 7700.0
+
+
+def measure(w: WL.Workload, args, B, dev, dist, world, local_rank, with_e2e: bool):
+    """Runs one workload: inputs resident in HBM, `preheat` untimed steps on fresh gradients so that the
+    residuals are those of a run in progress, `--warmup` untimed steps, `--steps` timed ones (CUDA events
+    on the launching stream, barrier and synchronize on both sides, max over ranks).  Returns the fields
+    of the JSON line that depend on the workload."""
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    nbytes = w.N * w.d * 4
+    pool_n = int(max(2, min(args.steps + args.warmup, POOL_BYTES // nbytes, 64)))
+    std = WL.std_vector(w, dev) if w.segments > 1 else None
+    err = WL.initial_err(w, device=dev)
+    out_idx = torch.empty(w.K, dtype=torch.int32, device=dev)
+    out_val = torch.empty(w.K, dtype=torch.float32, device=dev)
+    mode = {"auto": B.MV_MODE_AUTO, "general": B.MV_MODE_GENERAL, "track": B.MV_MODE_TRACK}[args.mode]
+    ctx = B.MvContext(w.N, w.d, w.K, device=dev, mode=mode)
+
+    if args.method == "ad":
+        K_ad = max(1, w.K // 10)
+        prev_bits = torch.zeros((w.N, (w.d + 31) // 32), dtype=torch.int32, device=dev)
+
+        def one_step(g):
+            ctx.mv_ad_step(g, err, prev_bits, K_ad, out_idx, out_val)
+    elif args.method == "rs":
+        draw = [0]
+
+        def one_step(g):
+            ctx.mv_rs_step(g, err, RS_SEED, draw[0], out_idx, out_val)
+            draw[0] += 1
+    else:
+        def one_step(g):
+            ctx.mv_sparse_step(g, err, out_idx, out_val)
+
+    # ---- the state of a run in progress: residuals built up over `preheat` steps of fresh gradients
+    preheat = args.preheat if args.preheat >= 0 else (PREHEAT_STEPS if w.steps > 1 else 0)
+    scratch = torch.empty((w.N, w.d), dtype=torch.float32, device=dev)
+    for s in range(preheat):
+        one_step(WL.gradients(w, 100_000 + s, out=scratch, std=std))
+    torch.cuda.synchronize()
+    del scratch
+    # ---- inputs resident in HBM before the timed region: gradient tensors not seen so far
+    pool = [WL.gradients(w, s, device=dev, std=std) for s in range(pool_n)]
+
+    sampler = ClockSampler(visible_gpu_index(local_rank))
+    sampler.start()
+    step_no = 0
+    for _ in range(args.warmup):
+        one_step(pool[step_no % pool_n])
+        step_no += 1
+    # CUDA events around the streaming kernel on one step in eight (each pair costs a few microseconds)
+    ctx.set_kernel_timing(8 if args.steps >= 8 else 1)
+    fb_before = ctx.fallback_count()
+    sampler.wait_for_first_sample()
+    barrier()
+    first_row = sampler.rows_so_far()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(args.steps):
+        one_step(pool[step_no % pool_n])
+        step_no += 1
+    ev1.record()
+    barrier()
+    time.sleep(0.03)
+    clocks = sampler.stop(first_row)
+    ms_total = ev0.elapsed_time(ev1)
+    launches_per_step = ctx.last_launches()
+    k_ms, k_cnt = ctx.read_kernel_timing()
+    ctx.set_kernel_timing(0)
+    fallbacks = ctx.fallback_count() - fb_before
+    diag = ctx.read_diag(w.N)
+    ms_total = max_over_ranks(ms_total, dist, dev)
+    ms_step = ms_total / args.steps
+
+    # ---- end to end through the host entry point: gradients start in pinned host memory
+    e2e = None
+    if with_e2e:
+        h_pool = [pool[i].cpu().pin_memory() for i in range(2)]
+        h_idx = torch.empty(w.K, dtype=torch.int32).pin_memory()
+        h_val = torch.empty(w.K, dtype=torch.float32).pin_memory()
+        d_grads = pool[-1]
+        e_steps = max(3, min(args.steps, 10))
+        for i in range(2):
+            ctx.mv_sparse_step_host(h_pool[i % 2], h_idx, h_val, d_grads, err, out_idx, out_val)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(e_steps):
+            ctx.mv_sparse_step_host(h_pool[i % 2], h_idx, h_val, d_grads, err, out_idx, out_val)
+        e1.record()
+        barrier()
+        te = max_over_ranks(e0.elapsed_time(e1), dist, dev)
+        e2e = {"value": job_steps_per_s(te, world, e_steps), "unit": UNIT,
+               "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": 8 * w.K, "steps": e_steps,
+               "note": "mv_sparse_step_host: gradients copied from pinned host memory every step, indices and "
+                       "values copied back; the residual stays on the device"}
+        del h_pool
+
+    peak, peak_kind = measured_peak()
+    alg_bytes = 12.0 * w.N * w.d                      # read grads, read err, write acc: 12 B per element
+    k_ms_avg = k_ms / max(k_cnt, 1)
+    achieved = alg_bytes / (k_ms_avg * 1e-3) / 1e9 if k_cnt else None
+    step_gbs = alg_bytes / (ms_step * 1e-3) / 1e9
+    frac = (achieved / peak) if achieved else None
+    roofline = {"bound": "hbm", "kernel": "k_acc_compact" if args.mode != "general" else "k_hist<1,true>",
+                "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                "frac": frac, "traffic": recorded_traffic(w.name, w.N * w.d),
+                "kernel_ms": k_ms_avg, "kernel_launches_timed": k_cnt, "algorithmic_bytes_per_launch": alg_bytes,
+                "peak_nominal": NOMINAL_HBM_GBS, "frac_of_nominal": (achieved / NOMINAL_HBM_GBS) if achieved else None}
+    if frac is not None and frac > 1.0:
+        roofline["note"] = ("above 1: the peak is the bandwidth of a plain device copy, which this kernel outruns; "
+                            "frac_of_nominal is the fraction of the HBM3e data-sheet figure")
+    out = {
+        "value": job_steps_per_s(ms_total, world, args.steps), "ms_per_step": ms_step,
+        "config": workload_config(w),
+        "setup": dict(method={"ad": "add-drop voting, K_ad=K/10", "rs": "random selection proportional to the votes",
+                              "mv": "majority voting"}[args.method],
+                      threshold={"track": "candidate threshold carried from the previous step's key histogram",
+                                 "auto": "candidate threshold sampled every step",
+                                 "general": "no candidate threshold (multi-pass select)"}[args.mode],
+                      preheat_steps=preheat, gradient_pool=pool_n),
+        "effective_gradient_gbs": w.N * w.d * 4 / (ms_step * 1e-3) / 1e9,
+        "step_roofline_frac": step_gbs / peak, "step_roofline_frac_of_nominal": step_gbs / NOMINAL_HBM_GBS,
+        "roofline": roofline, "clocks": clocks,
+        "gpu_launches": launches_per_step * args.steps, "launches_per_step": launches_per_step,
+        "fallback_workers": int(fallbacks),
+        "candidates_over_K_last_step": float(diag[:, 0].double().mean() / w.K),
+    }
+    if e2e is not None:
+        out["e2e"] = e2e
+    ctx.close()
+    del pool, err, ctx
+    torch.cuda.empty_cache()
+    return out
 
 
 def main():
@@ -305,8 +465,14 @@ def main():
     ap.add_argument("--method", default="mv", choices=["mv", "ad", "rs"],
                     help="mv: plain majority voting (Algorithm 1); ad: add-drop voting (Algorithm 2) with K_ad = K/10; "
                          "rs: random selection proportional to the votes (Algorithm 1, second variant)")
+    ap.add_argument("--preheat", type=int, default=-1,
+                    help="untimed steps on fresh gradients before warm-up, so that the timed steps see the residuals of a "
+                         f"run in progress (default: {PREHEAT_STEPS} for the multi-step workloads, 0 for c1)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-also", action="store_true",
+                    help="with the default workload c2 the line also carries c3 and c4 (the other two ResNet-scale "
+                         "configurations) under \"also\"; this switches that off")
     ap.add_argument("--sweep", action="store_true",
                     help="instead of the one bench line: time the 27 cells of the sweep (N x d x K/d), one JSON line per "
                          "cell, a single step timed after warm-up with the residual restored before every repeat")
@@ -337,125 +503,48 @@ def main():
         dist = dist_mod
         dist.init_process_group("nccl", device_id=dev)
 
-    def barrier():
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    # ---- inputs resident in HBM before the timed region: a pool of gradient tensors, cycled
-    nbytes = w.N * w.d * 4
-    pool_n = max(2, min(args.steps + args.warmup, int(8e9 // nbytes), 8))
-    std = WL.std_vector(w, dev) if w.segments > 1 else None
-    pool = [WL.gradients(w, s, device=dev, std=std) for s in range(pool_n)]
-    err = WL.initial_err(w, device=dev)
-    out_idx = torch.empty(w.K, dtype=torch.int32, device=dev)
-    out_val = torch.empty(w.K, dtype=torch.float32, device=dev)
-    ctx = B.MvContext(w.N, w.d, w.K, device=dev, mode={"auto": B.MV_MODE_AUTO, "general": B.MV_MODE_GENERAL, "track": B.MV_MODE_TRACK}[args.mode])
-
-    sampler = ClockSampler(visible_gpu_index(local_rank))
-    sampler.start()
-    if args.method == "ad":
-        K_ad = max(1, w.K // 10)
-        prev_bits = torch.zeros((w.N, (w.d + 31) // 32), dtype=torch.int32, device=dev)
-
-        def one_step(g):
-            ctx.mv_ad_step(g, err, prev_bits, K_ad, out_idx, out_val)
-    elif args.method == "rs":
-        draw = [0]
-
-        def one_step(g):
-            ctx.mv_rs_step(g, err, RS_SEED, draw[0], out_idx, out_val)
-            draw[0] += 1
-    else:
-        def one_step(g):
-            ctx.mv_sparse_step(g, err, out_idx, out_val)
-
-    step_no = 0
-    for _ in range(args.warmup):
-        one_step(pool[step_no % pool_n])
-        step_no += 1
-    # CUDA events around the streaming kernel on one step in eight (each pair costs a few microseconds)
-    ctx.set_kernel_timing(8 if args.steps >= 8 else 1)
-    sampler.wait_for_first_sample()
-    barrier()
-    first_row = sampler.rows_so_far()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ev0.record()
-    for _ in range(args.steps):
-        one_step(pool[step_no % pool_n])
-        step_no += 1
-    ev1.record()
-    barrier()
-    time.sleep(0.03)
-    clocks = sampler.stop(first_row)
-    ms_total = ev0.elapsed_time(ev1)
-    launches_per_step = ctx.last_launches()
-    k_ms, k_cnt = ctx.read_kernel_timing()
-    ctx.set_kernel_timing(0)
-    diag = ctx.read_diag(w.N)
-    ms_total = max_over_ranks(ms_total, dist, dev)
-    ms_step = ms_total / args.steps
-    value = job_steps_per_s(ms_total, world, args.steps)
-
-    # ---- end to end through the host entry point: gradients start in pinned host memory
-    e2e = None
-    if not args.no_e2e and args.method == "mv":
-        h_pool = [pool[i].cpu().pin_memory() for i in range(2)]
-        h_idx = torch.empty(w.K, dtype=torch.int32).pin_memory()
-        h_val = torch.empty(w.K, dtype=torch.float32).pin_memory()
-        d_grads = pool[-1]
-        e_steps = max(3, min(args.steps, 10))
-        for i in range(2):
-            ctx.mv_sparse_step_host(h_pool[i % 2], h_idx, h_val, d_grads, err, out_idx, out_val)
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for i in range(e_steps):
-            ctx.mv_sparse_step_host(h_pool[i % 2], h_idx, h_val, d_grads, err, out_idx, out_val)
-        e1.record()
-        barrier()
-        te = max_over_ranks(e0.elapsed_time(e1), dist, dev)
-        e2e = {"value": job_steps_per_s(te, world, e_steps), "unit": UNIT,
-               "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": 8 * w.K, "steps": e_steps,
-               "note": "mv_sparse_step_host: gradients copied from pinned host memory every step, indices and "
-                       "values copied back; the residual stays on the device"}
-        del h_pool
+    res = measure(w, args, B, dev, dist, world, local_rank, with_e2e=not args.no_e2e and args.method == "mv")
+    also = {}
+    if args.workload == "c2" and args.method == "mv" and not args.no_also:
+        # the other two ResNet-scale configurations, same process, same flags
+        for name in ("c3", "c4"):
+            r = measure(WL.resnet_like(name), args, B, dev, dist, world, local_rank, with_e2e=False)
+            also[name] = {"value": r["value"], "unit": UNIT, "ms_per_step": r["ms_per_step"],
+                          "step_roofline_frac": r["step_roofline_frac"],
+                          "step_roofline_frac_of_nominal": r["step_roofline_frac_of_nominal"],
+                          "effective_gradient_gbs": r["effective_gradient_gbs"],
+                          "roofline": {k: r["roofline"][k] for k in ("kernel", "achieved", "peak", "peak_kind", "frac", "frac_of_nominal", "kernel_ms")},
+                          "clocks": r["clocks"], "launches_per_step": r["launches_per_step"],
+                          "fallback_workers": r["fallback_workers"],
+                          "config": r["config"], "setup": r["setup"]}
 
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return
 
-    peak, peak_kind = measured_peak()
-    alg_bytes = 12.0 * w.N * w.d                      # read grads, read err, write acc: 12 B per element
-    k_ms_avg = k_ms / max(k_cnt, 1)
-    achieved = alg_bytes / (k_ms_avg * 1e-3) / 1e9 if k_cnt else None
-    traffic = recorded_traffic(w.name, w.N * w.d)
-    line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
-        "data": "synthetic", "config": dict(workload_config(w), method={"ad": "add-drop voting, K_ad=K/10", "rs": "random selection proportional to the votes",
-                                                  "mv": "majority voting"}[args.method],
-                                          threshold={"track": "candidate threshold carried from the previous step's key histogram",
-                                                     "auto": "candidate threshold sampled every step",
-                                                     "general": "no candidate threshold (multi-pass select)"}[args.mode]),
-        "effective_gradient_gbs": w.N * w.d * 4 / (ms_step * 1e-3) / 1e9 * 1.0,
-        "step_roofline_frac": alg_bytes / (ms_step * 1e-3) / 1e9 / peak,
-        "roofline": {"bound": "hbm", "kernel": "k_acc_compact" if args.mode != "general" else "k_row_hist<1,true>",
-                     "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
-                     "frac": (achieved / peak) if achieved else None, "traffic": traffic,
-                     "kernel_ms": k_ms_avg, "kernel_launches_timed": k_cnt, "algorithmic_bytes_per_launch": alg_bytes},
-        "clocks": clocks, "gpu_launches": launches_per_step * args.steps, "launches_per_step": launches_per_step,
-        "fallback_workers_last_step": int(diag[:, 2].sum()),
-        "candidates_over_K_last_step": float(diag[:, 0].double().mean() / w.K),
-    }
-    if e2e is not None:
-        line["e2e"] = e2e
+    line = {"metric": METRIC, "value": res.pop("value"), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": res.pop("ms_per_step"), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic"}
+    line.update(res)
+    if also:
+        line["also"] = also
     if world == 1 and not args.no_cpu_baseline:
-        sample_workers = min(w.N, 2 if w.d > 1_000_000 else w.N)
-        sps, sec, desc = oracle_steps_per_s(w, 1, sample_workers, method=args.method)
-        line["cpu_baseline"] = {"value": sps, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc,
-                                "host_cores_available": host_cores()}
+        # the oracle as it stands on this machine's host cores: whole steps of the whole workload, on one
+        # core and with its rows spread over the cores (a reported baseline, not a target)
+        cores = host_cores()
+        threads = max(1, min(cores, w.N)) if args.method == "mv" else 1
+        n1 = oracle_budget_steps(w, 3, 12.0)
+        sec1, ran1 = oracle_run(w, n1, 0, 1, method=args.method)
+        line["cpu_baseline"] = {
+            "value": 1.0 / sec1, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"whole workload: all {w.N} workers, d={w.d}, K={w.K}; {ran1} consecutive step(s) from zero "
+                      f"residuals, one host thread", "host_cores_available": cores}
+        if threads > 1:
+            secn, rann = oracle_run(w, oracle_budget_steps(w, 3, 12.0), 0, threads, method=args.method)
+            line["cpu_baseline"]["all_cores"] = {
+                "value": 1.0 / secn, "unit": UNIT, "cores": threads,
+                "sample": f"the same {rann} step(s) with {threads} host threads over the workers' rows"}
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()

@@ -58,7 +58,28 @@ enum {
                           its candidate threshold from that call's key histogram instead of sampling: meant
                           for the consecutive steps of one training run, where |acc| changes slowly.  Exact
                           for any input: a worker whose threshold turns out unusable (fewer than K or more
-                          than 4K + 4096 candidates) takes the multi-pass select for that call. */
+                          than 4K + 4096 candidates) takes the multi-pass select for that call.
+                          The carried thresholds belong to the context, not to a buffer: use one context
+                          per residual buffer (per training run).  A context that alternates between two
+                          residual buffers of the same shape stays exact but hands each the other's
+                          thresholds, and whenever those do not fit, the slow route is taken. */
+};
+
+/* Bits of the device status word of a checked build (see mv_debug_status).  The first three report a
+ * detour that leaves every result exact; the others report an index that was refused. */
+enum {
+  MV_DBG_CAND_OVERFLOW = 1,   /* streaming pass (S_top candidate filter): a worker had more candidates than its
+                                 buffer holds; the surplus was dropped and the worker takes the full-row select */
+  MV_DBG_WINDOW_OVERFLOW = 2, /* select (S_top, K-th key): the bin of the K-th key held more than 1024 keys; it was
+                                 resolved by the three-digit radix select instead */
+  MV_DBG_FALLBACK = 4,        /* select: a worker's K-th key was found over its full row (candidate count outside [K, cap]) */
+  MV_DBG_LIST_OVERFLOW = 8,   /* add-drop / random selection (Algorithm 2; Algorithm 1, S_rand line): a list outgrew its
+                                 room and was treated as empty */
+  MV_DBG_PICK_RANGE = 16,     /* picks (Eq. 9, inner sum): a candidate named a coordinate >= d and was skipped */
+  MV_DBG_LIST_RANGE = 32,     /* supp(M_n) lists: an entry beyond position K was not written */
+  MV_DBG_OUT_RANGE = 64,      /* supp(M) (Eq. 9, outer S_top): an entry beyond position K was not written */
+  MV_DBG_GATHER_RANGE = 128,  /* aggregate (Eq. 8): idx[k] outside [0, d); out_val[k] = 0 and the residual is untouched there */
+  MV_DBG_INTERNAL = 256       /* an index computed inside a kernel left its array and the access was skipped */
 };
 
 typedef struct mv_ctx mv_ctx;
@@ -92,7 +113,8 @@ int mv_sparse_step(mv_ctx* ctx, const float* grads, float* err, int N, int64_t d
  *   votes       [d] uint8       out     votes per coordinate                       (may be NULL)
  *   thresh      [N*3] uint32    out     per worker: K-th largest key T_n, number of keys above
  *                                       it, number of keys equal to it             (may be NULL)
- * Outputs passed as NULL are kept in the workspace. */
+ * An output passed as NULL is not delivered (the masks, votes and thresholds then live in the workspace
+ * only; the ascending lists are not built at all). */
 int mv_vote(mv_ctx* ctx, const float* grads, float* err, int N, int64_t d, int64_t K,
             int32_t* worker_idx, uint32_t* worker_bits, uint8_t* votes, uint32_t* thresh);
 
@@ -210,6 +232,12 @@ int mv_sparse_step_host(mv_ctx* ctx, const float* h_grads, int N, int64_t d, int
  *   lower bound on the threshold key, 1 if the exact multi-pass select was used, 0 (spare). */
 int mv_read_diag(mv_ctx* ctx, int N, uint32_t* per_worker);
 
+/* Running count, since the context's first call, of worker selections (one worker in one call) whose
+ * K-th key had to be found over the full row because the candidate threshold of the streaming pass
+ * admitted fewer than K or more than 4K + 4096 elements (S_top of Algorithm 1 stays exact either way;
+ * this is the slow route).  Counted on the device; the call waits for the stream.  total: host, out. */
+int mv_fallback_count(mv_ctx* ctx, uint32_t* total);
+
 /* Optional timing of the streaming pass (the kernel that reads grads and err and writes acc,
  * i.e. the accumulate line of Algorithm 1 fused with the candidate filter of S_top): with
  * every = n >= 1, each n-th mv_vote / mv_sparse_step records a CUDA-event pair around that one
@@ -234,6 +262,18 @@ int mv_read_phase_times(mv_ctx* ctx, float* ms, int capacity, int* count);
 
 /* Number of kernels the last call on this context enqueued. */
 int mv_last_launches(const mv_ctx* ctx);
+
+/* Checked build.  The library can be compiled with -DMV_DEBUG (paper_2011_06495_b200/build.py, debug=True,
+ * gives libmvsparse_debug.so): every place where a kernel clamps an index, drops an entry that does not fit
+ * or takes the exact but slower route then also sets one of the MV_DBG_* bits in a status word that lives in
+ * the first bytes of the context's workspace.  Nothing traps and nothing is asserted: the kernels do what the
+ * normal build does, and the context stays usable.  mv_debug_status waits for the context's stream, returns
+ * the bits collected since the previous read in *device_status and clears them.  In a normal build it
+ * returns MV_OK with *device_status = 0.  mv_debug_build returns 1 for a checked build, else 0.
+ * (Steps named by the bits: S_top of Eq. 6 / Algorithm 1 for the candidate, window and fallback bits, the
+ * vote sum and the outer S_top of Eq. 9, the aggregate of Eq. 8.) */
+int mv_debug_status(mv_ctx* ctx, int* device_status);
+int mv_debug_build(void);
 
 const char* mv_status_string(int status);
 

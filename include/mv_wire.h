@@ -46,7 +46,10 @@ int64_t mv_pos_stream_bits(int64_t d, int64_t B, int64_t K);
 size_t mv_pos_decode_workspace_bytes(int64_t nbits, int64_t B);
 
 /* Encodes an ascending index list (Section 4.3, sender side).
- *   idx   [K] int32 in   strictly ascending, 0 <= idx < d (as mv_sparse_step writes it)
+ *   idx   [K] int32 in   strictly ascending, 0 <= idx < d (as mv_sparse_step writes it); an entry
+ *                        outside [0, d) -- such as the -1 padding mv_select_rs leaves when fewer than K
+ *                        coordinates hold a vote -- is skipped and writes nothing (the stream is then
+ *                        the one of the list without it only if such entries come last)
  *   words [ceil(mv_pos_stream_bits / 32)] uint32 out, fully overwritten
  * Limits: 1 <= d < 2^31, 1 <= B <= d, 0 <= K <= d. */
 int mv_pos_encode(void* stream, const int32_t* idx, int64_t K, int64_t d, int64_t B, uint32_t* words);

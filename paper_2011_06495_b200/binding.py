@@ -15,6 +15,7 @@ import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmvsparse.so")
+LIB_DEBUG_PATH = os.path.join(_HERE, "libmvsparse_debug.so")     # the checked build, see MvContext.debug_status
 
 MV_OK = 0
 MV_ERR_INVALID_ARG = -1
@@ -25,8 +26,11 @@ MV_SELECT_STATIC_MAX_D = 1 << 24
 MV_MODE_AUTO = 0
 MV_MODE_GENERAL = 1
 MV_MODE_TRACK = 2
+MV_DBG_CAND_OVERFLOW, MV_DBG_WINDOW_OVERFLOW, MV_DBG_FALLBACK, MV_DBG_LIST_OVERFLOW = 1, 2, 4, 8
+MV_DBG_PICK_RANGE, MV_DBG_LIST_RANGE, MV_DBG_OUT_RANGE, MV_DBG_GATHER_RANGE, MV_DBG_INTERNAL = 16, 32, 64, 128, 256
 
 _lib = None
+_lib_debug = None
 
 
 class MvError(RuntimeError):
@@ -38,13 +42,24 @@ class MvError(RuntimeError):
 def load() -> ctypes.CDLL:
     """Loads libmvsparse.so (built in-tree by paper_2011_06495_b200.build); raises if absent."""
     global _lib
-    if _lib is not None:
-        return _lib
-    if not os.path.exists(LIB_PATH):
-        raise ImportError(
-            f"{LIB_PATH} is missing: build it with `python -m paper_2011_06495_b200.build` "
-            "(there is no CPU fallback)")
-    lib = ctypes.CDLL(LIB_PATH)
+    if _lib is None:
+        _lib = _open(LIB_PATH, "python -m paper_2011_06495_b200.build")
+    return _lib
+
+
+def load_debug() -> ctypes.CDLL:
+    """Loads the checked build libmvsparse_debug.so (same ABI; its kernels report clamped or refused
+    indices through mv_debug_status); raises if absent."""
+    global _lib_debug
+    if _lib_debug is None:
+        _lib_debug = _open(LIB_DEBUG_PATH, "python -m paper_2011_06495_b200.build --debug")
+    return _lib_debug
+
+
+def _open(path: str, how: str) -> ctypes.CDLL:
+    if not os.path.exists(path):
+        raise ImportError(f"{path} is missing: build it with `{how}` (there is no CPU fallback)")
+    lib = ctypes.CDLL(path)
     c_vp, c_i, c_i64, c_sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_size_t
     lib.mv_workspace_bytes.restype = c_sz
     lib.mv_workspace_bytes.argtypes = [c_i, c_i64, c_i64]
@@ -110,7 +125,12 @@ def load() -> ctypes.CDLL:
     lib.mv_quantize.argtypes = [c_vp, c_vp, c_i64, c_i, c_vp, c_vp, c_vp, c_sz]
     lib.mv_dequantize.restype = c_i
     lib.mv_dequantize.argtypes = [c_vp, c_vp, c_i64, c_i, c_vp]
-    _lib = lib
+    lib.mv_fallback_count.restype = c_i
+    lib.mv_fallback_count.argtypes = [c_vp, ctypes.POINTER(ctypes.c_uint32)]
+    lib.mv_debug_status.restype = c_i
+    lib.mv_debug_status.argtypes = [c_vp, ctypes.POINTER(c_i)]
+    lib.mv_debug_build.restype = c_i
+    lib.mv_debug_build.argtypes = []
     return lib
 
 
@@ -189,8 +209,8 @@ class MvContext:
     """A context bound to the current CUDA stream and to a workspace tensor it keeps alive."""
 
     def __init__(self, N: int, d: int, K: int, device="cuda", stream: Optional[torch.cuda.Stream] = None,
-                 mode: int = MV_MODE_AUTO):
-        self.lib = load()
+                 mode: int = MV_MODE_AUTO, debug: bool = False):
+        self.lib = load_debug() if debug else load()
         self.N, self.d, self.K = int(N), int(d), int(K)
         nbytes = workspace_bytes(N, d, K)
         if nbytes == 0:
@@ -301,3 +321,15 @@ class MvContext:
 
     def last_launches(self) -> int:
         return int(self.lib.mv_last_launches(self.handle))
+
+    def fallback_count(self) -> int:
+        """Worker selections that took the full-row route since the context's first call."""
+        total = ctypes.c_uint32()
+        _check(self.lib.mv_fallback_count(self.handle, ctypes.byref(total)), "mv_fallback_count")
+        return int(total.value)
+
+    def debug_status(self) -> int:
+        """MV_DBG_* bits collected by a checked build since the last read (always 0 in a normal build)."""
+        word = ctypes.c_int()
+        _check(self.lib.mv_debug_status(self.handle, ctypes.byref(word)), "mv_debug_status")
+        return int(word.value)

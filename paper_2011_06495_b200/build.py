@@ -10,6 +10,7 @@ SRC = os.path.join(HERE, "csrc", "mv_sparse.cu")
 SRCS = [SRC, os.path.join(HERE, "csrc", "mv_wire.cu")]
 HDRS = [os.path.join(os.path.dirname(HERE), "include", h) for h in ("mv_sparse.h", "mv_wire.h")]
 LIB = os.path.join(HERE, "libmvsparse.so")
+LIB_DEBUG = os.path.join(HERE, "libmvsparse_debug.so")      # the checked build (-DMV_DEBUG), see mv_debug_status
 
 NVCC_FLAGS = [
     "-O3", "-std=c++17", "-lineinfo",
@@ -27,17 +28,20 @@ def nvcc_path() -> str:
     return "nvcc"
 
 
-def needs_build() -> bool:
-    if not os.path.exists(LIB):
+def needs_build(lib: str = LIB) -> bool:
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     return any(os.path.getmtime(f) > t for f in (*SRCS, *HDRS, os.path.abspath(__file__)))
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not needs_build():
-        return LIB
-    cmd = [nvcc_path(), *NVCC_FLAGS, "-o", LIB, *SRCS]
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    """Compiles the library; debug=True compiles the checked variant (device-side bounds checks that set
+    status bits instead of clamping silently) into libmvsparse_debug.so."""
+    lib = LIB_DEBUG if debug else LIB
+    if not force and not needs_build(lib):
+        return lib
+    cmd = [nvcc_path(), *NVCC_FLAGS, *(["-DMV_DEBUG"] if debug else []), "-o", lib, *SRCS]
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")
@@ -47,8 +51,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
         raise RuntimeError("nvcc failed building libmvsparse.so")
     if verbose:
         print(res.stderr)
-    return LIB
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force=True, verbose="-v" in sys.argv))
+    print(build(force=True, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

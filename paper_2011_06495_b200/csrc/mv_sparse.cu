@@ -35,6 +35,7 @@
 #include <stdint.h>
 #include <stdlib.h>
 #include <math.h>
+#include <mutex>
 #include <new>
 
 #include "../../include/mv_sparse.h"
@@ -61,6 +62,7 @@ struct P {
   int force_general;
   int list_mode;          // 1: the rows are plain (key, index) lists to select min(K, length) from (add-drop)
   int apply_rows;         // list mode: rows < apply_rows are "add" lists, the others "drop" lists
+  int no_masks;           // 1: the picks only count votes; the workers' bit masks are neither cleared nor set
   const float* prefetch_acc;  // k_vote_write: if set, the rows whose elements at supp(M) the gather is about to read
   uint32_t* vote_words;   // cluster select: if set, every pick also adds one to its vote byte (four bytes per word)
   uint32_t* apply_bits;   // list mode, optional: the vote masks [apply_rows][W] to update in place instead of
@@ -99,7 +101,24 @@ struct P {
   uint16_t* chunk_vh;     // [N+1][nc_pad]: chunk_vh[v][c] = #{coordinates of chunk c with votes >= v}
   uint32_t* out_base;     // [nchunks]
   uint32_t* tie_take;     // [nchunks]
+  uint32_t* dbg;          // checked build (MV_DEBUG): status word that collects MV_DBG_* bits, or null
+  uint32_t* fb_total;     // running count of worker selections that went over the full row (or null)
 };
+
+// Checked build: a kernel that clamps, skips or falls back says so by setting a bit of the status word
+// (never a trap or an assert: the context stays usable and the host reads the word afterwards).
+#ifdef MV_DEBUG
+#define MV_DBG(ptr, bit)                         \
+  do {                                           \
+    if ((ptr) != nullptr) atomicOr((ptr), (uint32_t)(bit)); \
+  } while (0)
+constexpr bool kChecked = true;
+#else
+#define MV_DBG(ptr, bit) \
+  do {                   \
+  } while (0)
+constexpr bool kChecked = false;
+#endif
 
 // Programmatic dependent launch: every kernel first waits for the kernel before it on the stream
 // to finish (all of its memory operations visible), then lets the kernel after it be scheduled.
@@ -558,8 +577,10 @@ __global__ void __launch_bounds__(TPB, 4) k_acc_compact(P p, const float* __rest
     }
     __syncthreads();
     const uint32_t base = s_base;
-    for (uint32_t i = threadIdx.x; i < total; i += TPB)
+    for (uint32_t i = threadIdx.x; i < total; i += TPB) {
       if (base + i < p.cap) out[base + i] = s_q[i];
+      else MV_DBG(p.dbg, MV_DBG_CAND_OVERFLOW);
+    }
   } else {
     if (threadIdx.x == 0) {
       s_base = base_r;
@@ -570,6 +591,7 @@ __global__ void __launch_bounds__(TPB, 4) k_acc_compact(P p, const float* __rest
     const uint32_t cap = p.cap;
     emit_candidates(g, key, cm, xkey, xcm, s_w, [&](uint32_t pos, uint2 v) {
       if (base + pos < cap) out[base + pos] = v;
+      else MV_DBG(p.dbg, MV_DBG_CAND_OVERFLOW);
     });
   }
 }
@@ -963,6 +985,11 @@ __device__ __forceinline__ void store_vote_hist_impl(const P& p, int c, uint32_t
 // Puts the picked bits `bits` of mask word w of row n where they belong: into the row's bit mask, or
 // (add-drop, in-place update) into the vote mask, set for an "add" row and cleared for a "drop" row.
 __device__ __forceinline__ void put_bits(const P& p, int n, uint32_t w, uint32_t bits) {
+  if (p.no_masks) return;
+  if (kChecked && (int64_t)w >= p.W) {
+    MV_DBG(p.dbg, MV_DBG_INTERNAL);
+    return;
+  }
   if (p.apply_bits == nullptr) {
     atomicOr(p.worker_bits + (size_t)n * p.W + w, bits);
   } else if (n < p.apply_rows) {
@@ -977,7 +1004,14 @@ __global__ void __launch_bounds__(TPB) k_set_bits(P p, float* __restrict__ err) 
   __shared__ uint32_t s_we[9];
   const int n = blockIdx.y;
   const bool fast = worker_fast(p, n);
-  if (p.list_mode && !fast) return;  // empty list
+  if (p.list_mode && !fast) {  // empty list
+    if (kChecked && blockIdx.x == 0 && threadIdx.x == 0 && p.cand_cnt[n] > p.cap) MV_DBG(p.dbg, MV_DBG_LIST_OVERFLOW);
+    return;
+  }
+  if (!fast && !p.force_general && blockIdx.x == 0 && threadIdx.x == 0) {
+    MV_DBG(p.dbg, MV_DBG_FALLBACK);
+    if (p.fb_total != nullptr) atomicAdd(p.fb_total, 1u);
+  }
   const uint32_t* ws = p.wstate + (size_t)n * 8;
   const uint32_t T = ws[4], need = ws[7];
   const bool all_ties = need >= ws[6];
@@ -1053,9 +1087,9 @@ __global__ void __launch_bounds__(TPB) k_set_bits(P p, float* __restrict__ err) 
 #pragma unroll
           for (int e = 0; e < 4; e++)
             if (sm[i] & (1u << e)) {
-            atomicOr(bits_row + ((uint32_t)(jf + e) >> 5), 1u << ((uint32_t)(jf + e) & 31u));
-            if (p.vote_words) add_vote(p.vote_words, (uint32_t)(jf + e));
-          }
+              if (!p.no_masks) atomicOr(bits_row + ((uint32_t)(jf + e) >> 5), 1u << ((uint32_t)(jf + e) & 31u));
+              if (p.vote_words) add_vote(p.vote_words, (uint32_t)(jf + e));
+            }
         }
       }
       if (xsm) {
@@ -1064,7 +1098,7 @@ __global__ void __launch_bounds__(TPB) k_set_bits(P p, float* __restrict__ err) 
 #pragma unroll
         for (int e = 0; e < 4; e++)
           if (xsm & (1u << e)) {
-            atomicOr(bits_row + ((uint32_t)(jf + e) >> 5), 1u << ((uint32_t)(jf + e) & 31u));
+            if (!p.no_masks) atomicOr(bits_row + ((uint32_t)(jf + e) >> 5), 1u << ((uint32_t)(jf + e) & 31u));
             if (p.vote_words) add_vote(p.vote_words, (uint32_t)(jf + e));
           }
       }
@@ -1084,6 +1118,7 @@ __global__ void __launch_bounds__(TPB) k_set_bits(P p, float* __restrict__ err) 
       const uint32_t key = (q & 1) ? v[q >> 1].z : v[q >> 1].x;
       const uint32_t j = (q & 1) ? v[q >> 1].w : v[q >> 1].y;
       const bool sel = i0 + q < cnt && (key > T || (key == T && all_ties));
+      if (kChecked && sel && (int64_t)j >= p.d) MV_DBG(p.dbg, MV_DBG_PICK_RANGE);
       if (sel && (int64_t)j < p.d) {
         const uint32_t w = j >> 5;
         if (w != curw) {
@@ -1259,7 +1294,7 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(ST, 1) k_select_clu
     if ((int)blockIdx.y >= zero_first) {
       const size_t nblocks = (size_t)gridDim.x * (gridDim.y - zero_first);
       const size_t bid = (size_t)(blockIdx.y - zero_first) * gridDim.x + blockIdx.x;
-      zero_share(p.worker_bits, (size_t)p.N * (size_t)p.W, bid, nblocks);
+      if (!p.no_masks) zero_share(p.worker_bits, (size_t)p.N * (size_t)p.W, bid, nblocks);
       if (p.vote_words != nullptr) zero_share(p.vote_words, (size_t)p.nchunks * (CH / 4), bid, nblocks);
     }
   }
@@ -1336,6 +1371,7 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(ST, 1) k_select_clu
         if (((kk - tau) >> WIN_SHIFT) == bw) {
           const uint32_t at = atomicAdd(lcnt, 1u);
           if (at < (uint32_t)WIN_LIST) list[at] = kk;
+          else MV_DBG(p.dbg, MV_DBG_WINDOW_OVERFLOW);
         }
       }
       __threadfence();
@@ -1681,8 +1717,10 @@ __global__ void __launch_bounds__(TPB) k_lists(P p) {
       buf[o++] = (uint16_t)((q * 32 + lane) * 32 + b);
     }
     __syncwarp();
-    for (uint32_t t = lane; t < tot; t += 32)
+    for (uint32_t t = lane; t < tot; t += 32) {
       if (pos + t < (uint32_t)p.K) lst[pos + t] = c * CH + (int)buf[t];
+      else MV_DBG(p.dbg, MV_DBG_LIST_RANGE);
+    }
     __syncwarp();
     pos += tot;
   }
@@ -1839,6 +1877,7 @@ __global__ void __launch_bounds__(TPB) k_vote_write(P p, const uint8_t* __restri
         for (int n = 0; n < p.N; n++) asm volatile("prefetch.global.L2 [%0];" ::"l"(a + (size_t)n * (size_t)p.d));
       }
     }
+    else MV_DBG(p.dbg, MV_DBG_OUT_RANGE);
     pos++;
   }
   if (mask_bits != nullptr) {
@@ -1858,7 +1897,7 @@ __global__ void __launch_bounds__(TPB) k_vote_write(P p, const uint8_t* __restri
 __global__ void __launch_bounds__(TPB) k_gather(float* __restrict__ acc, int N, int64_t d, int64_t K,
                                                 const int32_t* __restrict__ idx, float* __restrict__ out_val,
                                                 uint4* __restrict__ zero_ptr, uint32_t zero_vecs,
-                                                double* __restrict__ out_sum) {
+                                                double* __restrict__ out_sum, uint32_t* __restrict__ dbg) {
   pdl_enter();
   for (uint32_t i = blockIdx.x * TPB + threadIdx.x; i < zero_vecs; i += gridDim.x * TPB)
     zero_ptr[i] = make_uint4(0, 0, 0, 0);
@@ -1866,6 +1905,7 @@ __global__ void __launch_bounds__(TPB) k_gather(float* __restrict__ acc, int N, 
   if (k >= K) return;
   const int64_t j = idx[k];
   if (j < 0 || j >= d) {
+    MV_DBG(dbg, MV_DBG_GATHER_RANGE);
     if (out_sum) out_sum[k] = 0.0;
     else out_val[k] = 0.f;
     return;
@@ -1973,11 +2013,15 @@ __global__ void __launch_bounds__(TPB) k_ad_fill(P p, P a, const uint32_t* __res
     for (uint32_t i = lane; i < rcnt; i += 32) {
       const uint2 kv = __ldcg(run + i);
       const uint32_t o = kv.y - (uint32_t)c * CH;  // offset within the chunk
-      if (o >= (uint32_t)CH) continue;             // cannot happen for a well-formed run
+      if (o >= (uint32_t)CH) {                      // cannot happen for a well-formed run
+        MV_DBG(p.dbg, MV_DBG_INTERNAL);
+        continue;
+      }
       const uint32_t w = s_A[warp][o >> 5], bit = o & 31u;
       if ((w >> bit) & 1u) {
         const uint32_t pos = ba + s_rank[warp][o >> 5] + __popc(w & ((1u << bit) - 1u));
         if (pos < a.cap) la[pos] = kv;
+        else MV_DBG(p.dbg, MV_DBG_LIST_OVERFLOW);
       }
     }
   }
@@ -1990,6 +2034,7 @@ __global__ void __launch_bounds__(TPB) k_ad_fill(P p, P a, const uint32_t* __res
       m &= m - 1;
       const int64_t j = j0 + b;
       if (j < p.d && posa < a.cap) la[posa] = make_uint2(fkey(row[j]), (uint32_t)j);
+      else MV_DBG(p.dbg, MV_DBG_LIST_OVERFLOW);
       posa++;
     }
     m = D[q];
@@ -1998,6 +2043,7 @@ __global__ void __launch_bounds__(TPB) k_ad_fill(P p, P a, const uint32_t* __res
       m &= m - 1;
       const int64_t j = j0 + b;
       if (j < p.d && posd < a.cap) ld[posd] = make_uint2(0x7fffffffu - fkey(row[j]), (uint32_t)j);  // smallest first
+      else MV_DBG(p.dbg, MV_DBG_LIST_OVERFLOW);
       posd++;
     }
   }
@@ -2097,6 +2143,7 @@ __global__ void __launch_bounds__(TPB) k_rs_fill(P p, P a, const uint8_t* __rest
     const double t = __ddiv_rn(neg_log_u(x), (double)s_v[i]);
     const uint32_t tb = __float_as_uint(__double2float_rn(t));
     if (base + i < a.cap) a.cand[base + i] = make_uint2(0x7fffffffu - tb, j);
+    else MV_DBG(p.dbg, MV_DBG_LIST_OVERFLOW);
   }
 }
 
@@ -2137,7 +2184,10 @@ struct Layout {
   int nchunks;
   int64_t W;
   uint32_t cap;
-  size_t zero_bytes;  // the leading region cleared at the start of every vote
+  size_t dbg;         // header, at the start of the workspace whatever the sizes: word 0 the checked build's status
+  size_t fb_total;    // word, word 1 the running count of full-row selections
+  size_t zero_off;    // start of ...
+  size_t zero_bytes;  // ... the region that is clear at the start of every vote
   size_t samp_hist, hist1, hist2, hist2b, hist3, cand_cnt, sample_done, count_done, votes_done, hot, vote_hist;
   size_t tau, tau_alt, tstate, diag_cnt, wstate, thresh, vstate, cand, chunk_base, chunk_cnt, chunk_eq, tie_base, chunk_sel;
   size_t worker_bits, worker_idx, votes, chunk_vh, out_base, tie_take;
@@ -2169,6 +2219,9 @@ Layout make_layout(int N, int64_t d, int64_t K) {
   L.cap = (uint32_t)((cap + 7) & ~(int64_t)7);  // multiple of 8: every worker's buffer is 64-byte aligned
   size_t off = 0;
   const size_t n = (size_t)N, nc = (size_t)L.nchunks;
+  L.dbg = take(off, 8);
+  L.fb_total = L.dbg + 4;
+  L.zero_off = off;
   L.samp_hist = take(off, n * SB_BINS * 4);
   L.hist1 = take(off, n * H1_BINS * 4);
   L.hist2 = take(off, n * H2_BINS * 4);
@@ -2180,7 +2233,7 @@ Layout make_layout(int N, int64_t d, int64_t K) {
   L.hot = take(off, (size_t)((L.nchunks + 7) & ~7));
   L.votes_done = take(off, 4);
   L.vote_hist = take(off, 256 * 4);
-  L.zero_bytes = off;
+  L.zero_bytes = off - L.zero_off;
   L.tau = take(off, n * 4);
   L.tau_alt = take(off, n * 4);
   L.tstate = take(off, n * 2 * 4);
@@ -2251,7 +2304,10 @@ struct mv_ctx {
   int phase_timing;
   cudaEvent_t pev[48];
   bool pev_made;
-  size_t clean_bytes;  // leading workspace bytes known to be zero (left so by the previous whole step)
+  size_t clean_bytes;  // bytes from the start of the cleared region known to be zero (left so by the previous whole step)
+  int sms;             // multiprocessors of the workspace's device (0 = not asked yet)
+  int cta_budget;      // the largest multiple of 8 CTAs that is not above sms: one CTA per SM for the cluster select
+  bool dbg_ready;      // the workspace's header has been cleared once
   // remembered for mv_read_diag
   int last_N;
   int64_t last_d, last_K;
@@ -2274,6 +2330,7 @@ P make_params(const mv_ctx* ctx, const Layout& L, int N, int64_t d, int64_t K) {
   p.force_general = ctx->mode == MV_MODE_GENERAL ? 1 : 0;
   p.list_mode = 0;
   p.apply_rows = 0;
+  p.no_masks = 0;
   p.vote_words = nullptr;
   p.prefetch_acc = nullptr;
   p.apply_bits = nullptr;
@@ -2311,7 +2368,30 @@ P make_params(const mv_ctx* ctx, const Layout& L, int N, int64_t d, int64_t K) {
   p.chunk_vh = (uint16_t*)(b + L.chunk_vh);
   p.out_base = (uint32_t*)(b + L.out_base);
   p.tie_take = (uint32_t*)(b + L.tie_take);
+  p.dbg = kChecked ? (uint32_t*)(b + L.dbg) : nullptr;
+  p.fb_total = (uint32_t*)(b + L.fb_total);
   return p;
+}
+
+// Properties of the device that holds the workspace, asked for once per context (grid sizes follow
+// the number of multiprocessors); the workspace's header (status word, fallback count) is cleared here too.
+int device_ready(mv_ctx* ctx) {
+  if (ctx->sms == 0) {
+    int dev = -1;
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, ctx->ws) == cudaSuccess && at.type == cudaMemoryTypeDevice) dev = at.device;
+    else cudaGetLastError();
+    if (dev < 0 && cudaGetDevice(&dev) != cudaSuccess) return MV_ERR_CUDA;
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) return MV_ERR_CUDA;
+    ctx->sms = sms;
+    ctx->cta_budget = sms >= 8 ? sms - sms % 8 : 8;
+  }
+  if (!ctx->dbg_ready) {
+    if (cudaMemsetAsync(ctx->ws, 0, 8, ctx->stream) != cudaSuccess) return MV_ERR_CUDA;
+    ctx->dbg_ready = true;
+  }
+  return MV_OK;
 }
 
 template <typename... KArgs, typename... Args>
@@ -2338,8 +2418,10 @@ cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream
 // kernel is told once per device
 bool cluster_select_ready() {
   static bool done[64] = {false};
+  static std::mutex mu;
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+  std::lock_guard<std::mutex> lock(mu);
   if (!done[dev]) {
     if (cudaFuncSetAttribute(k_select_cluster<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, SK_KEYS * 4) != cudaSuccess ||
         cudaFuncSetAttribute(k_select_cluster<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, SK_KEYS * 4) != cudaSuccess) {
@@ -2424,12 +2506,15 @@ int join_side(mv_ctx* ctx) {
 // `topk_only`: stop once the workers' bit masks are set (no vote count, no index lists); everything
 // then stays on the caller's stream
 // `need_hist` = false: the per-chunk vote histograms and offsets are not wanted (the caller selects by other means)
+// `want_lists` = false: the ascending per-worker index lists are not wanted (nothing later in a step reads them)
+// `want_masks` = false: nor are the workers' bit masks (unless the lists, which are built from them, are)
 int vote_impl(mv_ctx* ctx, P p, const Layout& L, const float* grads, float* err, bool topk_only = false,
-              bool need_hist = true) {
+              bool need_hist = true, bool want_lists = true, bool want_masks = true) {
   cudaStream_t st = ctx->stream;
   const int N = p.N;
+  const int SMS = ctx->sms, CTA_BUDGET = ctx->cta_budget;
   ctx->timing_now = ctx->timing > 0 && (ctx->timing_calls++ % ctx->timing) == 0;
-  if (ctx->clean_bytes < L.zero_bytes && cudaMemsetAsync(ctx->ws, 0, L.zero_bytes, st) != cudaSuccess)
+  if (ctx->clean_bytes < L.zero_bytes && cudaMemsetAsync(ctx->ws + L.zero_off, 0, L.zero_bytes, st) != cudaSuccess)
     return MV_ERR_CUDA;
   ctx->clean_bytes = 0;  // dirty from here on, until a whole step's last kernel has cleared it again
   // general mode: per-chunk outputs of the vote count start out cleared (only chunks with picks are
@@ -2447,8 +2532,8 @@ int vote_impl(mv_ctx* ctx, P p, const Layout& L, const float* grads, float* err,
     if (zs != st && cudaEventRecord(ctx->ev_zero, zs) != cudaSuccess) return MV_ERR_CUDA;
   }
   // CTAs per worker of the select kernels: enough for a full-row pass, not more than the candidates need
-  const int gh = p.force_general ? per_row_ctas(N, p.nchunks, 148 * 8)
-                                 : per_row_ctas(N, (int)((p.cap + TPB * 8 - 1) / (TPB * 8)), 148 * 2);
+  const int gh = p.force_general ? per_row_ctas(N, p.nchunks, SMS * 8)
+                                 : per_row_ctas(N, (int)((p.cap + TPB * 8 - 1) / (TPB * 8)), SMS * 2);
   if (!p.force_general) {
     // threshold tracking: the previous call on this context, if it had the same N, d and K, left a
     // threshold per worker in the other tau array; this call reads it instead of sampling and
@@ -2470,13 +2555,16 @@ int vote_impl(mv_ctx* ctx, P p, const Layout& L, const float* grads, float* err,
       uint32_t U, Ls, rank;
       int all;
       sample_plan(p.d, p.K, U, Ls, all, rank);
-      const int gs = per_row_ctas(N, (int)((U + 127) / 128), 148 * 2);
+      const int gs = per_row_ctas(N, (int)((U + 127) / 128), SMS * 2);
       launch_k(k_sample_hist, dim3(dim3(gs, N)), dim3(512), st, p, grads, err, U, Ls, all, rank);
       MV_LAUNCH_CHECK();
     }
     // the votes are counted while the picks are made, in the workspace's vote array (whole chunks long)
     uint8_t* const ws_votes = (uint8_t*)(ctx->ws + L.votes);
     p.vote_words = topk_only ? nullptr : (uint32_t*)ws_votes;
+    // Nothing reads the workers' bit masks when neither they nor the index lists are an output of the call
+    // (a whole step): the picks then only count votes
+    p.no_masks = (!topk_only && !want_lists && !want_masks) ? 1 : 0;
     if (ctx->timing_now) cudaEventRecord(ctx->ev[2 * (ctx->timed % 64)], st);
     launch_k(k_acc_compact, dim3(dim3(p.nchunks, N)), dim3(TPB), st, p, grads, err);
     MV_LAUNCH_CHECK();
@@ -2489,11 +2577,11 @@ int vote_impl(mv_ctx* ctx, P p, const Layout& L, const float* grads, float* err,
     // and the clusters only clear)
     const bool wide = p.cap > (1u << 20);
     const int nsel = wide ? 0 : N;
-    const int cl = nsel * 8 <= 144 ? 8 : 4;                       // one CTA per SM: keep all clusters resident if possible
-    const int zc = nsel * cl < 144 ? (144 - nsel * cl) / cl : 0;  // clusters that only clear
+    const int cl = nsel * 8 <= CTA_BUDGET ? 8 : 4;                              // one CTA per SM: keep all clusters resident if possible
+    const int zc = nsel * cl < CTA_BUDGET ? (CTA_BUDGET - nsel * cl) / cl : 0;  // clusters that only clear
     // the extra clusters clear alone if that does not take them longer than the select takes (measured:
     // about 450 KB per CTA); otherwise every CTA of the grid clears a share first
-    const size_t clear_bytes = (size_t)N * (size_t)p.W * 4 + (topk_only ? 0 : (size_t)p.nchunks * CH);
+    const size_t clear_bytes = (p.no_masks ? 0 : (size_t)N * (size_t)p.W * 4) + (topk_only ? 0 : (size_t)p.nchunks * CH);
     const int zero_first = (nsel > 0 && zc * cl >= 32 && clear_bytes / (size_t)(zc * cl) <= 450 * 1024) ? nsel : 0;
     if (cl == 8) launch_smem(k_select_cluster<8>, dim3(dim3(8, nsel + zc)), dim3(ST), SK_KEYS * 4, st, p, err, zero_first, nsel);
     else launch_smem(k_select_cluster<4>, dim3(dim3(4, nsel + zc)), dim3(ST), SK_KEYS * 4, st, p, err, zero_first, nsel);
@@ -2509,7 +2597,7 @@ int vote_impl(mv_ctx* ctx, P p, const Layout& L, const float* grads, float* err,
       MV_LAUNCH_CHECK();
     }
     // the picks: mask bits and votes, from the candidates (or the row), by the whole GPU
-    launch_k(k_set_bits, dim3(dim3(per_row_ctas(N, (int)((p.cap + TPB * 16 - 1) / (TPB * 16)), 148 * 4), N)), dim3(TPB), st, p,
+    launch_k(k_set_bits, dim3(dim3(per_row_ctas(N, (int)((p.cap + TPB * 16 - 1) / (TPB * 16)), SMS * 4), N)), dim3(TPB), st, p,
              err);
     MV_LAUNCH_CHECK();
     if (topk_only) return MV_OK;
@@ -2538,13 +2626,14 @@ int vote_impl(mv_ctx* ctx, P p, const Layout& L, const float* grads, float* err,
   if (topk_only) return MV_OK;
   if (p.force_general) {
     if (zs != st && cudaStreamWaitEvent(st, ctx->ev_zero, 0) != cudaSuccess) return MV_ERR_CUDA;
-    const dim3 gv(p.nchunks < 148 * 8 ? p.nchunks : 148 * 8);
+    const dim3 gv(p.nchunks < SMS * 8 ? p.nchunks : SMS * 8);
     if (N < 4) launch_k(k_votes<2>, gv, dim3(VT), st, p);
     else if (N < 16) launch_k(k_votes<4>, gv, dim3(VT), st, p);
     else if (N < 64) launch_k(k_votes<6>, gv, dim3(VT), st, p);
     else launch_k(k_votes<8>, gv, dim3(VT), st, p);
     MV_LAUNCH_CHECK();
   }
+  if (!want_lists) return MV_OK;
   // the index lists feed nothing later in the step: write them on the side stream
   cudaStream_t ls = st;
   if (ctx->phase_timing != 1 && side_ready(ctx) && cudaEventRecord(ctx->ev_fork, st) == cudaSuccess &&
@@ -2572,7 +2661,8 @@ int select_impl(mv_ctx* ctx, P p, const Layout& L, const uint8_t* votes, bool ha
   cudaStream_t st = ctx->stream;
   if (!have_hist) {
     ctx->clean_bytes = 0;
-    if (cudaMemsetAsync(ctx->ws + L.votes_done, 0, L.zero_bytes - L.votes_done, st) != cudaSuccess) return MV_ERR_CUDA;
+    if (cudaMemsetAsync(ctx->ws + L.votes_done, 0, L.zero_off + L.zero_bytes - L.votes_done, st) != cudaSuccess)
+      return MV_ERR_CUDA;
     launch_k(k_vote_hist, dim3((p.nchunks + VH_WARPS - 1) / VH_WARPS), dim3(TPB), st, p, votes, (uint8_t*)nullptr);
     MV_LAUNCH_CHECK();
   }
@@ -2584,8 +2674,10 @@ int select_impl(mv_ctx* ctx, P p, const Layout& L, const uint8_t* votes, bool ha
 // steps a5-a6
 int aggregate_impl(mv_ctx* ctx, float* acc, int N, int64_t d, int64_t K, const int32_t* idx, float* out_val,
                    size_t clear_bytes, double* out_sum = nullptr) {
+  const Layout L0 = make_layout(1, 1, 1);  // (the cleared region starts at the same offset for every size)
   launch_k(k_gather, dim3((unsigned)((K + TPB - 1) / TPB)), dim3(TPB), ctx->stream, acc, N, d, K, idx, out_val,
-           (uint4*)ctx->ws, (uint32_t)(clear_bytes / 16), out_sum);
+           (uint4*)(ctx->ws + L0.zero_off), (uint32_t)(clear_bytes / 16), out_sum,
+           kChecked ? (uint32_t*)(ctx->ws + L0.dbg) : (uint32_t*)nullptr);
   MV_LAUNCH_CHECK();
   if (clear_bytes) ctx->clean_bytes = clear_bytes;
   return MV_OK;
@@ -2627,6 +2719,9 @@ int mv_create(mv_ctx** out, void* stream, void* workspace, size_t workspace_byte
   c->track_valid = false;
   c->launches = 0;
   c->clean_bytes = 0;
+  c->sms = 0;
+  c->cta_budget = 8;
+  c->dbg_ready = false;
   c->timing = 0;
   c->timing_calls = 0;
   c->timing_now = false;
@@ -2737,6 +2832,7 @@ int mv_vote(mv_ctx* ctx, const float* grads, float* err, int N, int64_t d, int64
   if ((worker_idx && !aligned16(worker_idx)) || (worker_bits && !aligned16(worker_bits)) ||
       (votes && !aligned16(votes)) || (thresh && !aligned16(thresh)))
     return MV_ERR_INVALID_ARG;
+  if (const int rd = device_ready(ctx)) return rd;
   ctx->launches = 0;
   if (ctx->phase_timing) cudaEventRecord(ctx->pev[0], ctx->stream);
   P p = make_params(ctx, L, N, d, K);
@@ -2747,7 +2843,7 @@ int mv_vote(mv_ctx* ctx, const float* grads, float* err, int N, int64_t d, int64
   ctx->last_N = N;
   ctx->last_d = d;
   ctx->last_K = K;
-  const int rc2 = vote_impl(ctx, p, L, grads, err);
+  const int rc2 = vote_impl(ctx, p, L, grads, err, false, true, worker_idx != nullptr, worker_bits != nullptr);
   const int rc3 = join_side(ctx);
   return rc2 != MV_OK ? rc2 : rc3;
 }
@@ -2758,6 +2854,7 @@ int mv_select(mv_ctx* ctx, const uint8_t* votes, int N, int64_t d, int64_t K, in
   if (rc != MV_OK) return rc;
   if (votes == nullptr || out_idx == nullptr || !aligned16(votes) || !aligned16(out_idx)) return MV_ERR_INVALID_ARG;
   if (mask_bits && !aligned16(mask_bits)) return MV_ERR_INVALID_ARG;
+  if (const int rd = device_ready(ctx)) return rd;
   ctx->launches = 0;
   if (ctx->phase_timing) cudaEventRecord(ctx->pev[0], ctx->stream);
   P p = make_params(ctx, L, N, d, K);
@@ -2770,6 +2867,7 @@ int mv_aggregate(mv_ctx* ctx, float* acc, int N, int64_t d, int64_t K, const int
   if (rc != MV_OK) return rc;
   if (acc == nullptr || idx == nullptr || out_val == nullptr || !aligned16(acc) || !aligned16(idx) || !aligned16(out_val))
     return MV_ERR_INVALID_ARG;
+  if (const int rd = device_ready(ctx)) return rd;
   ctx->launches = 0;
   if (ctx->phase_timing) cudaEventRecord(ctx->pev[0], ctx->stream);
   return aggregate_impl(ctx, acc, N, d, K, idx, out_val, 0);
@@ -2782,6 +2880,7 @@ int mv_aggregate_partial(mv_ctx* ctx, float* acc, int N_local, int64_t d, int64_
   if (rc != MV_OK) return rc;
   if (acc == nullptr || idx == nullptr || out_sum == nullptr || !aligned16(acc) || !aligned16(idx) || !aligned16(out_sum))
     return MV_ERR_INVALID_ARG;
+  if (const int rd = device_ready(ctx)) return rd;
   ctx->launches = 0;
   if (ctx->phase_timing) cudaEventRecord(ctx->pev[0], ctx->stream);
   return aggregate_impl(ctx, acc, N_local, d, K, idx, nullptr, 0, out_sum);
@@ -2803,13 +2902,14 @@ int mv_sparse_step(mv_ctx* ctx, const float* grads, float* err, int N, int64_t d
   if (!aligned16(grads) || !aligned16(err) || !aligned16(out_idx) || !aligned16(out_val)) return MV_ERR_INVALID_ARG;
   const size_t nb = (size_t)N * (size_t)d * 4;
   if (overlap(grads, nb, err, nb)) return MV_ERR_INVALID_ARG;
+  if (const int rd = device_ready(ctx)) return rd;
   ctx->launches = 0;
   if (ctx->phase_timing) cudaEventRecord(ctx->pev[0], ctx->stream);
   P p = make_params(ctx, L, N, d, K);
   ctx->last_N = N;
   ctx->last_d = d;
   ctx->last_K = K;
-  rc = vote_impl(ctx, p, L, grads, err);
+  rc = vote_impl(ctx, p, L, grads, err, false, true, false, false);  // (the workers' lists and masks are no output of the step)
   p.prefetch_acc = err;
   if (rc == MV_OK) rc = select_impl(ctx, p, L, p.votes, true, out_idx, nullptr);
   if (rc == MV_OK) rc = aggregate_impl(ctx, err, N, d, K, out_idx, out_val, L.zero_bytes);
@@ -2831,6 +2931,7 @@ int mv_ad_step(mv_ctx* ctx, const float* grads, float* err, uint32_t* prev_bits,
     return MV_ERR_INVALID_ARG;
   const size_t nb = (size_t)N * (size_t)d * 4;
   if (overlap(grads, nb, err, nb)) return MV_ERR_INVALID_ARG;
+  if (const int rd = device_ready(ctx)) return rd;
   ctx->launches = 0;
   if (ctx->phase_timing) cudaEventRecord(ctx->pev[0], ctx->stream);
   cudaStream_t st = ctx->stream;
@@ -2873,11 +2974,11 @@ int mv_ad_step(mv_ctx* ctx, const float* grads, float* err, uint32_t* prev_bits,
   launch_k(k_ad_fill, dim3(dim3((p.nchunks + TPB / 32 - 1) / (TPB / 32), N)), dim3(TPB), st, p, a,
            (const uint32_t*)prev_bits, (const float*)err);
   MV_LAUNCH_CHECK();
-  const int ga = per_row_ctas(2 * N, (int)((a.cap + TPB * 8 - 1) / (TPB * 8)), 148 * 2);
+  const int ga = per_row_ctas(2 * N, (int)((a.cap + TPB * 8 - 1) / (TPB * 8)), ctx->sms * 2);
   if (a.cap <= (1u << 20) && cluster_select_ready()) {
     // a cluster per list finds the key of its K_ad-th entry (three radix digits; nothing is cleared here)
     const int rows = 2 * N;
-    if (rows * 8 <= 144) launch_smem(k_select_cluster<8>, dim3(dim3(8, rows)), dim3(ST), SK_KEYS * 4, st, a, err, rows, rows);
+    if (rows * 8 <= ctx->cta_budget) launch_smem(k_select_cluster<8>, dim3(dim3(8, rows)), dim3(ST), SK_KEYS * 4, st, a, err, rows, rows);
     else launch_smem(k_select_cluster<4>, dim3(dim3(4, rows)), dim3(ST), SK_KEYS * 4, st, a, err, rows, rows);
     MV_LAUNCH_CHECK();
   } else {
@@ -2904,7 +3005,7 @@ int mv_ad_step(mv_ctx* ctx, const float* grads, float* err, uint32_t* prev_bits,
   if (msum) v.votes = msum;
   if (cudaMemsetAsync(p.hot, 1, (size_t)p.nc_pad, st) != cudaSuccess) return MV_ERR_CUDA;  // every chunk may hold votes
   {
-    const dim3 gv(p.nchunks < 148 * 8 ? p.nchunks : 148 * 8);
+    const dim3 gv(p.nchunks < ctx->sms * 8 ? p.nchunks : ctx->sms * 8);
     if (N < 4) launch_k(k_votes<2>, gv, dim3(VT), st, v);
     else if (N < 16) launch_k(k_votes<4>, gv, dim3(VT), st, v);
     else if (N < 64) launch_k(k_votes<6>, gv, dim3(VT), st, v);
@@ -2957,6 +3058,10 @@ int rs_select_impl(mv_ctx* ctx, const P& p, const Layout& L, const uint8_t* vote
                    int32_t* out_idx, uint32_t* mask_bits) {
   cudaStream_t st = ctx->stream;
   char* b = ctx->ws;
+  // The list regions written here sit at offsets of this call's own (N, d, K): they may overlap the
+  // region that a whole step of another size left cleared, so nothing counts as clean from here on
+  // (a whole step that follows gets the zeros back from its last kernel).
+  ctx->clean_bytes = 0;
   // one list that can hold every voted coordinate (at most min(d, N K) of them)
   const uint64_t room = (uint64_t)2 * (uint64_t)p.N * (uint64_t)L.ad_cap;
   P a = list_params(ctx, L, p, 1, p.K, (uint32_t)(room < 0xfffffff8ull ? room : 0xfffffff8ull));
@@ -2967,7 +3072,7 @@ int rs_select_impl(mv_ctx* ctx, const P& p, const Layout& L, const uint8_t* vote
   MV_LAUNCH_CHECK();
   uint64_t most = (uint64_t)p.N * (uint64_t)p.K;
   if (most > (uint64_t)p.d) most = (uint64_t)p.d;
-  const int ga = per_row_ctas(1, (int)((most + TPB * 8 - 1) / (TPB * 8)), 148 * 2);
+  const int ga = per_row_ctas(1, (int)((most + TPB * 8 - 1) / (TPB * 8)), ctx->sms * 2);
   launch_k(k_hist<1, false>, dim3(dim3(ga, 1)), dim3(TPB), st, a, nullptr, nullptr);
   MV_LAUNCH_CHECK();
   launch_k(k_hist<2, false>, dim3(dim3(ga, 1)), dim3(TPB), st, a, nullptr, nullptr);
@@ -3006,6 +3111,7 @@ int mv_select_rs(mv_ctx* ctx, const uint8_t* votes, int N, int64_t d, int64_t K,
   if (rc != MV_OK) return rc;
   if (votes == nullptr || out_idx == nullptr || !aligned16(votes) || !aligned16(out_idx)) return MV_ERR_INVALID_ARG;
   if (mask_bits && !aligned16(mask_bits)) return MV_ERR_INVALID_ARG;
+  if (const int rd = device_ready(ctx)) return rd;
   ctx->launches = 0;
   if (ctx->phase_timing) cudaEventRecord(ctx->pev[0], ctx->stream);
   const P p = make_params(ctx, L, N, d, K);
@@ -3021,13 +3127,14 @@ int mv_rs_step(mv_ctx* ctx, const float* grads, float* err, int N, int64_t d, in
   if (!aligned16(grads) || !aligned16(err) || !aligned16(out_idx) || !aligned16(out_val)) return MV_ERR_INVALID_ARG;
   const size_t nb = (size_t)N * (size_t)d * 4;
   if (overlap(grads, nb, err, nb)) return MV_ERR_INVALID_ARG;
+  if (const int rd = device_ready(ctx)) return rd;
   ctx->launches = 0;
   if (ctx->phase_timing) cudaEventRecord(ctx->pev[0], ctx->stream);
   P p = make_params(ctx, L, N, d, K);
   ctx->last_N = N;
   ctx->last_d = d;
   ctx->last_K = K;
-  rc = vote_impl(ctx, p, L, grads, err, false, false);  // the random selection reads the votes themselves
+  rc = vote_impl(ctx, p, L, grads, err, false, false, false, false);  // the random selection reads the votes themselves
   // the union of N top-K sets holds at least K coordinates, so the mask is always full
   if (rc == MV_OK) rc = rs_select_impl(ctx, p, L, p.votes, seed, draw, out_idx, nullptr);
   if (rc == MV_OK) rc = aggregate_impl(ctx, err, N, d, K, out_idx, out_val, L.zero_bytes);
@@ -3083,6 +3190,29 @@ int mv_read_diag(mv_ctx* ctx, int N, uint32_t* per_worker) {
 
 int mv_last_launches(const mv_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
+int mv_fallback_count(mv_ctx* ctx, uint32_t* total) {
+  if (ctx == nullptr || total == nullptr) return MV_ERR_INVALID_ARG;
+  *total = 0;
+  if (!ctx->dbg_ready) return MV_OK;  // no call yet
+  if (cudaMemcpyAsync(total, ctx->ws + 4, 4, cudaMemcpyDeviceToHost, ctx->stream) != cudaSuccess) return MV_ERR_CUDA;
+  if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return MV_ERR_CUDA;
+  return MV_OK;
+}
+
+int mv_debug_build(void) { return kChecked ? 1 : 0; }
+
+int mv_debug_status(mv_ctx* ctx, int* device_status) {
+  if (ctx == nullptr || device_status == nullptr) return MV_ERR_INVALID_ARG;
+  *device_status = 0;
+  if (!kChecked || !ctx->dbg_ready) return MV_OK;  // an unchecked build sets no bits; no call yet: nothing to read
+  uint32_t word = 0;
+  if (cudaMemcpyAsync(&word, ctx->ws, 4, cudaMemcpyDeviceToHost, ctx->stream) != cudaSuccess) return MV_ERR_CUDA;
+  if (cudaMemsetAsync(ctx->ws, 0, 4, ctx->stream) != cudaSuccess) return MV_ERR_CUDA;
+  if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return MV_ERR_CUDA;
+  *device_status = (int)word;
+  return MV_OK;
+}
+
 // ---------------------------------------------------------------------------------------------
 // mv_select_static: the shared-mask selection with its scratch in a fixed device array
 // ---------------------------------------------------------------------------------------------
@@ -3110,8 +3240,10 @@ constexpr int MAX_DEVICES = 64;
 unsigned char* g_select_scratch_addr[MAX_DEVICES] = {nullptr};
 
 int select_scratch_address(unsigned char** out) {
+  static std::mutex mu;
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return MV_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(mu);
   if (g_select_scratch_addr[dev] == nullptr) {
     void* ptr = nullptr;
     if (cudaGetSymbolAddress(&ptr, g_select_scratch) != cudaSuccess || ptr == nullptr) return MV_ERR_CUDA;

@@ -41,12 +41,18 @@ __device__ __forceinline__ uint64_t window(const uint32_t* words, int64_t nwords
 }
 
 // ------------------------------------------------------------------------------------------ position encoder
-__global__ void k_pos_encode(const int32_t* __restrict__ idx, int64_t K, uint32_t B, int w, uint32_t* __restrict__ words) {
+// An entry that is not a coordinate (negative, e.g. the -1 padding of a short list, or >= d), or whose token
+// would not fit the stream, is skipped: nothing is written outside `words`.
+__global__ void k_pos_encode(const int32_t* __restrict__ idx, int64_t K, uint32_t B, int w, uint32_t d, int64_t nbits,
+                             uint32_t* __restrict__ words) {
   int64_t k = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
   if (k >= K) return;
-  uint32_t j = uint32_t(idx[k]);
+  const int32_t ji = idx[k];
+  if (ji < 0 || uint32_t(ji) >= d) return;
+  uint32_t j = uint32_t(ji);
   uint32_t blk = j / B, o = j - blk * B;
   int64_t pos = k * (1 + w) + blk;
+  if (pos + 1 + w > nbits) return;
   uint64_t token = 1u | (w ? (uint64_t(__brev(o) >> (32 - w)) << 1) : 0u);     // offset bits, most significant first
   uint64_t val = token << (pos & 31);
   atomicOr(words + (pos >> 5), uint32_t(val));
@@ -341,7 +347,7 @@ int mv_pos_encode(void* stream, const int32_t* idx, int64_t K, int64_t d, int64_
   if (nbits < 0 || !words || (K > 0 && !idx) || misaligned(words, 4) || misaligned(idx, 4)) return MV_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (cudaMemsetAsync(words, 0, size_t((nbits + 31) / 32) * 4, st) != cudaSuccess) return MV_ERR_CUDA;
-  if (K > 0) k_pos_encode<<<unsigned((K + 255) / 256), 256, 0, st>>>(idx, K, uint32_t(B), offset_bits(B), words);
+  if (K > 0) k_pos_encode<<<unsigned((K + 255) / 256), 256, 0, st>>>(idx, K, uint32_t(B), offset_bits(B), uint32_t(d), nbits, words);
   return cuda_ok();
 }
 

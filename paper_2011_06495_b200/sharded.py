@@ -8,6 +8,7 @@ under Eq. 8).  With one rank it degenerates to the single-GPU step.
 """
 from __future__ import annotations
 
+import contextlib
 from typing import Optional
 
 import torch
@@ -16,7 +17,11 @@ import torch.distributed as dist
 
 class ShardedStep:
     """ctx: an MvContext-like object sized for (N_total, d, K); group: a torch.distributed process group
-    (None = the default group); N_total: workers over all ranks."""
+    (None = the default group); N_total: workers over all ranks.
+
+    The library enqueues on the stream the context was created with, the collectives on torch's current
+    stream: `step` makes the context's stream current for its whole body, so the two are one stream and
+    every call sees the results of the one before it."""
 
     def __init__(self, ctx, N_total: int, d: int, K: int, device, group: Optional[dist.ProcessGroup] = None):
         self.ctx, self.N_total, self.d, self.K, self.group = ctx, int(N_total), int(d), int(K), group
@@ -28,9 +33,16 @@ class ShardedStep:
         residual; out_idx / out_val [K] receive the shared mask and the mean over all N_total workers."""
         if self.N_total > 255:
             raise ValueError("at most 255 workers in total (votes are counted in a byte)")
-        self.ctx.mv_vote(grads_local, err_local, votes=self.votes, K=self.K)
-        dist.all_reduce(self.votes, op=dist.ReduceOp.SUM, group=self.group)
-        self.ctx.mv_select(self.votes, self.N_total, out_idx, K=self.K)
-        self.ctx.mv_aggregate_partial(err_local, out_idx, self.partial)
-        dist.all_reduce(self.partial, op=dist.ReduceOp.SUM, group=self.group)
-        self.ctx.mv_finish_mean(self.partial, self.N_total, out_val)
+        with self._on_context_stream():
+            self.ctx.mv_vote(grads_local, err_local, votes=self.votes, K=self.K)
+            dist.all_reduce(self.votes, op=dist.ReduceOp.SUM, group=self.group)
+            self.ctx.mv_select(self.votes, self.N_total, out_idx, K=self.K)
+            self.ctx.mv_aggregate_partial(err_local, out_idx, self.partial)
+            dist.all_reduce(self.partial, op=dist.ReduceOp.SUM, group=self.group)
+            self.ctx.mv_finish_mean(self.partial, self.N_total, out_val)
+
+    def _on_context_stream(self):
+        stream = getattr(self.ctx, "stream", None)
+        if isinstance(stream, torch.cuda.Stream):
+            return torch.cuda.stream(stream)
+        return contextlib.nullcontext()      # a CPU stand-in for the context has no stream

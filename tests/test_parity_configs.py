@@ -4,13 +4,16 @@ benchmark times (mv_sparse_step on the current stream, automatic threshold mode)
 c2, c3, c4: every step of the run is compared with the CPU oracle (shared mask, aggregated values,
 residual), the residual being carried on both sides; the first and last step also compare the
 per-worker lists, masks, votes and thresholds.  The sweep cells (c5) compare everything for the
-small and middle sizes and, for the 2^27-coordinate cells, sampled rows and sampled outputs plus
-properties that hold at any size.  Inputs are generated on the GPU and the same bytes go to the
-oracle.
+small and middle sizes at once and, for the cells whose N x d is too large for that, stream the rows
+through the oracle one by one: every row's accumulated values, support, mask and threshold, the votes,
+the shared mask, all K aggregated values and every row's residual are compared.  Inputs are generated
+on the GPU and the same bytes go to the oracle.
 """
 import os
+from concurrent.futures import ThreadPoolExecutor
 
 import numpy as np
+import psutil
 import pytest
 import torch
 
@@ -72,6 +75,13 @@ def test_named_config_every_step(name, mode):
     assert sum(settled) == 0, f"worker-steps that fell back to the full-row select on smooth data, per step: {fallbacks}"
 
 
+def _row_threads(d):
+    """Host threads for the row-by-row oracle of a large cell: each holds about ten arrays of d four-byte
+    elements at its peak; stay within the cores and within half of the free host memory."""
+    by_memory = int(psutil.virtual_memory().available // 2 // (40 * d))
+    return max(1, min(THREADS, by_memory))
+
+
 def _cells():
     cells = WL.sweep_cells()
     if FULL:
@@ -93,7 +103,8 @@ def test_sweep_cell(w):
         PT.compare_all(ctx, grads, err0, w.K, ref=O.mv_sparse_step(PT.npy(grads), PT.npy(err0), w.K, threads=THREADS),
                        label=f"[{w.name}] ")
         return
-    # ---- large cell: sampled rows through the oracle, the rest through size-independent properties
+    # ---- large cell: N x d does not fit the host comfortably, so the rows stream through the oracle one
+    # at a time (copied to the host, processed, discarded), several rows in flight on host threads
     N, d, K = w.N, w.d, w.K
     W = (d + 31) // 32
     acc = err0.clone()
@@ -103,45 +114,55 @@ def test_sweep_cell(w):
     thresh = torch.empty((N, 3), dtype=torch.int32, device=DEV)
     ctx.mv_vote(grads, acc, worker_idx, worker_bits, votes, thresh)
     torch.cuda.synchronize()
-    rows = sorted({0, N // 2, N - 1})
-    for n in rows:
+    tag = f"[{w.name}] "
+
+    def vote_row(n):
+        """Algorithm 1, worker side, for row n on the host: accumulate, S_top; everything the GPU wrote
+        for that row is compared here; returns the row's support."""
         acc_row = O.accumulate(PT.npy(grads[n])[None, :], PT.npy(err0[n])[None, :])[0]
-        PT.first_diff(PT.bits(PT.npy(acc[n])), PT.bits(acc_row), f"[{w.name}] acc row {n}")
+        PT.first_diff(PT.bits(PT.npy(acc[n])), PT.bits(acc_row), tag + f"acc row {n}")
         idx, T, cnt_gt, cnt_eq = O.worker_topk(acc_row, K)
-        PT.first_diff(PT.npy(worker_idx[n]), idx, f"[{w.name}] worker_idx row {n}")
-        assert PT.npy(thresh[n], np.uint32).tolist() == [T, cnt_gt, cnt_eq]
-        PT.first_diff(PT.npy(worker_bits[n], np.uint32), O.support_to_bits(idx, d), f"[{w.name}] worker_bits row {n}")
-    # properties: lists strictly ascending, masks hold exactly the listed bits, votes = sum of the lists
-    assert bool((worker_idx[:, 1:] > worker_idx[:, :-1]).all())
-    tally = torch.zeros(d, dtype=torch.int32, device=DEV)
-    for n in range(N):
-        tally.index_add_(0, worker_idx[n].long(), torch.ones(K, dtype=torch.int32, device=DEV))
-    assert torch.equal(tally.to(torch.uint8), votes), "votes differ from the tally of the index lists"
-    assert int(votes.sum(dtype=torch.int64)) == N * K
-    del tally
-    # shared mask: the oracle on the full vote vector
+        del acc_row
+        PT.first_diff(PT.npy(worker_idx[n]), idx, tag + f"worker_idx row {n}")
+        assert PT.npy(thresh[n], np.uint32).tolist() == [T, cnt_gt, cnt_eq], tag + f"thresh row {n}"
+        PT.first_diff(PT.npy(worker_bits[n], np.uint32), O.support_to_bits(idx, d), tag + f"worker_bits row {n}")
+        return idx
+
+    threads = _row_threads(d)
+    votes_ref = np.zeros(d, dtype=np.uint8)
+    with ThreadPoolExecutor(max_workers=threads) as pool:
+        for idx in pool.map(vote_row, range(N)):
+            votes_ref[idx.astype(np.int64)] += 1          # Eq. 9, inner sum (one row at a time, in this thread)
+    PT.first_diff(PT.npy(votes), votes_ref, tag + "votes")
+    # shared mask: the oracle on the oracle's own vote vector
     out_idx = torch.empty(K, dtype=torch.int32, device=DEV)
     mask_bits = torch.empty(W, dtype=torch.int32, device=DEV)
     ctx.mv_select(votes, N, out_idx, mask_bits)
     torch.cuda.synchronize()
-    ref_idx, vstar, vgt, veq = O.select_mask(PT.npy(votes), K)
-    PT.first_diff(PT.npy(out_idx), ref_idx, f"[{w.name}] out_idx")
-    PT.first_diff(PT.npy(mask_bits, np.uint32), O.support_to_bits(ref_idx, d), f"[{w.name}] mask_bits")
+    ref_idx, vstar, vgt, veq = O.select_mask(votes_ref, K)
+    PT.first_diff(PT.npy(out_idx), ref_idx, tag + "out_idx")
+    PT.first_diff(PT.npy(mask_bits, np.uint32), O.support_to_bits(ref_idx, d), tag + "mask_bits")
     assert vstar >= 1
-    # aggregate: sampled outputs one by one, residual: sampled rows in full, the others by property
+    # aggregate: all K outputs from the N x K accumulated values on the mask (acc was compared above)
     out_val = torch.empty(K, dtype=torch.float32, device=DEV)
-    acc_before = {n: PT.npy(acc[n]).copy() for n in rows}
-    sample_k = np.unique(np.linspace(0, K - 1, 4096).astype(np.int64))
-    cols = torch.from_numpy(ref_idx[sample_k].astype(np.int64)).to(DEV)
-    acc_cols = PT.npy(acc[:, cols])
+    cols = torch.from_numpy(ref_idx.astype(np.int64)).to(DEV)
+    acc_cols = np.stack([PT.npy(acc[n][cols]) for n in range(N)])
     ctx.mv_aggregate(acc, out_idx, out_val)
     torch.cuda.synchronize()
-    want = O.aggregate(acc_cols, np.arange(acc_cols.shape[1]))
-    PT.check_out_val(PT.npy(out_val)[sample_k], want, acc_cols, np.arange(acc_cols.shape[1]), f"[{w.name}] out_val sample")
-    for n in rows:
-        want_row = O.residual(acc_before[n][None, :], ref_idx)[0]
-        PT.first_diff(PT.bits(PT.npy(acc[n])), PT.bits(want_row), f"[{w.name}] err row {n}")
-    assert int((acc[:, out_idx.long()].view(torch.int32) != 0).sum()) == 0, "residual not +0 on the mask"
+    want = O.aggregate(acc_cols, np.arange(K))
+    PT.check_out_val(PT.npy(out_val), want, acc_cols, np.arange(K), tag + "out_val")
+    del acc_cols, cols
+
+    def residual_row(n):
+        """Algorithm 1, error update, for row n: the oracle's accumulate and residual against the GPU's row."""
+        acc_row = O.accumulate(PT.npy(grads[n])[None, :], PT.npy(err0[n])[None, :])
+        want_row = O.residual(acc_row, ref_idx)[0]
+        del acc_row
+        PT.first_diff(PT.bits(PT.npy(acc[n])), PT.bits(want_row), tag + f"err row {n}")
+        return n
+
+    with ThreadPoolExecutor(max_workers=threads) as pool:
+        assert list(pool.map(residual_row, range(N))) == list(range(N))
     # the fused step (run in place on err0) gives the same bytes as the phases
     oi2 = torch.empty_like(out_idx)
     ov2 = torch.empty_like(out_val)

@@ -489,3 +489,92 @@ def test_argument_errors_on_device_pointers():
     assert ei.value.status == B.MV_ERR_WORKSPACE
     ctx.mv_sparse_step(g, e, oi, ov)                        # the context is still usable
     torch.cuda.synchronize()
+
+
+def test_random_selection_of_another_size_between_steps():
+    """A stand-alone mv_select_rs of a much smaller problem writes its list state at the offsets of its
+    own (N, d, K), inside what a whole step of the larger problem left cleared: the step that follows
+    must start from clean counters all the same (compared with the oracle, residual carried)."""
+    from oracle import rs_oracle as R
+    N, d, K = 16, 120_011, 1200
+    ctx = B.MvContext(N, d, K, device=DEV, mode=B.MV_MODE_TRACK)
+    g = torch.Generator().manual_seed(4242)
+    err_gpu = torch.zeros(N, d, device=DEV)
+    err_ref = np.zeros((N, d), dtype=np.float32)
+    out_idx = torch.empty(K, dtype=torch.int32, device=DEV)
+    out_val = torch.empty(K, dtype=torch.float32, device=DEV)
+    N2, d2, K2 = 2, 9001, 40
+    for step in range(4):
+        grads = torch.randn(N, d, generator=g)
+        ref = O.mv_sparse_step(grads.numpy(), err_ref, K)
+        ctx.mv_sparse_step(grads.to(DEV), err_gpu, out_idx, out_val)
+        torch.cuda.synchronize()
+        PT.first_diff(PT.npy(out_idx), ref["out_idx"], f"step {step} out_idx")
+        PT.check_out_val(PT.npy(out_val), ref, ref["acc"], ref["out_idx"].astype(np.int64), f"step {step} out_val")
+        PT.first_diff(PT.bits(PT.npy(err_gpu)), PT.bits(ref["err"]), f"step {step} err")
+        err_ref = ref["err"]
+        # the small random selection in between (votes of N2 workers with K2 votes each)
+        votes2 = np.zeros(d2, dtype=np.uint8)
+        rng = np.random.default_rng(step)
+        for _ in range(N2):
+            votes2[rng.choice(d2, K2, replace=False)] += 1
+        idx2 = torch.empty(K2, dtype=torch.int32, device=DEV)
+        ctx.mv_select_rs(torch.from_numpy(votes2).to(DEV), N2, 77, step, idx2, None, K=K2)
+        torch.cuda.synchronize()
+        PT.first_diff(PT.npy(idx2), R.select_mask_rs(votes2, K2, 77, step), f"step {step} small random selection")
+
+
+def _debug_context(N, d, K, mode=B.MV_MODE_AUTO):
+    from paper_2011_06495_b200 import build as BLD
+    BLD.build(debug=True)                      # no-op when the checked library is up to date
+    ctx = B.MvContext(N, d, K, device=DEV, mode=mode, debug=True)
+    assert ctx.lib.mv_debug_build() == 1 and B.load().mv_debug_build() == 0
+    return ctx
+
+
+@pytest.mark.parametrize("name", ["c1", "c1_ties"])
+def test_checked_build_reports_nothing_on_valid_input(name):
+    """The checked build (device-side bounds checks that set status bits) runs the tiny configuration,
+    with and without ties, to the oracle's results and with an empty status word."""
+    w = WL.resnet_like(name)
+    ctx = _debug_context(w.N, w.d, w.K)
+    grads, err = WL.gradients(w, 0).to(DEV), WL.initial_err(w).to(DEV)
+    PT.compare_all(ctx, grads, err, w.K, label=f"[checked {name}] ")
+    assert ctx.debug_status() == 0
+    assert ctx.debug_status() == 0             # reading clears; still nothing
+    # the normal build answers 0 whatever happened
+    plain = B.MvContext(w.N, w.d, w.K, device=DEV)
+    PT.run_step(plain, grads, err, w.K)
+    assert plain.debug_status() == 0
+
+
+def test_checked_build_reports_the_fallback_and_the_overflow():
+    """Valid inputs that take the slow but exact routes: a jump of scale under threshold tracking (the
+    carried threshold admits every element: candidate overflow, then the full-row select) and a row of
+    equal magnitudes.  The results are the oracle's; the status word names the detours and nothing else."""
+    N, d, K = 3, 300_007, 3000
+    ctx = _debug_context(N, d, K, mode=B.MV_MODE_TRACK)
+    grads, err = make(N, d, "gauss", seed=77)
+    seen = []
+    for step, sc in enumerate([1.0, 1.0, 1e3, 1e3]):
+        g, e = (grads * sc).roll(step, dims=1).contiguous(), (err * sc).contiguous()
+        ref = O.mv_sparse_step(g.numpy(), e.numpy(), K)
+        fu = PT.run_step(ctx, g.to(DEV), e.to(DEV), K)
+        PT.first_diff(PT.npy(fu["out_idx"]), ref["out_idx"], f"step {step} out_idx")
+        PT.first_diff(PT.bits(PT.npy(fu["err"])), PT.bits(ref["err"]), f"step {step} err")
+        seen.append(ctx.debug_status())
+    assert seen[0] == 0 and seen[1] == 0 and seen[3] == 0
+    assert seen[2] == B.MV_DBG_CAND_OVERFLOW | B.MV_DBG_FALLBACK
+    # equal magnitudes: every element is a candidate of the sampled threshold
+    g2, e2 = make(N, d, "equal", seed=1)
+    ctx.set_mode(B.MV_MODE_AUTO)
+    PT.compare_all(ctx, g2.to(DEV), e2.to(DEV), K, label="[checked equal] ")
+    assert ctx.debug_status() == B.MV_DBG_CAND_OVERFLOW | B.MV_DBG_FALLBACK
+    # an index list that is not one: mv_aggregate refuses the entries outside [0, d) and says so
+    idx = torch.tensor([5, -1, d, 7], dtype=torch.int32, device=DEV)
+    val = torch.full((4,), float("nan"), device=DEV)
+    acc = g2.to(DEV).clone()
+    ctx.mv_aggregate(acc, idx, val)
+    torch.cuda.synchronize()
+    assert ctx.debug_status() == B.MV_DBG_GATHER_RANGE
+    assert val.cpu().tolist()[1:3] == [0.0, 0.0]

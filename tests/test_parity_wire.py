@@ -66,6 +66,29 @@ def test_clustered_and_edge_positions():
         assert result.tolist()[:3] == [idx.size, 1001, 0] and np.array_equal(got_idx, idx)
 
 
+def test_encoder_skips_entries_that_are_not_coordinates():
+    """A list padded with -1 (what mv_select_rs leaves when fewer than K coordinates hold a vote), or
+    holding an index >= d, must write nothing outside the stream: the valid entries land where the
+    oracle puts them for the list without the padding, every other bit stays zero."""
+    d, Bk = 100_003, 100
+    rng = np.random.default_rng(5)
+    good = random_support(rng, d, 700)
+    for tail in (np.full(300, -1, np.int32), np.array([d, d + 5, 2**31 - 1, -2**31], np.int64).astype(np.int32)):
+        padded = np.concatenate([good, tail]).astype(np.int32)
+        guard = torch.full((4096,), 0x5A5A5A5A, dtype=torch.int32, device=DEV)      # the stream sits in the middle
+        nbits = B.pos_stream_bits(d, Bk, padded.size)
+        nw = (nbits + 31) // 32
+        words = guard[1024:1024 + nw]
+        assert nw < 2048
+        B.mv_pos_encode(torch.from_numpy(padded).to(DEV), d, Bk, words)
+        torch.cuda.synchronize()
+        g = guard.cpu().numpy().view(np.uint32)
+        assert np.all(g[:1024] == 0x5A5A5A5A) and np.all(g[1024 + nw:] == 0x5A5A5A5A), "wrote outside the stream"
+        want = W.encode_positions(good, d, Bk)
+        got = g[1024:1024 + nw]
+        assert np.array_equal(got[:want.size], want) and not got[want.size:].any()
+
+
 def test_decoder_reads_an_oracle_stream_and_reports_malformed_ones():
     d, Bk, K = 50_000, 128, 3000
     rng = np.random.default_rng(5)

@@ -4,8 +4,9 @@ Some users of this library run where cudaMalloc is off limits (a real-time loop,
 host forbids allocation after start-up, a process whose memory pool is fully handed out), so they
 cannot provide the workspace that mv_create wants.  mv_select_static keeps its scratch in an array
 compiled into the library instead.  These tests call it through the C ABI and require the same bytes
-as mv_select gives, on two calls in a row (the array keeps the first call's leftovers, which the
-second call must not see), and check that a size beyond the array's limit is refused.
+as mv_select gives -- and as the CPU oracle's S_top over the votes gives -- on two calls in a row (the
+array keeps the first call's leftovers, which the second call must not see), at the largest size the
+array is built for, and check that a size beyond that limit is refused.
 
 This file is named so that pytest collects it last.
 """
@@ -15,6 +16,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import mv_oracle as O
 from paper_2011_06495_b200 import binding as B
 
 pytestmark = pytest.mark.gpu
@@ -53,6 +55,10 @@ def test_two_calls_in_a_row_match_mv_select():
         ref_idx, ref_bits, got_idx, got_bits = _both(votes, N, K)
         assert torch.equal(got_idx, ref_idx), f"out_idx differs for N={N} d={d} K={K}"
         assert torch.equal(got_bits, ref_bits), f"mask_bits differs for N={N} d={d} K={K}"
+        # the oracle's selection over the same votes (Eq. 9, outer S_top; ties to the lowest index)
+        want_idx = O.select_mask(votes.cpu().numpy(), K)[0]
+        assert np.array_equal(got_idx.cpu().numpy(), want_idx), f"out_idx differs from the oracle for N={N} d={d} K={K}"
+        assert np.array_equal(got_bits.cpu().numpy().view(np.uint32), O.support_to_bits(want_idx, d))
         # and both are right: K strictly ascending indices, every chosen vote >= every other vote
         idx = got_idx.cpu().numpy().astype(np.int64)
         v = votes.cpu().numpy()
@@ -60,6 +66,18 @@ def test_two_calls_in_a_row_match_mv_select():
         inside = np.zeros(d, bool)
         inside[idx] = True
         assert v[inside].min() >= v[~inside].max()
+
+
+def test_largest_size_the_array_is_built_for():
+    """d = MV_SELECT_STATIC_MAX_D exactly (every per-chunk slot of the array in use), twice in a row with
+    different votes, against mv_select and against the oracle."""
+    d = B.MV_SELECT_STATIC_MAX_D
+    for N, K, dense, seed in [(64, d // 100, False, 11), (3, 4194, True, 12)]:
+        votes = _votes(d, N, seed, dense)
+        ref_idx, ref_bits, got_idx, got_bits = _both(votes, N, K)
+        assert torch.equal(got_idx, ref_idx) and torch.equal(got_bits, ref_bits)
+        want_idx = O.select_mask(votes.cpu().numpy(), K)[0]
+        assert np.array_equal(got_idx.cpu().numpy(), want_idx), f"out_idx differs from the oracle for N={N} K={K}"
 
 
 def test_mask_may_be_omitted_and_small_inputs_work():
