@@ -48,7 +48,11 @@ enum {
   MV_ERR_INVALID_ARG = -1, /* null or misaligned pointer, N/d/K out of range, grads aliasing err */
   MV_ERR_WORKSPACE = -2,   /* workspace smaller than mv_workspace_bytes(N, d, K) */
   MV_ERR_CUDA = -3,        /* the CUDA runtime refused a launch or a copy */
-  MV_ERR_TOO_LARGE = -4    /* mv_select_static only: d is larger than MV_SELECT_STATIC_MAX_D */
+  MV_ERR_TOO_LARGE = -4,   /* mv_select_static only: d is larger than MV_SELECT_STATIC_MAX_D */
+  MV_ERR_TIMEOUT = -5      /* a bounded wait between the CTAs of a kernel gave up (never expected: the kernel that
+                              waits is launched so that all its CTAs run together); the results of that call and
+                              of later calls on the context are not valid.  Reported by the calls that wait for
+                              the stream: mv_sparse_step_host, mv_read_diag, mv_fallback_count, mv_debug_status */
 };
 
 enum {
@@ -96,6 +100,17 @@ int mv_destroy(mv_ctx* ctx);
 
 /* Chooses how the per-worker threshold is found (MV_MODE_*).  Results are identical. */
 int mv_set_mode(mv_ctx* ctx, int mode);
+
+/* How mv_sparse_step runs what follows its pass over grads and err (S_top from the candidates on, the votes of
+ * Eq. 9, the shared mask, the aggregate of Eq. 8 and the residual): either as the sequence of kernels that mv_vote,
+ * mv_select and mv_aggregate use, or as ONE kernel whose CTAs (one per multiprocessor, launched cooperatively) stay
+ * resident and meet at grid barriers.  The single kernel can run when the device supports cooperative launches,
+ * N is at most the number of multiprocessors, d <= 8192 * 4096 and the mode is not MV_MODE_GENERAL.
+ *   enable = 1 (default): the single kernel where it can run and K >= 65536 (many picks and outputs: there it is
+ *                         faster), the sequence otherwise;  0: always the sequence;  2: the single kernel wherever
+ *                         it can run.
+ * The bytes of every result are the same either way.  The barrier waits are bounded: see MV_ERR_TIMEOUT. */
+int mv_set_tail_kernel(mv_ctx* ctx, int enable);
 
 /* The whole step (Algorithm 1 from the accumulate line to the aggregate line).
  *   grads   [N*d] in      the workers' model differences / gradients

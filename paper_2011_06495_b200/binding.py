@@ -22,6 +22,7 @@ MV_ERR_INVALID_ARG = -1
 MV_ERR_WORKSPACE = -2
 MV_ERR_CUDA = -3
 MV_ERR_TOO_LARGE = -4
+MV_ERR_TIMEOUT = -5
 MV_SELECT_STATIC_MAX_D = 1 << 24
 MV_MODE_AUTO = 0
 MV_MODE_GENERAL = 1
@@ -125,6 +126,8 @@ def _open(path: str, how: str) -> ctypes.CDLL:
     lib.mv_quantize.argtypes = [c_vp, c_vp, c_i64, c_i, c_vp, c_vp, c_vp, c_sz]
     lib.mv_dequantize.restype = c_i
     lib.mv_dequantize.argtypes = [c_vp, c_vp, c_i64, c_i, c_vp]
+    lib.mv_set_tail_kernel.restype = c_i
+    lib.mv_set_tail_kernel.argtypes = [c_vp, c_i]
     lib.mv_fallback_count.restype = c_i
     lib.mv_fallback_count.argtypes = [c_vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.mv_debug_status.restype = c_i
@@ -233,6 +236,11 @@ class MvContext:
             self.close()
         except Exception:
             pass
+
+    def set_tail_kernel(self, enable: int):
+        """Whole steps as two kernels (streaming pass + one persistent tail kernel): 0 never, 1 where it pays
+        (the default), 2 wherever it can run."""
+        _check(self.lib.mv_set_tail_kernel(self.handle, int(enable)), "mv_set_tail_kernel")
 
     def set_mode(self, mode: int):
         _check(self.lib.mv_set_mode(self.handle, int(mode)), "mv_set_mode")

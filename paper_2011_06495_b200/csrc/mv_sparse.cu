@@ -33,6 +33,7 @@
 #include <cuda_runtime.h>
 #include <cooperative_groups.h>
 #include <stdint.h>
+#include <stdio.h>
 #include <stdlib.h>
 #include <math.h>
 #include <mutex>
@@ -999,9 +1000,116 @@ __device__ __forceinline__ void put_bits(const P& p, int n, uint32_t w, uint32_t
   }
 }
 
+// The picks of a worker whose K-th key was found over its full row, read off the row itself (err holds acc):
+// every element above T_n, and the threshold ties -- all of them, or (ordered = !all_ties) those whose rank in
+// index order over the whole row, tie_base[chunk] + rank inside the chunk, is below `need`.  The calling CTA has
+// NSUB x 256 threads; each group of 256 takes one chunk at a time: chunks c_first + sub, + c_stride, ...
+// All threads of the CTA must call it (it synchronises the CTA).
+template <int NSUB>
+__device__ __forceinline__ void fullrow_picks(const P& p, int n, float* __restrict__ err, uint32_t T, uint32_t need,
+                                              bool all_ties, int c_first, int c_stride, uint32_t (*s_we)[9]) {
+  uint32_t* bits_row = p.worker_bits + (size_t)n * p.W;
+  const int sub = threadIdx.x >> 8, t = threadIdx.x & 255;
+  const int warp = t >> 5, lane = t & 31;
+  const uint32_t lt = lanemask_lt();
+  for (int c0 = c_first; c0 < p.nchunks; c0 += c_stride) {  // uniform over the CTA
+    const int c = c0 + sub;
+    const bool valid = c < p.nchunks;
+    Geom g = chunk_geom(n, valid ? c : 0, p.d);
+    uint32_t key[4][4], vm[4], em[4], sm[4];
+    uint32_t xkey[4] = {0, 0, 0, 0}, xvm = 0, xem = 0, xsm = 0;
+    if (valid) {
+      load_keys<false>(g, nullptr, err, key, vm, t);
+      if (t == TPB - 1) {
+        load_extra<false>(g, nullptr, err, xkey, xvm);
+        xem = xvm & eq_mask(xkey, T);
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < 4; i++) {
+        vm[i] = 0;
+        key[i][0] = key[i][1] = key[i][2] = key[i][3] = 0;
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; i++) em[i] = vm[i] & eq_mask(key[i], T);
+    if (all_ties) {
+#pragma unroll
+      for (int i = 0; i < 4; i++) sm[i] = (vm[i] & gt_mask(key[i], T)) | em[i];
+      if (t == TPB - 1) xsm = (xvm & gt_mask(xkey, T)) | xem;
+    } else {
+      // keep the threshold ties whose rank (in index order, over the whole row) is below `need`
+      uint32_t weq = 0;
+#pragma unroll
+      for (int i = 0; i < 4; i++) weq += __popc(em[i]);
+      weq = __reduce_add_sync(FULL, weq);
+      __syncthreads();  // previous chunk's readers of s_we are done
+      if (lane == 0) s_we[sub][warp] = weq;
+      if (t == TPB - 1) s_we[sub][8] = __popc(xem);
+      __syncthreads();
+      const uint32_t tb = valid ? p.tie_base[(size_t)n * p.nchunks + c] : 0u;
+      uint32_t eoff = tb;
+      for (int w = 0; w < warp; w++) eoff += s_we[sub][w];
+#pragma unroll
+      for (int i = 0; i < 4; i++) {
+        uint32_t rank0, tot;
+        iter_ranks(em[i], lt, rank0, tot);
+        uint32_t take = 0;
+#pragma unroll
+        for (int e = 0; e < 4; e++) {
+          if (em[i] & (1u << e)) {
+            const uint32_t r = eoff + rank0 + __popc(em[i] & ((1u << e) - 1u));
+            if (r < need) take |= 1u << e;
+          }
+        }
+        sm[i] = (vm[i] & gt_mask(key[i], T)) | take;
+        eoff += tot;
+      }
+      if (t == TPB - 1) {
+        uint32_t xoff = tb;
+        for (int w = 0; w < 8; w++) xoff += s_we[sub][w];
+        uint32_t take = 0;
+#pragma unroll
+        for (int e = 0; e < 4; e++) {
+          if (xem & (1u << e)) {
+            const uint32_t r = xoff + __popc(xem & ((1u << e) - 1u));
+            if (r < need) take |= 1u << e;
+          }
+        }
+        xsm = (xvm & gt_mask(xkey, T)) | take;
+      }
+    }
+    bool any = false;
+#pragma unroll
+    for (int i = 0; i < 4; i++) {
+      if (sm[i]) {
+        any = true;
+        const int jf = g.j0 - g.h + 4 * (warp * 128 + i * 32 + lane);
+#pragma unroll
+        for (int e = 0; e < 4; e++)
+          if (sm[i] & (1u << e)) {
+            if (!p.no_masks) atomicOr(bits_row + ((uint32_t)(jf + e) >> 5), 1u << ((uint32_t)(jf + e) & 31u));
+            if (p.vote_words) add_vote(p.vote_words, (uint32_t)(jf + e));
+          }
+      }
+    }
+    if (xsm) {
+      any = true;
+      const int jf = g.j0 - g.h + 4096;
+#pragma unroll
+      for (int e = 0; e < 4; e++)
+        if (xsm & (1u << e)) {
+          if (!p.no_masks) atomicOr(bits_row + ((uint32_t)(jf + e) >> 5), 1u << ((uint32_t)(jf + e) & 31u));
+          if (p.vote_words) add_vote(p.vote_words, (uint32_t)(jf + e));
+        }
+    }
+    if (any && valid) p.hot[c] = 1;  // same value from every thread
+  }
+}
+
 __global__ void __launch_bounds__(TPB) k_set_bits(P p, float* __restrict__ err) {
   pdl_enter();
-  __shared__ uint32_t s_we[9];
+  __shared__ uint32_t s_we[1][9];
   const int n = blockIdx.y;
   const bool fast = worker_fast(p, n);
   if (p.list_mode && !fast) {  // empty list
@@ -1015,95 +1123,10 @@ __global__ void __launch_bounds__(TPB) k_set_bits(P p, float* __restrict__ err) 
   const uint32_t* ws = p.wstate + (size_t)n * 8;
   const uint32_t T = ws[4], need = ws[7];
   const bool all_ties = need >= ws[6];
-  uint32_t* bits_row = p.worker_bits + (size_t)n * p.W;
   if (blockIdx.x == 0 && threadIdx.x == 0) p.diag_cnt[n] = p.cand_cnt[n];
   if (!fast) {
     // full-row worker: its picks are read off the row itself (err holds acc), chunk by chunk
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t lt = lanemask_lt();
-    for (int c = blockIdx.x; c < p.nchunks; c += gridDim.x) {
-      const Geom g = chunk_geom(n, c, p.d);
-      uint32_t key[4][4], vm[4], em[4], sm[4];
-      load_keys<false>(g, nullptr, err, key, vm);
-      uint32_t xkey[4], xvm = 0, xem = 0, xsm = 0;
-      if (threadIdx.x == TPB - 1) {
-        load_extra<false>(g, nullptr, err, xkey, xvm);
-        xem = xvm & eq_mask(xkey, T);
-      }
-#pragma unroll
-      for (int i = 0; i < 4; i++) em[i] = vm[i] & eq_mask(key[i], T);
-      if (all_ties) {
-#pragma unroll
-        for (int i = 0; i < 4; i++) sm[i] = (vm[i] & gt_mask(key[i], T)) | em[i];
-        if (threadIdx.x == TPB - 1) xsm = (xvm & gt_mask(xkey, T)) | xem;
-      } else {
-        // keep the threshold ties whose rank (in index order, over the whole row) is below `need`
-        uint32_t weq = 0;
-#pragma unroll
-        for (int i = 0; i < 4; i++) weq += __popc(em[i]);
-        weq = __reduce_add_sync(FULL, weq);
-        __syncthreads();  // previous chunk's readers of s_we are done
-        if (lane == 0) s_we[warp] = weq;
-        if (threadIdx.x == TPB - 1) s_we[8] = __popc(xem);
-        __syncthreads();
-        const uint32_t tb = p.tie_base[(size_t)n * p.nchunks + c];
-        uint32_t eoff = tb;
-        for (int w = 0; w < warp; w++) eoff += s_we[w];
-#pragma unroll
-        for (int i = 0; i < 4; i++) {
-          uint32_t rank0, tot;
-          iter_ranks(em[i], lt, rank0, tot);
-          uint32_t take = 0;
-#pragma unroll
-          for (int e = 0; e < 4; e++) {
-            if (em[i] & (1u << e)) {
-              const uint32_t r = eoff + rank0 + __popc(em[i] & ((1u << e) - 1u));
-              if (r < need) take |= 1u << e;
-            }
-          }
-          sm[i] = (vm[i] & gt_mask(key[i], T)) | take;
-          eoff += tot;
-        }
-        if (threadIdx.x == TPB - 1) {
-          uint32_t xoff = tb;
-          for (int w = 0; w < 8; w++) xoff += s_we[w];
-          uint32_t take = 0;
-#pragma unroll
-          for (int e = 0; e < 4; e++) {
-            if (xem & (1u << e)) {
-              const uint32_t r = xoff + __popc(xem & ((1u << e) - 1u));
-              if (r < need) take |= 1u << e;
-            }
-          }
-          xsm = (xvm & gt_mask(xkey, T)) | take;
-        }
-      }
-      bool any = false;
-#pragma unroll
-      for (int i = 0; i < 4; i++) {
-        if (sm[i]) {
-          any = true;
-          const int jf = g.j0 - g.h + 4 * (warp * 128 + i * 32 + lane);
-#pragma unroll
-          for (int e = 0; e < 4; e++)
-            if (sm[i] & (1u << e)) {
-              if (!p.no_masks) atomicOr(bits_row + ((uint32_t)(jf + e) >> 5), 1u << ((uint32_t)(jf + e) & 31u));
-              if (p.vote_words) add_vote(p.vote_words, (uint32_t)(jf + e));
-            }
-        }
-      }
-      if (xsm) {
-        any = true;
-        const int jf = g.j0 - g.h + 4096;
-#pragma unroll
-        for (int e = 0; e < 4; e++)
-          if (xsm & (1u << e)) {
-            if (!p.no_masks) atomicOr(bits_row + ((uint32_t)(jf + e) >> 5), 1u << ((uint32_t)(jf + e) & 31u));
-            if (p.vote_words) add_vote(p.vote_words, (uint32_t)(jf + e));
-          }
-      }
-      if (any) p.hot[c] = 1;  // same value from every thread
-    }
+    fullrow_picks<1>(p, n, err, T, need, all_ties, blockIdx.x, gridDim.x, s_we);
     return;
   }
   const uint32_t cnt = p.cand_cnt[n];
@@ -1892,8 +1915,66 @@ __global__ void __launch_bounds__(TPB) k_vote_write(P p, const uint8_t* __restri
 // ---------------------------------------------------------------------------------------------
 // aggregate: out_val[k] = fl32( (sum_n (double)acc[n][idx[k]]) / N ), then acc[n][idx[k]] = +0
 // ---------------------------------------------------------------------------------------------
+// One output of the aggregate.  G = lanes that share the coordinate: 1, or 8 (lane g then loads rows g, g + 8,
+// ..., so that a coordinate's N scattered loads are in flight together even with many workers).  The sum is the
+// same sequence of binary64 additions in worker order either way: with G = 8 the values are passed to it by
+// shuffles, so all 32 lanes of a warp must call together (`live` = false for lanes without an output).
+template <int G>
+__device__ __forceinline__ void gather_one(float* __restrict__ acc, int N, int64_t d, int64_t k, bool live, int g,
+                                           const int32_t* __restrict__ idx, float* __restrict__ out_val,
+                                           double* __restrict__ out_sum, uint32_t* __restrict__ dbg) {
+  const int64_t j = live ? (int64_t)__ldcg(idx + k) : -1;  // (from L2: the index may have been written by this very kernel)
+  const bool bad = j < 0 || j >= d;
+  if (live && bad && g == 0) {
+    MV_DBG(dbg, MV_DBG_GATHER_RANGE);
+    if (out_sum) out_sum[k] = 0.0;
+    else out_val[k] = 0.f;
+  }
+  if (G == 1 && bad) return;
+  float* col = acc + (bad ? 0 : j);
+  // all loads before any store: a store to acc followed by a load from acc (another row) would
+  // otherwise be kept in program order and serialise the memory latency row by row
+  double s = 0.0;
+  if (G == 1) {
+    for (int n0 = 0; n0 < N; n0 += 16) {
+      float v[16];
+#pragma unroll
+      for (int q = 0; q < 16; q++) v[q] = n0 + q < N ? __ldcg(col + (size_t)(n0 + q) * (size_t)d) : 0.f;
+#pragma unroll
+      for (int q = 0; q < 16; q++)
+        if (n0 + q < N) s += (double)v[q];
+    }
+    for (int n = 0; n < N; n++) __stcg(col + (size_t)n * (size_t)d, 0.0f);
+  } else {
+    const int lane = threadIdx.x & 31, gbase = lane - g;
+    for (int n0 = 0; n0 < N; n0 += 4 * G) {  // uniform over the warp
+      float v[4];
+#pragma unroll
+      for (int q = 0; q < 4; q++) {
+        const int n = n0 + q * G + g;
+        v[q] = (!bad && n < N) ? __ldcg(col + (size_t)n * (size_t)d) : 0.f;
+      }
+#pragma unroll
+      for (int q = 0; q < 4; q++)
+#pragma unroll
+        for (int h = 0; h < G; h++) {  // workers n0 + q G + h, in this order
+          const float x = __shfl_sync(FULL, v[q], gbase + h);
+          if (n0 + q * G + h < N) s += (double)x;
+        }
+    }
+    if (bad) return;
+    for (int n = g; n < N; n += G) __stcg(col + (size_t)n * (size_t)d, 0.0f);
+    if (g != 0) return;
+  }
+  // a rank that holds only some of the workers hands back its binary64 partial sum instead
+  if (out_sum) out_sum[k] = s;
+  else out_val[k] = (float)(s / (double)N);
+}
+
 // The last kernel of a whole step also clears the leading scratch region (counters and histograms)
 // so that the next step can start without a separate memset; zero_vecs = 0 switches that off.
+// G = 8 when K is small: the grid is then eight times larger.
+template <int G>
 __global__ void __launch_bounds__(TPB) k_gather(float* __restrict__ acc, int N, int64_t d, int64_t K,
                                                 const int32_t* __restrict__ idx, float* __restrict__ out_val,
                                                 uint4* __restrict__ zero_ptr, uint32_t zero_vecs,
@@ -1901,31 +1982,10 @@ __global__ void __launch_bounds__(TPB) k_gather(float* __restrict__ acc, int N, 
   pdl_enter();
   for (uint32_t i = blockIdx.x * TPB + threadIdx.x; i < zero_vecs; i += gridDim.x * TPB)
     zero_ptr[i] = make_uint4(0, 0, 0, 0);
-  const int64_t k = (int64_t)blockIdx.x * TPB + threadIdx.x;
-  if (k >= K) return;
-  const int64_t j = idx[k];
-  if (j < 0 || j >= d) {
-    MV_DBG(dbg, MV_DBG_GATHER_RANGE);
-    if (out_sum) out_sum[k] = 0.0;
-    else out_val[k] = 0.f;
-    return;
-  }
-  float* col = acc + j;
-  // all loads before any store: a store to acc followed by a load from acc (another row) would
-  // otherwise be kept in program order and serialise the memory latency row by row
-  double s = 0.0;
-  for (int n0 = 0; n0 < N; n0 += 16) {
-    float v[16];
-#pragma unroll
-    for (int q = 0; q < 16; q++) v[q] = n0 + q < N ? __ldcg(col + (size_t)(n0 + q) * (size_t)d) : 0.f;
-#pragma unroll
-    for (int q = 0; q < 16; q++)
-      if (n0 + q < N) s += (double)v[q];
-  }
-  for (int n = 0; n < N; n++) __stcg(col + (size_t)n * (size_t)d, 0.0f);
-  // a rank that holds only some of the workers hands back its binary64 partial sum instead
-  if (out_sum) out_sum[k] = s;
-  else out_val[k] = (float)(s / (double)N);
+  const int64_t t = (int64_t)blockIdx.x * TPB + threadIdx.x;
+  const int64_t k = t / G;
+  if (G == 1 && k >= K) return;
+  gather_one<G>(acc, N, d, k, k < K, (int)(t % G), idx, out_val, out_sum, dbg);
 }
 
 // worker-sharded step: mean over all workers from the summed partial sums
@@ -2177,6 +2237,9 @@ __global__ void __launch_bounds__(TPB) k_ad_apply(uint32_t* __restrict__ prev_bi
   }
 }
 
+#include "mv_tail.cuh"
+static_assert(F_RADIX <= SB_BINS, "the three-digit counts live in the sample histogram's rows");
+
 // ---------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------
@@ -2185,7 +2248,9 @@ struct Layout {
   int64_t W;
   uint32_t cap;
   size_t dbg;         // header, at the start of the workspace whatever the sizes: word 0 the checked build's status
-  size_t fb_total;    // word, word 1 the running count of full-row selections
+  size_t fb_total;    // word, word 1 the running count of full-row selections, word 2 set for good once a bounded
+  size_t abort_flag;  // device-side wait has given up (MV_ERR_TIMEOUT)
+  size_t tail_words;  // [16] grid barrier, exit ticket and flags of the single-kernel tail (in the cleared region)
   size_t zero_off;    // start of ...
   size_t zero_bytes;  // ... the region that is clear at the start of every vote
   size_t samp_hist, hist1, hist2, hist2b, hist3, cand_cnt, sample_done, count_done, votes_done, hot, vote_hist;
@@ -2219,8 +2284,9 @@ Layout make_layout(int N, int64_t d, int64_t K) {
   L.cap = (uint32_t)((cap + 7) & ~(int64_t)7);  // multiple of 8: every worker's buffer is 64-byte aligned
   size_t off = 0;
   const size_t n = (size_t)N, nc = (size_t)L.nchunks;
-  L.dbg = take(off, 8);
+  L.dbg = take(off, 12);
   L.fb_total = L.dbg + 4;
+  L.abort_flag = L.dbg + 8;
   L.zero_off = off;
   L.samp_hist = take(off, n * SB_BINS * 4);
   L.hist1 = take(off, n * H1_BINS * 4);
@@ -2233,6 +2299,7 @@ Layout make_layout(int N, int64_t d, int64_t K) {
   L.hot = take(off, (size_t)((L.nchunks + 7) & ~7));
   L.votes_done = take(off, 4);
   L.vote_hist = take(off, 256 * 4);
+  L.tail_words = take(off, 16 * 4);
   L.zero_bytes = off - L.zero_off;
   L.tau = take(off, n * 4);
   L.tau_alt = take(off, n * 4);
@@ -2308,6 +2375,9 @@ struct mv_ctx {
   int sms;             // multiprocessors of the workspace's device (0 = not asked yet)
   int cta_budget;      // the largest multiple of 8 CTAs that is not above sms: one CTA per SM for the cluster select
   bool dbg_ready;      // the workspace's header has been cleared once
+  int tail_state;      // single-kernel tail: 0 = not tried, 1 = usable on this device, -1 = not
+  int tail_mode;       // (mv_set_tail_kernel) 0 = never, 1 = where it pays, 2 = wherever it can run
+  int tail_pdl;        // -1: the runtime refused a cooperative launch with programmatic stream serialisation
   // remembered for mv_read_diag
   int last_N;
   int64_t last_d, last_K;
@@ -2388,7 +2458,7 @@ int device_ready(mv_ctx* ctx) {
     ctx->cta_budget = sms >= 8 ? sms - sms % 8 : 8;
   }
   if (!ctx->dbg_ready) {
-    if (cudaMemsetAsync(ctx->ws, 0, 8, ctx->stream) != cudaSuccess) return MV_ERR_CUDA;
+    if (cudaMemsetAsync(ctx->ws, 0, 12, ctx->stream) != cudaSuccess) return MV_ERR_CUDA;
     ctx->dbg_ready = true;
   }
   return MV_OK;
@@ -2508,8 +2578,11 @@ int join_side(mv_ctx* ctx) {
 // `need_hist` = false: the per-chunk vote histograms and offsets are not wanted (the caller selects by other means)
 // `want_lists` = false: the ascending per-worker index lists are not wanted (nothing later in a step reads them)
 // `want_masks` = false: nor are the workers' bit masks (unless the lists, which are built from them, are)
+// `stream_only`: stop after the streaming pass (the single-kernel tail follows); *p_out gets the parameters as
+// completed here (thresholds of this and the next call, vote array)
 int vote_impl(mv_ctx* ctx, P p, const Layout& L, const float* grads, float* err, bool topk_only = false,
-              bool need_hist = true, bool want_lists = true, bool want_masks = true) {
+              bool need_hist = true, bool want_lists = true, bool want_masks = true, bool stream_only = false,
+              P* p_out = nullptr) {
   cudaStream_t st = ctx->stream;
   const int N = p.N;
   const int SMS = ctx->sms, CTA_BUDGET = ctx->cta_budget;
@@ -2569,6 +2642,10 @@ int vote_impl(mv_ctx* ctx, P p, const Layout& L, const float* grads, float* err,
     launch_k(k_acc_compact, dim3(dim3(p.nchunks, N)), dim3(TPB), st, p, grads, err);
     MV_LAUNCH_CHECK();
     if (ctx->timing_now) cudaEventRecord(ctx->ev[2 * (ctx->timed++ % 64) + 1], st);
+    if (stream_only) {
+      if (p_out) *p_out = p;
+      return MV_OK;
+    }
     if (!cluster_select_ready()) return MV_ERR_CUDA;
     // a cluster per worker resolves T_n, sets the worker's mask bits and adds its votes
     // (with few workers, extra clusters that only help clearing fill the GPU)
@@ -2675,12 +2752,109 @@ int select_impl(mv_ctx* ctx, P p, const Layout& L, const uint8_t* votes, bool ha
 int aggregate_impl(mv_ctx* ctx, float* acc, int N, int64_t d, int64_t K, const int32_t* idx, float* out_val,
                    size_t clear_bytes, double* out_sum = nullptr) {
   const Layout L0 = make_layout(1, 1, 1);  // (the cleared region starts at the same offset for every size)
-  launch_k(k_gather, dim3((unsigned)((K + TPB - 1) / TPB)), dim3(TPB), ctx->stream, acc, N, d, K, idx, out_val,
-           (uint4*)(ctx->ws + L0.zero_off), (uint32_t)(clear_bytes / 16), out_sum,
-           kChecked ? (uint32_t*)(ctx->ws + L0.dbg) : (uint32_t*)nullptr);
+  uint4* const zp = (uint4*)(ctx->ws + L0.zero_off);
+  uint32_t* const dbg = kChecked ? (uint32_t*)(ctx->ws + L0.dbg) : (uint32_t*)nullptr;
+  // few coordinates, several workers: eight lanes per coordinate keep the scattered loads in flight together
+  if (K <= 65536 && N >= 4)
+    launch_k(k_gather<8>, dim3((unsigned)((K * 8 + TPB - 1) / TPB)), dim3(TPB), ctx->stream, acc, N, d, K, idx, out_val, zp,
+             (uint32_t)(clear_bytes / 16), out_sum, dbg);
+  else
+    launch_k(k_gather<1>, dim3((unsigned)((K + TPB - 1) / TPB)), dim3(TPB), ctx->stream, acc, N, d, K, idx, out_val, zp,
+             (uint32_t)(clear_bytes / 16), out_sum, dbg);
   MV_LAUNCH_CHECK();
   if (clear_bytes) ctx->clean_bytes = clear_bytes;
   return MV_OK;
+}
+
+// The single-kernel tail needs a cooperative launch with one CTA of FT threads and SK_KEYS keys of shared memory
+// per multiprocessor; asked once per context.
+bool tail_ready(mv_ctx* ctx) {
+  if (ctx->tail_state == 0) {
+    ctx->tail_state = -1;
+    int dev = -1, coop = 0, per_sm = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) == cudaSuccess &&
+        coop != 0 &&
+        cudaFuncSetAttribute(k_tail, cudaFuncAttributeMaxDynamicSharedMemorySize, SK_KEYS * 4) == cudaSuccess &&
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_tail, FT, SK_KEYS * 4) == cudaSuccess && per_sm >= 1)
+      ctx->tail_state = 1;
+    else
+      cudaGetLastError();
+  }
+  return ctx->tail_state == 1;
+}
+
+// Do this call's steps after the streaming pass run as the single kernel?  It can when the mode is not the general
+// one, every worker gets a CTA of its own and the chunks' output offsets fit its shared-memory table.  It pays
+// (measured: some microseconds per step) when there are many picks to make and outputs to gather, K >= 2^16; with
+// a small K the steps are all latency, and the separate kernels, each launched while its predecessor still runs,
+// are as fast or faster.
+bool tail_usable(mv_ctx* ctx, const Layout& L, int N, int64_t K) {
+  if (ctx->tail_mode == 0 || (ctx->tail_mode == 1 && K < 65536)) return false;
+  return ctx->mode != MV_MODE_GENERAL && N <= ctx->sms && ((L.nchunks + 7) & ~7) <= F_MAXCH && tail_ready(ctx);
+}
+
+// steps a2 (from the candidates on) to a6 as one cooperative kernel; p: the parameters as vote_impl completed them
+int tail_impl(mv_ctx* ctx, const P& p, const Layout& L, float* err, int32_t* out_idx, float* out_val) {
+  char* b = ctx->ws;
+  TailArgs a;
+  a.err = err;
+  a.out_idx = out_idx;
+  a.out_val = out_val;
+  a.words = (uint32_t*)(b + L.tail_words);
+  a.abort_flag = (uint32_t*)(b + L.abort_flag);
+  a.radix = (uint32_t*)(b + L.samp_hist);  // (N x SB_BINS words, free once the thresholds are known; F_RADIX <= SB_BINS)
+  a.zero_ptr = (uint4*)(b + L.zero_off);
+  a.zero_vecs = (uint32_t)((L.votes_done - L.zero_off) / 16);
+  a.last_zero = (uint32_t*)(b + L.votes_done);
+  a.last_zero_words = (uint32_t)((L.zero_off + L.zero_bytes - L.votes_done) / 4);
+  a.spin_limit = 1u << 21;
+  a.dbg = p.dbg;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)ctx->sms);
+  cfg.blockDim = dim3(FT);
+  cfg.dynamicSmemBytes = SK_KEYS * 4;
+  cfg.stream = ctx->stream;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeCooperative;
+  attr[0].val.cooperative = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  // launched early like the other kernels (it waits for the streaming pass at its start) if the runtime takes a
+  // cooperative launch that way; otherwise as a plain cooperative launch
+  cfg.numAttrs = ctx->tail_pdl >= 0 ? 2 : 1;
+  cudaError_t le = cudaLaunchKernelEx(&cfg, k_tail, p, a);
+  if (le != cudaSuccess && cfg.numAttrs == 2) {
+    cudaGetLastError();
+    ctx->tail_pdl = -1;
+    cfg.numAttrs = 1;
+    le = cudaLaunchKernelEx(&cfg, k_tail, p, a);
+  }
+  if (le != cudaSuccess) {
+    cudaGetLastError();
+    return MV_ERR_CUDA;
+  }
+#ifdef MV_TAIL_STAMPS
+  {
+    static bool told = false;
+    if (!told) {
+      told = true;
+      fprintf(stderr, "tail kernel launched with %d attribute(s)\n", (int)cfg.numAttrs);
+    }
+  }
+#endif
+  MV_LAUNCH_CHECK();
+  ctx->clean_bytes = L.zero_bytes;
+  return MV_OK;
+}
+
+// has a bounded device-side wait given up on this context?  (reads the workspace header; the stream must be idle)
+int abort_status(mv_ctx* ctx) {
+  if (!ctx->dbg_ready) return MV_OK;
+  uint32_t flag = 0;
+  if (cudaMemcpyAsync(&flag, ctx->ws + 8, 4, cudaMemcpyDeviceToHost, ctx->stream) != cudaSuccess) return MV_ERR_CUDA;
+  if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return MV_ERR_CUDA;
+  return flag != 0 ? MV_ERR_TIMEOUT : MV_OK;
 }
 
 bool overlap(const void* a, size_t na, const void* b, size_t nb) {
@@ -2722,6 +2896,9 @@ int mv_create(mv_ctx** out, void* stream, void* workspace, size_t workspace_byte
   c->sms = 0;
   c->cta_budget = 8;
   c->dbg_ready = false;
+  c->tail_state = 0;
+  c->tail_mode = 1;
+  c->tail_pdl = 0;
   c->timing = 0;
   c->timing_calls = 0;
   c->timing_now = false;
@@ -2810,6 +2987,13 @@ int mv_read_kernel_timing(mv_ctx* ctx, float* total_ms, int* launches) {
   *total_ms = sum;
   *launches = cnt;
   ctx->timed = 0;
+  return MV_OK;
+}
+
+int mv_set_tail_kernel(mv_ctx* ctx, int enable) {
+  if (ctx == nullptr) return MV_ERR_INVALID_ARG;
+  if (enable < 0 || enable > 2) return MV_ERR_INVALID_ARG;
+  ctx->tail_mode = enable;
   return MV_OK;
 }
 
@@ -2909,6 +3093,13 @@ int mv_sparse_step(mv_ctx* ctx, const float* grads, float* err, int N, int64_t d
   ctx->last_N = N;
   ctx->last_d = d;
   ctx->last_K = K;
+  if (tail_usable(ctx, L, N, K)) {
+    // two kernels: the streaming pass, then everything else (select, picks, votes, shared mask, aggregate) in one
+    P pt = p;
+    rc = vote_impl(ctx, p, L, grads, err, false, true, false, false, true, &pt);
+    if (rc == MV_OK) rc = tail_impl(ctx, pt, L, err, out_idx, out_val);
+    return rc;
+  }
   rc = vote_impl(ctx, p, L, grads, err, false, true, false, false);  // (the workers' lists and masks are no output of the step)
   p.prefetch_acc = err;
   if (rc == MV_OK) rc = select_impl(ctx, p, L, p.votes, true, out_idx, nullptr);
@@ -3159,8 +3350,7 @@ int mv_sparse_step_host(mv_ctx* ctx, const float* h_grads, int N, int64_t d, int
     return MV_ERR_CUDA;
   if (cudaMemcpyAsync(h_out_val, d_out_val, (size_t)K * 4, cudaMemcpyDeviceToHost, ctx->stream) != cudaSuccess)
     return MV_ERR_CUDA;
-  if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return MV_ERR_CUDA;
-  return MV_OK;
+  return abort_status(ctx);  // (waits for the stream)
 }
 
 int mv_read_diag(mv_ctx* ctx, int N, uint32_t* per_worker) {
@@ -3173,9 +3363,10 @@ int mv_read_diag(mv_ctx* ctx, int N, uint32_t* per_worker) {
   if (e == cudaSuccess)
     e = cudaMemcpyAsync(tau, ctx->ws + (ctx->tau_flip ? L.tau_alt : L.tau), (size_t)N * 4, cudaMemcpyDeviceToHost, ctx->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
-  if (e != cudaSuccess) {
+  const int ab = e == cudaSuccess ? abort_status(ctx) : MV_ERR_CUDA;
+  if (ab != MV_OK) {
     free(cnt);
-    return MV_ERR_CUDA;
+    return ab;
   }
   for (int n = 0; n < N; n++) {
     const bool general = ctx->mode == MV_MODE_GENERAL || cnt[n] < (uint32_t)ctx->last_K || cnt[n] > L.cap;
@@ -3195,8 +3386,7 @@ int mv_fallback_count(mv_ctx* ctx, uint32_t* total) {
   *total = 0;
   if (!ctx->dbg_ready) return MV_OK;  // no call yet
   if (cudaMemcpyAsync(total, ctx->ws + 4, 4, cudaMemcpyDeviceToHost, ctx->stream) != cudaSuccess) return MV_ERR_CUDA;
-  if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return MV_ERR_CUDA;
-  return MV_OK;
+  return abort_status(ctx);  // (waits for the stream)
 }
 
 int mv_debug_build(void) { return kChecked ? 1 : 0; }
@@ -3210,7 +3400,7 @@ int mv_debug_status(mv_ctx* ctx, int* device_status) {
   if (cudaMemsetAsync(ctx->ws, 0, 4, ctx->stream) != cudaSuccess) return MV_ERR_CUDA;
   if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return MV_ERR_CUDA;
   *device_status = (int)word;
-  return MV_OK;
+  return abort_status(ctx);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -3296,6 +3486,7 @@ const char* mv_status_string(int status) {
     case MV_ERR_INVALID_ARG: return "invalid argument (null or misaligned pointer, size out of range, or grads overlapping err)";
     case MV_ERR_WORKSPACE: return "workspace smaller than mv_workspace_bytes(N, d, K)";
     case MV_ERR_CUDA: return "the CUDA runtime reported an error";
+    case MV_ERR_TIMEOUT: return "a bounded wait between the CTAs of a kernel gave up; results of this context are not valid";
     case MV_ERR_TOO_LARGE: return "d exceeds MV_SELECT_STATIC_MAX_D, the size the built-in scratch array of mv_select_static was compiled for";
     default: return "unknown status";
   }

@@ -101,4 +101,15 @@ def compare_all(ctx, grads_t, err_t, K, ref=None, by_sort=False, label=""):
     fu2 = run_step(ctx, grads_t, err_t, K)   # same input again: identical bytes
     for k in ("out_idx", "out_val", "err"):
         assert torch.equal(fu[k].view(torch.int32), fu2[k].view(torch.int32)), L + f"{k} differs between two runs"
+    # the whole step has two implementations of what follows the streaming pass (a sequence of kernels, and one
+    # persistent kernel with grid barriers): both, forced, against the oracle and against each other
+    for setting, name in ((2, "single-kernel tail"), (0, "kernel sequence")):
+        ctx.set_tail_kernel(setting)
+        try:
+            fv = run_step(ctx, grads_t, err_t, K)
+        finally:
+            ctx.set_tail_kernel(1)
+        first_diff(npy(fv["out_idx"]), ref["out_idx"], L + f"out_idx ({name})")
+        first_diff(bits(npy(fv["err"])), bits(ref["err"]), L + f"err ({name})")
+        first_diff(bits(npy(fv["out_val"])), bits(npy(fu["out_val"])), L + f"out_val bytes ({name})")
     return ref, ph, fu

@@ -578,3 +578,38 @@ def test_checked_build_reports_the_fallback_and_the_overflow():
     torch.cuda.synchronize()
     assert ctx.debug_status() == B.MV_DBG_GATHER_RANGE
     assert val.cpu().tolist()[1:3] == [0.0, 0.0]
+
+
+@pytest.mark.parametrize("tail", [2, 0], ids=["single-kernel", "sequence"])
+def test_both_tails_through_fallbacks_and_tracking(tail):
+    """Whole steps with either implementation of the part after the streaming pass, over a run that visits the
+    rare routes: a tracked threshold that misses after a jump of scale (full-row select), rows with heavy ties
+    (threshold ties kept in part), equal rows, and ordinary steps in between; residual carried, every step
+    compared with the oracle."""
+    N, d, K = 5, 260_003, 2600
+    ctx = B.MvContext(N, d, K, device=DEV, mode=B.MV_MODE_TRACK)
+    ctx.set_tail_kernel(tail)
+    g = torch.Generator().manual_seed(777)
+    err_gpu = torch.zeros(N, d, device=DEV)
+    err_ref = np.zeros((N, d), dtype=np.float32)
+    out_idx = torch.empty(K, dtype=torch.int32, device=DEV)
+    out_val = torch.empty(K, dtype=torch.float32, device=DEV)
+    fell = []
+    for step, kind in enumerate(["gauss", "gauss", "big", "big", "ties", "ties", "gauss", "equal", "gauss", "gauss"]):
+        grads = torch.randn(N, d, generator=g)
+        if kind == "big":
+            grads[1:] *= 1e3
+        elif kind == "ties":
+            grads = (grads * 8).round() / 8
+        elif kind == "equal":
+            grads[2] = 0.5
+        ref = O.mv_sparse_step(grads.numpy(), err_ref, K)
+        ctx.mv_sparse_step(grads.to(DEV), err_gpu, out_idx, out_val)
+        torch.cuda.synchronize()
+        fell.append(int(ctx.read_diag(N)[:, 2].sum()))
+        PT.first_diff(PT.npy(out_idx), ref["out_idx"], f"step {step} ({kind}) out_idx")
+        PT.check_out_val(PT.npy(out_val), ref, ref["acc"], ref["out_idx"].astype(np.int64), f"step {step} out_val")
+        PT.first_diff(PT.bits(PT.npy(err_gpu)), PT.bits(ref["err"]), f"step {step} ({kind}) err")
+        err_ref = ref["err"]
+    assert fell[0] == 0 and fell[2] >= 1, fell          # the jump of scale sends workers over their full rows
+    assert ctx.last_launches() == (2 if tail == 2 else 6)
