@@ -282,3 +282,46 @@ def mv_ad_step(grads, err, prev, K: int, K_ad: int):
     return dict(acc=acc, worker_idx=worker_idx, add=adds, drop=drops, prev=new_prev, msum=msum,
                 out_idx=out_idx, vote_thresh=(vstar, vgt, veq), out_val=aggregate(acc, out_idx),
                 err=residual(acc, out_idx))
+
+
+# ============================================================================
+# SSGD-top-K (the paper's comparison scheme: Section 2, first paragraph, the
+# masked gradient of Eq. 6 and the update of Eq. 7; Table 1, row "SSGD-top-K")
+#
+# Every worker keeps the K largest |acc_n| under its OWN mask and the server
+# averages what it receives:
+#   M_n   = S_top(|acc_n|, K)
+#   G     = (1/N) sum_n M_n (x) acc_n        non-zero only on the union of the masks
+#   err_n = acc_n - M_n (x) acc_n            each worker's residual on its own mask
+# The union holds between K and N K coordinates (the masks need not match: this
+# is why the scheme's downlink is up to N times heavier than its uplink).
+#
+# Readings: error accumulation as in Algorithm 1 (the paper runs all schemes
+# with it); the union is reported as an ascending index list, defined by the
+# masks and not by the values (a coordinate whose kept values cancel stays in
+# it); a value is the binary64 sum, in worker order, over the workers that kept
+# the coordinate, divided by N (all N workers, as in Eq. 7's 1/N), rounded once
+# to binary32; ties in S_top to the lowest index; the residual is +0.0 where the
+# worker's own mask is set and a bit copy elsewhere.
+# ============================================================================
+def topk_union_step(grads, err, K: int, by_sort: bool = False, threads: int = 1):
+    """One SSGD-top-K step.  Returns a dict with acc, worker_idx [N,K], worker_bits, votes [d],
+    union_idx (ascending int32), union_val (float32, same length) and the new err [N,d]."""
+    r = mv_vote(grads, err, K, by_sort=by_sort, threads=threads)
+    acc = r["acc"]
+    N, d = acc.shape
+    union = np.flatnonzero(r["votes"] > 0).astype(np.int32)          # coordinates at least one worker kept
+    cols = union.astype(np.int64)
+    total = np.zeros(cols.shape[0], dtype=np.float64)
+    new_err = np.array(acc, dtype=np.float32, copy=True)
+    with np.errstate(all="ignore"):
+        for n in range(N):                                             # worker order
+            kept = np.zeros(d, dtype=bool)
+            kept[r["worker_idx"][n].astype(np.int64)] = True
+            k = kept[cols]
+            total[k] = total[k] + acc[n, cols[k]].astype(np.float64)
+            new_err[n, kept] = np.float32(0.0)
+        r["union_val"] = (total / np.float64(N)).astype(np.float32)
+    r["union_idx"] = union
+    r["err"] = new_err
+    return r
