@@ -158,6 +158,20 @@ int mv_ad_step(mv_ctx* ctx, const float* grads, float* err, uint32_t* prev_bits,
                int64_t K_ad, int32_t* out_idx, float* out_val, uint32_t* add_bits, uint32_t* drop_bits,
                uint8_t* msum);
 
+/* One step of SSGD-top-K, the scheme the paper compares majority voting with (Section 2, first paragraph: every
+ * worker sends acc_n (x) S_top(|acc_n|, K), Eq. 6, and the server forms (1/N) sum_n of what it receives, the
+ * estimate of Eq. 7; Table 1, row SSGD-top-K).  No consensus: the masks differ from worker to worker, so the
+ * aggregate is non-zero on their union, between K and min(d, N K) coordinates.
+ *   grads    [N*d] in;  err [N*d] in/out: e_n on entry, acc_n - M_n (x) acc_n on exit (each worker's residual is
+ *                       zeroed on its OWN mask)
+ *   out_idx  [capacity] out  the union of the workers' masks, ascending; entries from *count on are -1
+ *   out_val  [capacity] out  per union coordinate: the binary64 sum, in worker order, over the workers whose mask
+ *                            holds it, divided by N (all N workers), rounded once to binary32; 0 from *count on
+ *   capacity            >= min(d, N K), else MV_ERR_INVALID_ARG
+ *   count    [1] int32 out (DEVICE): the size of the union */
+int mv_topk_union_step(mv_ctx* ctx, const float* grads, float* err, int N, int64_t d, int64_t K,
+                       int32_t* out_idx, float* out_val, int64_t capacity, int32_t* count);
+
 /* Worker-sharded step (the paper's remark under Eq. 8 that a shared mask lets the values be summed by
  * an all-reduce): when the N workers are spread over several GPUs, each rank runs mv_vote on its
  * N_local rows, the vote counts (uint8 [d]) are summed over the ranks, every rank runs mv_select on

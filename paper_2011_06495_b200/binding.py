@@ -78,6 +78,8 @@ def _open(path: str, how: str) -> ctypes.CDLL:
     lib.mv_select.argtypes = [c_vp, c_vp, c_i, c_i64, c_i64, c_vp, c_vp]
     lib.mv_ad_step.restype = c_i
     lib.mv_ad_step.argtypes = [c_vp, c_vp, c_vp, c_vp, c_i, c_i64, c_i64, c_i64, c_vp, c_vp, c_vp, c_vp, c_vp]
+    lib.mv_topk_union_step.restype = c_i
+    lib.mv_topk_union_step.argtypes = [c_vp, c_vp, c_vp, c_i, c_i64, c_i64, c_vp, c_vp, c_i64, c_vp]
     lib.mv_select_static.restype = c_i
     lib.mv_select_static.argtypes = [c_vp, c_vp, c_i, c_i64, c_i64, c_vp, c_vp]
     lib.mv_aggregate.restype = c_i
@@ -271,6 +273,12 @@ class MvContext:
         _check(self.lib.mv_ad_step(self.handle, _ptr(grads), _ptr(err), _ptr(prev_bits), N, d, K or self.K, int(K_ad),
                                    _ptr(out_idx), _ptr(out_val), _ptr(add_bits), _ptr(drop_bits), _ptr(msum)),
                "mv_ad_step")
+
+    def mv_topk_union_step(self, grads, err, out_idx, out_val, count, K: Optional[int] = None):
+        """SSGD-top-K: out_idx / out_val [capacity >= min(d, N K)], count: int32 [1] on the device."""
+        N, d = grads.shape
+        _check(self.lib.mv_topk_union_step(self.handle, _ptr(grads), _ptr(err), N, d, K or self.K, _ptr(out_idx),
+                                           _ptr(out_val), out_idx.numel(), _ptr(count)), "mv_topk_union_step")
 
     def mv_select_rs(self, votes, N: int, seed: int, draw: int, out_idx, mask_bits=None, K: Optional[int] = None):
         _check(self.lib.mv_select_rs(self.handle, _ptr(votes), int(N), votes.numel(), int(K or self.K), int(seed), int(draw),

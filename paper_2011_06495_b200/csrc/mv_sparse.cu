@@ -63,6 +63,7 @@ struct P {
   int force_general;
   int list_mode;          // 1: the rows are plain (key, index) lists to select min(K, length) from (add-drop)
   int apply_rows;         // list mode: rows < apply_rows are "add" lists, the others "drop" lists
+  int take_all;           // vote_scan: the "mask" is every coordinate that holds a vote (the union of the workers' masks)
   int no_masks;           // 1: the picks only count votes; the workers' bit masks are neither cleared nor set
   const float* prefetch_acc;  // k_vote_write: if set, the rows whose elements at supp(M) the gather is about to read
   uint32_t* vote_words;   // cluster select: if set, every pick also adds one to its vote byte (four bytes per word)
@@ -868,26 +869,34 @@ __device__ void vote_scan(const P& p) {
     uint32_t voted = 0;
     for (int v = 1; v <= p.N; v++) voted += s_h[v];
     s_h[0] = (uint32_t)p.d - voted;  // coordinates nobody voted for
-    uint32_t acc = 0, vstar = 0, cgt = 0, ceq = 0;
-    for (int v = p.N; v >= 0; v--) {
-      const uint32_t h = s_h[v];
-      if (acc + h >= (uint32_t)p.K) {
-        vstar = (uint32_t)v;
-        cgt = acc;
-        ceq = h;
-        break;
+    uint32_t acc = 0, vstar = 0, cgt = 0, ceq = 0, total = (uint32_t)p.K;
+    if (p.take_all) {  // every voted coordinate: "votes >= 1", all ties at one vote kept
+      vstar = 1;
+      ceq = s_h[1];
+      cgt = voted - ceq;
+      total = voted;
+    } else {
+      for (int v = p.N; v >= 0; v--) {
+        const uint32_t h = s_h[v];
+        if (acc + h >= (uint32_t)p.K) {
+          vstar = (uint32_t)v;
+          cgt = acc;
+          ceq = h;
+          break;
+        }
+        acc += h;
       }
-      acc += h;
     }
     s_v[0] = vstar;
-    s_v[3] = (uint32_t)p.K - cgt;
+    s_v[1] = total;
+    s_v[3] = total - cgt;
     p.vstate[0] = vstar;
     p.vstate[1] = cgt;
     p.vstate[2] = ceq;
-    p.vstate[3] = (uint32_t)p.K - cgt;
+    p.vstate[3] = total - cgt;
   }
   __syncthreads();
-  const uint32_t vstar = s_v[0], quota = s_v[3];
+  const uint32_t vstar = s_v[0], quota = s_v[3], n_out = s_v[1];
   // Tiles of NT*8 chunks, a thread taking 8 neighbouring chunks of a tile (one 16-byte load per
   // count array); the loads of TB tiles are issued together, then every tile costs two block scans.
   // ecarry / scarry: v*-ties seen and outputs placed in the tiles before.
@@ -934,7 +943,7 @@ __device__ void vote_scan(const P& p) {
       for (int q = 0; q < 8; q++) {
         const uint32_t take = run >= quota ? 0u : min(eqv[q], quota - run);
         tk[q] = take;
-        ob[q] = c + q == p.nchunks ? (uint32_t)p.K : srun;
+        ob[q] = c + q == p.nchunks ? n_out : srun;
         run += eqv[q];
         srun += gtv[q] + take;
       }
@@ -951,7 +960,7 @@ __device__ void vote_scan(const P& p) {
     }
   }
   __syncthreads();
-  if (threadIdx.x == 0) p.out_base[p.nchunks] = (uint32_t)p.K;  // sentinel: end of the last chunk
+  if (threadIdx.x == 0) p.out_base[p.nchunks] = n_out;  // sentinel: end of the last chunk
 }
 
 // s_vh[v] (v >= 1) holds how many coordinates of chunk c got exactly v votes.  Stores, per chunk,
@@ -1995,6 +2004,54 @@ __global__ void __launch_bounds__(TPB) k_finish_mean(const double* __restrict__ 
   if (k < K) out_val[k] = (float)(sum[k] / n_total);
 }
 
+// SSGD-top-K (the comparison scheme: every worker under its own mask, the server averages what arrives).
+// idx[0 .. *n_out) = the union of the workers' masks, ascending.  out_val[k] = fl32( (sum over the workers n whose
+// mask holds idx[k], in worker order, of (double) acc[n][idx[k]]) / N ); those workers' residual becomes +0 there.
+// Entries from *n_out up to `capacity` are set to -1 / 0.  Also clears the leading scratch region like k_gather.
+__global__ void __launch_bounds__(TPB) k_union_gather(float* __restrict__ acc, int N, int64_t d, int64_t W,
+                                                      const uint32_t* __restrict__ bits, int32_t* __restrict__ idx,
+                                                      const uint32_t* __restrict__ n_out, float* __restrict__ out_val,
+                                                      int64_t capacity, int32_t* __restrict__ count,
+                                                      uint4* __restrict__ zero_ptr, uint32_t zero_vecs) {
+  pdl_enter();
+  for (uint32_t i = blockIdx.x * TPB + threadIdx.x; i < zero_vecs; i += gridDim.x * TPB)
+    zero_ptr[i] = make_uint4(0, 0, 0, 0);
+  const int64_t k = (int64_t)blockIdx.x * TPB + threadIdx.x;
+  const int64_t U = (int64_t)__ldcg(n_out);
+  if (k == 0) *count = (int32_t)(U < capacity ? U : capacity);
+  if (k >= capacity) return;
+  if (k >= U) {
+    idx[k] = -1;
+    out_val[k] = 0.f;
+    return;
+  }
+  const int64_t j = __ldcg(idx + k);
+  if (j < 0 || j >= d) {
+    out_val[k] = 0.f;
+    return;
+  }
+  const uint32_t bit = 1u << (uint32_t)(j & 31);
+  const uint32_t* wcol = bits + (j >> 5);
+  float* col = acc + j;
+  double s = 0.0;
+  for (int n0 = 0; n0 < N; n0 += 16) {
+    uint32_t has = 0;
+    float v[16];
+#pragma unroll
+    for (int q = 0; q < 16; q++)
+      if (n0 + q < N && (__ldcg(wcol + (size_t)(n0 + q) * (size_t)W) & bit)) has |= 1u << q;
+#pragma unroll
+    for (int q = 0; q < 16; q++) v[q] = (has >> q) & 1u ? __ldcg(col + (size_t)(n0 + q) * (size_t)d) : 0.f;
+#pragma unroll
+    for (int q = 0; q < 16; q++)
+      if ((has >> q) & 1u) s += (double)v[q];
+#pragma unroll
+    for (int q = 0; q < 16; q++)
+      if ((has >> q) & 1u) __stcg(col + (size_t)(n0 + q) * (size_t)d, 0.0f);
+  }
+  out_val[k] = (float)(s / (double)N);
+}
+
 // ---------------------------------------------------------------------------------------------
 // add-drop voting (Algorithm 2): from this step's top-K masks M_n and the previous vote masks Mt_n,
 //   k_ad_fill   lists, per worker, the coordinates of  M_n & ~Mt_n  (with their keys) and of
@@ -2401,6 +2458,7 @@ P make_params(const mv_ctx* ctx, const Layout& L, int N, int64_t d, int64_t K) {
   p.list_mode = 0;
   p.apply_rows = 0;
   p.no_masks = 0;
+  p.take_all = 0;
   p.vote_words = nullptr;
   p.prefetch_acc = nullptr;
   p.apply_bits = nullptr;
@@ -3106,6 +3164,42 @@ int mv_sparse_step(mv_ctx* ctx, const float* grads, float* err, int N, int64_t d
   if (rc == MV_OK) rc = aggregate_impl(ctx, err, N, d, K, out_idx, out_val, L.zero_bytes);
   const int rcj = join_side(ctx);
   return rc != MV_OK ? rc : rcj;
+}
+
+int mv_topk_union_step(mv_ctx* ctx, const float* grads, float* err, int N, int64_t d, int64_t K, int32_t* out_idx,
+                       float* out_val, int64_t capacity, int32_t* count) {
+  Layout L;
+  int rc = check_common(ctx, N, d, K, L);
+  if (rc != MV_OK) return rc;
+  if (grads == nullptr || err == nullptr || out_idx == nullptr || out_val == nullptr || count == nullptr)
+    return MV_ERR_INVALID_ARG;
+  if (!aligned16(grads) || !aligned16(err) || !aligned16(out_idx) || !aligned16(out_val) || ((uintptr_t)count & 3u) != 0)
+    return MV_ERR_INVALID_ARG;
+  const int64_t most = (int64_t)N * K < d ? (int64_t)N * K : d;  // the union cannot hold more
+  if (capacity < most || capacity >= ((int64_t)1 << 31)) return MV_ERR_INVALID_ARG;
+  const size_t nb = (size_t)N * (size_t)d * 4;
+  if (overlap(grads, nb, err, nb)) return MV_ERR_INVALID_ARG;
+  if (const int rd = device_ready(ctx)) return rd;
+  ctx->launches = 0;
+  if (ctx->phase_timing) cudaEventRecord(ctx->pev[0], ctx->stream);
+  P p = make_params(ctx, L, N, d, K);
+  p.take_all = 1;
+  ctx->last_N = N;
+  ctx->last_d = d;
+  ctx->last_K = K;
+  // the workers' masks (kept in the workspace), the votes, and the offsets of all voted coordinates
+  rc = vote_impl(ctx, p, L, grads, err, false, true, false, true);
+  if (rc != MV_OK) return rc;
+  P w = p;
+  w.K = capacity;  // room of the list that k_vote_write fills
+  rc = select_impl(ctx, w, L, p.votes, true, out_idx, nullptr);
+  if (rc != MV_OK) return rc;
+  launch_k(k_union_gather, dim3((unsigned)((capacity + TPB - 1) / TPB)), dim3(TPB), ctx->stream, err, N, d, L.W,
+           (const uint32_t*)p.worker_bits, out_idx, (const uint32_t*)(p.out_base + p.nchunks), out_val, capacity, count,
+           (uint4*)(ctx->ws + L.zero_off), (uint32_t)(L.zero_bytes / 16));
+  MV_LAUNCH_CHECK();
+  ctx->clean_bytes = L.zero_bytes;
+  return join_side(ctx);
 }
 
 int mv_ad_step(mv_ctx* ctx, const float* grads, float* err, uint32_t* prev_bits, int N, int64_t d, int64_t K,
