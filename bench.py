@@ -10,7 +10,8 @@ region.  Before the warm-up the residuals are carried through 300 untimed steps,
 steps are those of a run in progress (every chunk of every worker holds candidates) and not of its
 first iterations.  One JSON line is printed by rank 0; with the default workload it also carries the
 other two ResNet-scale configurations under "also".  With --gpus N > 1 (launched through torchrun) every
-rank runs an independent replica of the same workload: the path does not shard across devices.
+rank runs an independent replica of the same workload (the one-GPU step does not shard); `--sharded` instead
+spreads the workload's N workers over the ranks and all-reduces the votes and the partial sums.
 """
 from __future__ import annotations
 
@@ -452,6 +453,121 @@ def measure(w: WL.Workload, args, B, dev, dist, world, local_rank, with_e2e: boo
     return out
 
 
+def shard_rows(N: int, world: int, rank: int):
+    """Rows [lo, hi) of the N workers that rank `rank` of `world` holds in the worker-sharded step."""
+    return rank * N // world, (rank + 1) * N // world
+
+
+def run_sharded(args, w: WL.Workload):
+    """The worker-sharded step (launched through torchrun, one rank per GPU): the N workers of the workload are
+    spread over the ranks, every rank streams and selects its own rows, the vote counts (d bytes) and the
+    binary64 partial sums on the shared mask (8K bytes) are all-reduced over NCCL, every rank ends up with
+    the same mask and values.  Total work is fixed, so scaling is strong; the step time is the slowest
+    rank's (CUDA events on the context's stream, barrier and synchronize on both sides)."""
+    import torch.distributed as dist
+    from paper_2011_06495_b200 import binding as B
+    from paper_2011_06495_b200.sharded import ShardedStep
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    if world > w.N:
+        raise SystemExit(f"--sharded: {world} ranks for {w.N} workers (every rank needs at least one)")
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    os.environ.setdefault("MASTER_PORT", "29655")
+    dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
+
+    def barrier():
+        dist.barrier()
+        torch.cuda.synchronize()
+
+    lo, hi = shard_rows(w.N, world, rank)
+    n_local = hi - lo
+    std = WL.std_vector(w, dev) if w.segments > 1 else None
+    mode = {"auto": B.MV_MODE_AUTO, "general": B.MV_MODE_GENERAL, "track": B.MV_MODE_TRACK}[args.mode]
+    ctx = B.MvContext(w.N, w.d, w.K, device=dev, mode=mode)
+    step = ShardedStep(ctx, w.N, w.d, w.K, dev)
+    err = WL.initial_err(w, device=dev)[lo:hi].clone()
+    out_idx = torch.empty(w.K, dtype=torch.int32, device=dev)
+    out_val = torch.empty(w.K, dtype=torch.float32, device=dev)
+    full = torch.empty((w.N, w.d), dtype=torch.float32, device=dev)
+    preheat = args.preheat if args.preheat >= 0 else (PREHEAT_STEPS if w.steps > 1 else 0)
+    for s in range(preheat):                       # every rank draws the whole step's gradients and keeps its rows
+        step.step(WL.gradients(w, 100_000 + s, out=full, std=std)[lo:hi], err, out_idx, out_val)
+    nbytes_local = n_local * w.d * 4
+    pool_n = int(max(2, min(args.steps + args.warmup, POOL_BYTES // max(nbytes_local, 1), 64)))
+    pool = [WL.gradients(w, s, out=full, std=std)[lo:hi].clone() for s in range(pool_n)]
+    del full
+    torch.cuda.synchronize()
+    # kernels per step, counted once outside the timed region
+    # (one whole step written out call by call, as ShardedStep.step makes them)
+    launches = 0
+    ctx.mv_vote(pool[0], err, votes=step.votes, K=w.K)
+    launches += ctx.last_launches()
+    dist.all_reduce(step.votes, op=dist.ReduceOp.SUM)
+    ctx.mv_select(step.votes, w.N, out_idx, K=w.K)
+    launches += ctx.last_launches()
+    ctx.mv_aggregate_partial(err, out_idx, step.partial)
+    launches += ctx.last_launches() + 1            # + the kernel of mv_finish_mean
+    dist.all_reduce(step.partial, op=dist.ReduceOp.SUM)
+    ctx.mv_finish_mean(step.partial, w.N, out_val)
+    sampler = ClockSampler(visible_gpu_index(local_rank))
+    sampler.start()
+    k = 0
+    for _ in range(args.warmup):
+        step.step(pool[k % pool_n], err, out_idx, out_val)
+        k += 1
+    ctx.set_kernel_timing(8 if args.steps >= 8 else 1)
+    sampler.wait_for_first_sample()
+    barrier()
+    first_row = sampler.rows_so_far()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(args.steps):
+        step.step(pool[k % pool_n], err, out_idx, out_val)
+        k += 1
+    ev1.record()
+    barrier()
+    time.sleep(0.03)
+    clocks = sampler.stop(first_row)
+    k_ms, k_cnt = ctx.read_kernel_timing()
+    ms_total = max_over_ranks(ev0.elapsed_time(ev1), dist, dev)
+    checksum = int(out_idx.sum(dtype=torch.int64).item())
+    sums = torch.tensor([checksum], dtype=torch.int64, device=dev)
+    gathered = [torch.zeros_like(sums) for _ in range(world)]
+    dist.all_gather(gathered, sums)
+    same_mask = all(int(g.item()) == checksum for g in gathered)
+    if rank == 0:
+        peak, peak_kind = measured_peak()
+        ms_step = ms_total / args.steps
+        alg_local = 12.0 * n_local * w.d
+        k_ms_avg = k_ms / max(k_cnt, 1)
+        achieved = alg_local / (k_ms_avg * 1e-3) / 1e9 if k_cnt else None
+        line = {
+            "metric": METRIC, "value": args.steps / (ms_total * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "strong",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": dict(workload_config(w), parallelism="workers sharded over ranks: all-reduce of u8 votes (d B) and "
+                                                           "of binary64 partial sums (8K B)"),
+            "setup": {"workers_per_rank": [shard_rows(w.N, world, r)[1] - shard_rows(w.N, world, r)[0] for r in range(world)],
+                      "preheat_steps": preheat, "gradient_pool": pool_n, "collectives": "NCCL all_reduce x 2 per step",
+                      "collective_bytes_per_step": w.d + 8 * w.K},
+            "effective_gradient_gbs": w.N * w.d * 4 / (ms_step * 1e-3) / 1e9,
+            "step_roofline_frac": 12.0 * w.N * w.d / world / (ms_step * 1e-3) / 1e9 / peak,
+            "roofline": {"bound": "hbm", "kernel": "k_acc_compact", "achieved": achieved, "peak": peak,
+                         "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": (achieved / peak) if achieved else None,
+                         "traffic": None, "kernel_ms": k_ms_avg, "algorithmic_bytes_per_launch": alg_local,
+                         "note": "rank 0's streaming pass over its own workers' rows"},
+            "clocks": clocks, "gpu_launches": launches * args.steps, "launches_per_step": launches,
+            "same_mask_on_every_rank": same_mask,
+        }
+        print(json.dumps(line), flush=True)
+    dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -473,6 +589,9 @@ def main():
     ap.add_argument("--no-also", action="store_true",
                     help="with the default workload c2 the line also carries c3 and c4 (the other two ResNet-scale "
                          "configurations) under \"also\"; this switches that off")
+    ap.add_argument("--sharded", action="store_true",
+                    help="the worker-sharded step: the workload's N workers spread over the ranks (torchrun), votes and "
+                         "partial sums all-reduced; strong scaling.  Without it, N GPUs run N replicas")
     ap.add_argument("--sweep", action="store_true",
                     help="instead of the one bench line: time the 27 cells of the sweep (N x d x K/d), one JSON line per "
                          "cell, a single step timed after warm-up with the residual restored before every repeat")
@@ -486,6 +605,9 @@ def main():
 
     if args.impl == "reference":
         run_reference(args, w)
+        return
+    if args.sharded:
+        run_sharded(args, w)
         return
 
     from paper_2011_06495_b200 import binding as B

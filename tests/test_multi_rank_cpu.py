@@ -124,3 +124,29 @@ def test_worker_sharded_step_equals_the_unsharded_step(tmp_path):
             np.testing.assert_allclose(val.numpy(), ref["out_val"], rtol=1e-6, atol=1e-12)
     got_err = np.concatenate([res[r]["err"].numpy() for r in range(world)], axis=0)
     assert np.array_equal(got_err.view(np.uint32), err.view(np.uint32))              # residuals, rank by rank
+
+
+def _rows_rank(rank, world, port, out_dir):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    sys.path.insert(0, ROOT)
+    import bench
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    seen = {}
+    for N in (2, 5, 10, 25):
+        lo, hi = bench.shard_rows(N, world, rank)
+        mine = torch.zeros(N, dtype=torch.int32)
+        mine[lo:hi] = 1
+        dist.all_reduce(mine)                        # every worker row is held by exactly one rank
+        seen[N] = (lo, hi, mine.tolist())
+    with open(os.path.join(out_dir, f"rows{rank}.json"), "w") as f:
+        json.dump(seen, f)
+    dist.destroy_process_group()
+
+
+def test_sharded_bench_splits_the_workers_over_the_ranks(tmp_path):
+    world = 2
+    mp.spawn(_rows_rank, args=(world, 29634, str(tmp_path)), nprocs=world, join=True)
+    for rank in range(world):
+        seen = json.load(open(tmp_path / f"rows{rank}.json"))
+        for N, (lo, hi, cover) in seen.items():
+            assert cover == [1] * int(N) and hi > lo

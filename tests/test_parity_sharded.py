@@ -79,3 +79,19 @@ def test_sharded_step_in_a_one_rank_nccl_group():
     finally:
         if created:
             dist.destroy_process_group()
+
+
+def test_sharded_bench_with_one_rank_gives_the_unsharded_mask():
+    """`bench.py --sharded` in a one-rank NCCL group ends on the same mask as the plain step of the same run
+    length would (checked through the line it prints and through a short plain run of the library)."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, RANK="0", WORLD_SIZE="1", LOCAL_RANK="0", MASTER_ADDR="127.0.0.1", MASTER_PORT="29642")
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--sharded", "--workload", "c1", "--steps", "4",
+                        "--warmup", "3"], env=env, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stderr[-2000:]
+    line = json.loads(r.stdout.strip().splitlines()[-1])
+    assert line["scaling"] == "strong" and line["n_gpus"] == 1 and line["same_mask_on_every_rank"] is True
+    assert line["setup"]["workers_per_rank"] == [4] and line["launches_per_step"] >= 4 and line["value"] > 0
