@@ -2295,6 +2295,7 @@ __global__ void __launch_bounds__(TPB) k_ad_apply(uint32_t* __restrict__ prev_bi
 }
 
 #include "mv_tail.cuh"
+#include "mv_small.cuh"
 static_assert(F_RADIX <= SB_BINS, "the three-digit counts live in the sample histogram's rows");
 
 // ---------------------------------------------------------------------------------------------
@@ -2313,6 +2314,7 @@ struct Layout {
   size_t samp_hist, hist1, hist2, hist2b, hist3, cand_cnt, sample_done, count_done, votes_done, hot, vote_hist;
   size_t tau, tau_alt, tstate, diag_cnt, wstate, thresh, vstate, cand, chunk_base, chunk_cnt, chunk_eq, tie_base, chunk_sel;
   size_t worker_bits, worker_idx, votes, chunk_vh, out_base, tie_take;
+  size_t votes_alt;   // rows that fit one CTA (d <= SMALL_MAX_D): the second vote array of the single-kernel step
   // add-drop voting: the select state once more, for 2N lists of at most ad_cap entries
   uint32_t ad_cap;
   size_t ad_zero, ad_zero_bytes;  // cleared at the start of every add-drop vote
@@ -2377,6 +2379,7 @@ Layout make_layout(int N, int64_t d, int64_t K) {
   L.chunk_vh = take(off, (size_t)(((L.nchunks + 7) & ~7)) * (n + 1) * 2);
   L.out_base = take(off, (nc + 1) * 4);
   L.tie_take = take(off, nc * 4);
+  L.votes_alt = take(off, d <= SMALL_MAX_D ? nc * CH : 0);
   {
     const size_t m = 2 * n;
     L.ad_cap = (uint32_t)((K + 7) & ~(int64_t)7);
@@ -2434,6 +2437,11 @@ struct mv_ctx {
   bool dbg_ready;      // the workspace's header has been cleared once
   int tail_state;      // single-kernel tail: 0 = not tried, 1 = usable on this device, -1 = not
   int tail_mode;       // (mv_set_tail_kernel) 0 = never, 1 = where it pays, 2 = wherever it can run
+  int small_state;     // single-kernel small step: 0 = not tried, 1 = usable on this device, -1 = not
+  bool small_ready;    // the vote array that the next small step of size (small_N, small_d, small_K) uses is known to be zero
+  int small_N;
+  int64_t small_d, small_K;
+  int small_flip;      // which of the two holds the next call's votes
   int tail_pdl;        // -1: the runtime refused a cooperative launch with programmatic stream serialisation
   // remembered for mv_read_diag
   int last_N;
@@ -2648,6 +2656,7 @@ int vote_impl(mv_ctx* ctx, P p, const Layout& L, const float* grads, float* err,
   if (ctx->clean_bytes < L.zero_bytes && cudaMemsetAsync(ctx->ws + L.zero_off, 0, L.zero_bytes, st) != cudaSuccess)
     return MV_ERR_CUDA;
   ctx->clean_bytes = 0;  // dirty from here on, until a whole step's last kernel has cleared it again
+  ctx->small_ready = false;  // (the vote array is about to be written)
   // general mode: per-chunk outputs of the vote count start out cleared (only chunks with picks are
   // visited later); cleared on the side stream, concurrently with the first pass
   cudaStream_t zs = st;
@@ -2906,6 +2915,76 @@ int tail_impl(mv_ctx* ctx, const P& p, const Layout& L, float* err, int32_t* out
   return MV_OK;
 }
 
+bool small_ready_dev(mv_ctx* ctx) {
+  if (ctx->small_state == 0) {
+    ctx->small_state = -1;
+    int dev = -1, coop = 0, per_sm = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) == cudaSuccess &&
+        coop != 0 &&
+        cudaFuncSetAttribute(k_small, cudaFuncAttributeMaxDynamicSharedMemorySize, SK_KEYS * 4) == cudaSuccess &&
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_small, FT, SK_KEYS * 4) == cudaSuccess && per_sm >= 1)
+      ctx->small_state = 1;
+    else
+      cudaGetLastError();
+  }
+  return ctx->small_state == 1;
+}
+
+// rows that fit a CTA's shared memory: the whole step as one kernel, a CTA per worker
+bool small_usable(mv_ctx* ctx, int N, int64_t d) {
+  return ctx->tail_mode != 0 && ctx->mode != MV_MODE_GENERAL && d <= SMALL_MAX_D && N <= ctx->sms && small_ready_dev(ctx);
+}
+
+int small_impl(mv_ctx* ctx, const P& p, const Layout& L, const float* grads, float* err, int32_t* out_idx, float* out_val) {
+  char* b = ctx->ws;
+  cudaStream_t st = ctx->stream;
+  // the barrier words live in the region that is clear between steps; the two vote arrays are cleared here the
+  // first time (and after any other call that used the vote array), from then on by the kernel itself
+  if (ctx->clean_bytes < L.zero_bytes) {
+    if (cudaMemsetAsync(b + L.zero_off, 0, L.zero_bytes, st) != cudaSuccess) return MV_ERR_CUDA;
+    ctx->clean_bytes = L.zero_bytes;
+  }
+  const size_t vbytes = (size_t)L.nchunks * CH;
+  if (!ctx->small_ready || ctx->small_N != p.N || ctx->small_d != p.d || ctx->small_K != p.K) {
+    if (cudaMemsetAsync(b + L.votes, 0, vbytes, st) != cudaSuccess) return MV_ERR_CUDA;
+    if (cudaMemsetAsync(b + L.votes_alt, 0, vbytes, st) != cudaSuccess) return MV_ERR_CUDA;
+    ctx->small_flip = 0;
+  }
+  SmallArgs a;
+  a.grads = grads;
+  a.err = err;
+  a.out_idx = out_idx;
+  a.out_val = out_val;
+  a.votes_now = (uint32_t*)(b + (ctx->small_flip ? L.votes_alt : L.votes));
+  a.votes_next = (uint32_t*)(b + (ctx->small_flip ? L.votes : L.votes_alt));
+  a.words = (uint32_t*)(b + L.tail_words);
+  a.abort_flag = (uint32_t*)(b + L.abort_flag);
+  a.spin_limit = 1u << 21;
+  a.dbg = p.dbg;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)p.N);
+  cfg.blockDim = dim3(FT);
+  cfg.dynamicSmemBytes = SK_KEYS * 4;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeCooperative;
+  attr[0].val.cooperative = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, k_small, p, a) != cudaSuccess) {
+    cudaGetLastError();
+    return MV_ERR_CUDA;
+  }
+  MV_LAUNCH_CHECK();
+  ctx->small_flip ^= 1;
+  ctx->small_ready = true;  // (the kernel cleared the array that the next call votes in)
+  ctx->small_N = p.N;
+  ctx->small_d = p.d;
+  ctx->small_K = p.K;
+  ctx->track_valid = false;  // no threshold is carried out of this path
+  return MV_OK;
+}
+
 // has a bounded device-side wait given up on this context?  (reads the workspace header; the stream must be idle)
 int abort_status(mv_ctx* ctx) {
   if (!ctx->dbg_ready) return MV_OK;
@@ -2957,6 +3036,10 @@ int mv_create(mv_ctx** out, void* stream, void* workspace, size_t workspace_byte
   c->tail_state = 0;
   c->tail_mode = 1;
   c->tail_pdl = 0;
+  c->small_state = 0;
+  c->small_ready = false;
+  c->small_d = 0;
+  c->small_flip = 0;
   c->timing = 0;
   c->timing_calls = 0;
   c->timing_now = false;
@@ -3151,6 +3234,10 @@ int mv_sparse_step(mv_ctx* ctx, const float* grads, float* err, int N, int64_t d
   ctx->last_N = N;
   ctx->last_d = d;
   ctx->last_K = K;
+  if (small_usable(ctx, N, d)) {
+    P ps = p;
+    return small_impl(ctx, ps, L, grads, err, out_idx, out_val);
+  }
   if (tail_usable(ctx, L, N, K)) {
     // two kernels: the streaming pass, then everything else (select, picks, votes, shared mask, aggregate) in one
     P pt = p;

@@ -285,7 +285,10 @@ def test_threshold_tracking_over_steps(N, d, K):
         if step >= 2:
             assert (diag[:, 2] == 0).all(), f"step {step}: fallback with a tracked threshold: {diag.tolist()}"
         err_ref = ref["err"]
-    assert launches[0] == launches[1] + 1 and len(set(launches[1:])) == 1      # the sampling kernel runs once
+    if d <= 32768:
+        assert set(launches) == {1}            # a row that fits a CTA's shared memory: the whole step is one kernel
+    else:
+        assert launches[0] == launches[1] + 1 and len(set(launches[1:])) == 1      # the sampling kernel runs once
 
 
 @pytest.mark.parametrize("mode", [B.MV_MODE_AUTO, B.MV_MODE_TRACK], ids=["auto", "track"])
@@ -613,3 +616,36 @@ def test_both_tails_through_fallbacks_and_tracking(tail):
         err_ref = ref["err"]
     assert fell[0] == 0 and fell[2] >= 1, fell          # the jump of scale sends workers over their full rows
     assert ctx.last_launches() == (2 if tail == 2 else 6)
+
+
+@pytest.mark.parametrize("mode", [B.MV_MODE_AUTO, B.MV_MODE_TRACK], ids=["auto", "track"])
+def test_single_kernel_step_for_rows_that_fit_a_cta(mode):
+    """d <= 32768: the whole step is one kernel (a CTA per worker, exact select in shared memory, two vote arrays
+    that alternate).  Several steps with the residual carried, ties, K changing on the same context, another entry
+    point in between (which uses the vote array), and the sequence of kernels forced for comparison."""
+    N, d = 7, 20_011
+    g = torch.Generator().manual_seed(2024)
+    ctx = B.MvContext(N, d, 2000, device=DEV, mode=mode)
+    err_gpu = torch.zeros(N, d, device=DEV)
+    err_ref = np.zeros((N, d), dtype=np.float32)
+    for step, (K, kind) in enumerate([(200, "g"), (200, "g"), (200, "ties"), (2000, "g"), (200, "g"), (1, "g"), (200, "votes"),
+                                      (200, "g"), (200, "seq"), (200, "g")]):
+        grads = torch.randn(N, d, generator=g)
+        if kind == "ties":
+            grads = (grads * 2).round() / 2
+        if kind == "votes":      # the phases in between: mv_vote counts into the workspace's vote array
+            acc2 = torch.zeros(N, d, device=DEV)
+            ctx.mv_vote(torch.randn(N, d, generator=g).to(DEV), acc2, K=300)
+        ctx.set_tail_kernel(0 if kind == "seq" else 1)
+        ref = O.mv_sparse_step(grads.numpy(), err_ref, K)
+        out_idx = torch.full((K,), -7, dtype=torch.int32, device=DEV)
+        out_val = torch.full((K,), float("nan"), dtype=torch.float32, device=DEV)
+        ctx.mv_sparse_step(grads.to(DEV), err_gpu, out_idx, out_val, K=K)
+        torch.cuda.synchronize()
+        assert ctx.last_launches() == (1 if kind != "seq" else ctx.last_launches())
+        if kind != "seq":
+            assert ctx.last_launches() == 1
+        PT.first_diff(PT.npy(out_idx), ref["out_idx"], f"step {step} ({kind}, K={K}) out_idx")
+        PT.check_out_val(PT.npy(out_val), ref, ref["acc"], ref["out_idx"].astype(np.int64), f"step {step} out_val")
+        PT.first_diff(PT.bits(PT.npy(err_gpu)), PT.bits(ref["err"]), f"step {step} ({kind}) err")
+        err_ref = ref["err"]
