@@ -1768,15 +1768,48 @@ __global__ void __launch_bounds__(TPB) k_lists(P p) {
 // global counts and one ticket.
 constexpr int VH_WARPS = TPB / 32;
 
+// Vote counts of chunk c from its 4096 vote bytes, held by a warp as eight 16-byte pieces per lane: stores
+// chunk_vh[v][c] = #{votes >= v} for v = 0..N and adds the exact counts #{votes == v}, v >= 1, to s_tot (shared
+// memory).  #{votes >= v} comes from byte compares over the lane's registers, summed over the warp: no
+// per-coordinate atomics, however the votes crowd.  The count is the same in all lanes, so the loop may stop for
+// the whole warp once it reaches zero (the rows above are then written as zeros).  All 32 lanes call it.
+__device__ __forceinline__ void chunk_vote_counts(const P& p, int c, const uint4 (&q)[8], int lane, uint32_t* s_tot) {
+  const int64_t remd = p.d - (int64_t)c * CH;
+  uint32_t prev = (uint32_t)(remd < CH ? remd : CH);  // #{votes >= 0}: every coordinate of the chunk
+  if (lane == 0) p.chunk_vh[c] = (uint16_t)prev;
+  int v = 1;
+  for (; v <= p.N; v++) {
+    const uint32_t v4 = (uint32_t)v * 0x01010101u;
+    uint32_t cnt = 0;
+#pragma unroll
+    for (int u = 0; u < 8; u++) {
+      const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+#pragma unroll
+      for (int i = 0; i < 4; i++)
+        if (w[i]) cnt += __popc(__vcmpgeu4(w[i], v4));
+    }
+    cnt = __reduce_add_sync(FULL, cnt) >> 3;  // (eight bits per matching byte)
+    if (lane == 0) {
+      p.chunk_vh[(size_t)v * p.nc_pad + c] = (uint16_t)cnt;
+      if (v > 1 && prev != cnt) atomicAdd(&s_tot[v - 1], prev - cnt);  // coordinates with exactly v - 1 votes
+    }
+    prev = cnt;
+    if (cnt == 0) break;
+  }
+  if (v > p.N) {
+    if (lane == 0 && prev) atomicAdd(&s_tot[p.N], prev);  // exactly N votes (or more, if the input breaks its contract)
+  } else {
+    for (int z = v + 1 + lane; z <= p.N; z += 32) p.chunk_vh[(size_t)z * p.nc_pad + c] = 0;
+  }
+}
+
+
 __global__ void __launch_bounds__(TPB) k_vote_hist(P p, const uint8_t* __restrict__ votes, uint8_t* __restrict__ copy) {
   pdl_enter();
-  __shared__ uint32_t s_vh[VH_WARPS][256];  // exact counts per vote value, one row per warp
   __shared__ uint32_t s_tot[256];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int c = blockIdx.x * VH_WARPS + warp;
   s_tot[tid] = 0;
-#pragma unroll
-  for (int k = 0; k < 8; k++) s_vh[warp][k * 32 + lane] = 0;
   __syncthreads();
   if (c < p.nchunks) {
     uint4 q[8];
@@ -1803,39 +1836,8 @@ __global__ void __launch_bounds__(TPB) k_vote_hist(P p, const uint8_t* __restric
           for (int b = 0; b < 16 && jb + b < p.d; b++) copy[jb + b] = (uint8_t)((w[b >> 2] >> (8 * (b & 3))) & 0xffu);
         }
       }
-      if (w[0] | w[1] | w[2] | w[3]) {
-#pragma unroll
-        for (int b = 0; b < 16; b++) {
-          const uint32_t v = (w[b >> 2] >> (8 * (b & 3))) & 0xffu;
-          if (v) atomicAdd(&s_vh[warp][v], 1u);
-        }
-      }
     }
-    __syncwarp();
-    // cum[v] = #{votes >= v}: lane l owns the values 8l .. 8l+7
-    uint32_t ex[8], lsum = 0;
-#pragma unroll
-    for (int k = 0; k < 8; k++) {
-      const int v = lane * 8 + k;
-      ex[k] = (v >= 1 && v <= p.N) ? s_vh[warp][v] : 0u;
-      lsum += ex[k];
-    }
-    uint32_t x = lsum;  // inclusive suffix sum over the lanes
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-      const uint32_t y = __shfl_down_sync(FULL, x, off);
-      if (lane + off < 32) x += y;
-    }
-    uint32_t run = x - lsum;  // counts of the values owned by higher lanes
-    const int64_t rem = p.d - (int64_t)c * CH;
-    const uint32_t valid = (uint32_t)(rem < CH ? rem : CH);
-#pragma unroll
-    for (int k = 7; k >= 0; k--) {
-      const int v = lane * 8 + k;
-      run += ex[k];
-      if (v <= p.N) p.chunk_vh[(size_t)v * p.nc_pad + c] = (uint16_t)(v == 0 ? valid : run);
-      if (ex[k]) atomicAdd(&s_tot[v], ex[k]);
-    }
+    chunk_vote_counts(p, c, q, lane, s_tot);
   }
   __syncthreads();
   if (tid >= 1 && tid <= p.N && s_tot[tid]) atomicAdd(&p.vote_hist[tid], s_tot[tid]);  // the zero-vote count is derived later

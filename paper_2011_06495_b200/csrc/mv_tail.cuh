@@ -25,7 +25,7 @@
 __device__ unsigned g_stamp_calls;
 #define TAIL_STAMP(i)                                                        \
   do {                                                                       \
-    if (blockIdx.x == 0 && threadIdx.x == 0) {                               \
+    if (threadIdx.x == 0) {                                                  \
       unsigned long long t_;                                                 \
       asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                 \
       stamps[i] = t_;                                                        \
@@ -163,7 +163,6 @@ __global__ void __launch_bounds__(FT, 1) k_tail(P p, TailArgs a) {
   __shared__ uint32_t s_lastout;
 #ifdef MV_TAIL_STAMPS
   unsigned long long stamps[16];
-  const unsigned stamps_dummy = 0;
 #endif
 #ifdef MV_TAIL_STAMPS
   unsigned long long t_begin_;
@@ -514,78 +513,18 @@ __global__ void __launch_bounds__(FT, 1) k_tail(P p, TailArgs a) {
   TAIL_STAMP(8);
   // ---- vote histogram: per chunk the counts #{votes >= v}, over the vector the exact counts; a warp per chunk ----
   {
-    uint32_t* s_vh = dsm + warp * 256;   // this warp's counts per vote value
-    uint32_t* s_tot = dsm + 32 * 256;    // the CTA's
+    uint32_t* s_tot = dsm;               // the CTA's exact counts per vote value
     __syncthreads();                      // (the keys are not needed any more)
     if (tid < 256) s_tot[tid] = 0;
     __syncthreads();
     for (int c = warp * G + b; c < p.nchunks; c += G * (FT / 32)) {  // neighbouring chunks go to different CTAs
-#pragma unroll
-      for (int k = 0; k < 8; k++) s_vh[k * 32 + lane] = 0;
-      __syncwarp();
       uint4 q[8];
 #pragma unroll
       for (int u = 0; u < 8; u++) {
         const int64_t jb = (int64_t)c * CH + (int64_t)(u * 32 + lane) * 16;
         q[u] = jb < p.d ? __ldcg(reinterpret_cast<const uint4*>(p.votes + jb)) : make_uint4(0, 0, 0, 0);
       }
-      // Most voted coordinates hold one, two or three votes: those are counted by byte compares in registers and
-      // added once per lane; only the rarer larger counts go through shared-memory atomics one by one.
-      uint32_t c1 = 0, c2 = 0, c3 = 0;
-#pragma unroll
-      for (int u = 0; u < 8; u++) {
-        const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
-        if (w[0] | w[1] | w[2] | w[3]) {
-#pragma unroll
-          for (int i = 0; i < 4; i++) {
-            const uint32_t x = w[i];
-            if (x == 0) continue;
-            c1 += __popc(__vcmpeq4(x, 0x01010101u));
-            c2 += __popc(__vcmpeq4(x, 0x02020202u));
-            c3 += __popc(__vcmpeq4(x, 0x03030303u));
-            uint32_t big = __vcmpgtu4(x, 0x03030303u);  // 0xff in every byte that holds four votes or more
-            while (big) {
-              const int bb = (__ffs(big) - 1) >> 3;
-              big &= ~(0xffu << (8 * bb));
-              atomicAdd(&s_vh[(x >> (8 * bb)) & 0xffu], 1u);
-            }
-          }
-        }
-      }
-      c1 = __reduce_add_sync(FULL, c1);
-      c2 = __reduce_add_sync(FULL, c2);
-      c3 = __reduce_add_sync(FULL, c3);
-      if (lane == 0) {  // (popc counted eight bits per matching byte)
-        s_vh[1] += c1 >> 3;
-        s_vh[2] += c2 >> 3;
-        s_vh[3] += c3 >> 3;
-      }
-      __syncwarp();
-      // cum[v] = #{votes >= v}: lane l owns the values 8l .. 8l+7
-      uint32_t ex[8], lsum = 0;
-#pragma unroll
-      for (int k = 0; k < 8; k++) {
-        const int v = lane * 8 + k;
-        ex[k] = (v >= 1 && v <= p.N) ? s_vh[v] : 0u;
-        lsum += ex[k];
-      }
-      uint32_t x = lsum;  // inclusive suffix sum over the lanes
-#pragma unroll
-      for (int off = 1; off < 32; off <<= 1) {
-        const uint32_t y = __shfl_down_sync(FULL, x, off);
-        if (lane + off < 32) x += y;
-      }
-      uint32_t run = x - lsum;  // counts of the values owned by higher lanes
-      const int64_t remd = p.d - (int64_t)c * CH;
-      const uint32_t valid = (uint32_t)(remd < CH ? remd : CH);
-#pragma unroll
-      for (int k = 7; k >= 0; k--) {
-        const int v = lane * 8 + k;
-        run += ex[k];
-        if (v <= p.N) p.chunk_vh[(size_t)v * p.nc_pad + c] = (uint16_t)(v == 0 ? valid : run);
-        if (ex[k]) atomicAdd(&s_tot[v], ex[k]);
-      }
-      __syncwarp();
+      chunk_vote_counts(p, c, q, lane, s_tot);
     }
     __syncthreads();
     if (tid >= 1 && tid <= p.N && s_tot[tid]) atomicAdd(&p.vote_hist[tid], s_tot[tid]);
@@ -767,7 +706,7 @@ __global__ void __launch_bounds__(FT, 1) k_tail(P p, TailArgs a) {
     unsigned long long t_;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));
     p.out_base[4 * blockIdx.x + 2] = (uint32_t)t_;
-    p.out_base[4 * blockIdx.x + 3] = (uint32_t)stamps_dummy;
+    p.out_base[4 * blockIdx.x + 3] = (uint32_t)(stamps[9] - stamps[8]);  // this CTA's vote-histogram phase
   }
 #endif
   __threadfence();
@@ -785,6 +724,15 @@ __global__ void __launch_bounds__(FT, 1) k_tail(P p, TailArgs a) {
     for (int i = 0; i < G; i++) {
       const uint32_t tb = __ldcg(p.out_base + 4 * i), tw = __ldcg(p.out_base + 4 * i + 1), te = __ldcg(p.out_base + 4 * i + 2);
       b0 = min(b0, tb); b1 = max(b1, tb); w0 = min(w0, tw); w1 = max(w1, tw); e0 = min(e0, te); e1 = max(e1, te);
+    }
+    {
+      uint32_t hmin = 0xffffffffu, hmax = 0, hsum = 0, harg = 0;
+      for (int i = 0; i < G; i++) {
+        const uint32_t h = __ldcg(p.out_base + 4 * i + 3);
+        hmin = min(hmin, h); hsum += h;
+        if (h > hmax) { hmax = h; harg = i; }
+      }
+      printf("hist phase per cta: min %.1f avg %.1f max %.1f us (cta %u)\n", hmin * 1e-3, hsum * 1e-3 / G, hmax * 1e-3, harg);
     }
     printf("ctas: first start 0, last start %.1f, wait over %.1f .. %.1f, first end %.1f, last end %.1f us\n", (b1 - b0) * 1e-3,
            (w0 - b0) * 1e-3, (w1 - b0) * 1e-3, (e0 - b0) * 1e-3, (e1 - b0) * 1e-3);
