@@ -1770,25 +1770,50 @@ constexpr int VH_WARPS = TPB / 32;
 
 // Vote counts of chunk c from its 4096 vote bytes, held by a warp as eight 16-byte pieces per lane: stores
 // chunk_vh[v][c] = #{votes >= v} for v = 0..N and adds the exact counts #{votes == v}, v >= 1, to s_tot (shared
-// memory).  #{votes >= v} comes from byte compares over the lane's registers, summed over the warp: no
-// per-coordinate atomics, however the votes crowd.  The count is the same in all lanes, so the loop may stop for
-// the whole warp once it reaches zero (the rows above are then written as zeros).  All 32 lanes call it.
-__device__ __forceinline__ void chunk_vote_counts(const P& p, int c, const uint4 (&q)[8], int lane, uint32_t* s_tot) {
+// memory).  #{votes >= v} comes from byte-wise compares over the lane's registers, summed over the warp: no
+// per-coordinate atomics, however the votes crowd.  With N <= 127 a compare of four bytes is one subtraction:
+// with bit 7 of every byte set beforehand, (byte | 0x80) - v keeps bit 7 exactly when byte >= v, and no borrow
+// leaves its byte; the kept bits are added up per byte lane over the 32 words (at most 32 each) and summed once.
+// The count is the same in all lanes, so the loop may stop for the whole warp once it reaches zero (the rows
+// above are then written as zeros).  All 32 lanes call it.  (The votes are not needed afterwards: q is changed.)
+__device__ __forceinline__ void chunk_vote_counts(const P& p, int c, uint4 (&q)[8], int lane, uint32_t* s_tot) {
   const int64_t remd = p.d - (int64_t)c * CH;
   uint32_t prev = (uint32_t)(remd < CH ? remd : CH);  // #{votes >= 0}: every coordinate of the chunk
   if (lane == 0) p.chunk_vh[c] = (uint16_t)prev;
+  const bool narrow = p.N <= 127;
+  if (narrow) {
+#pragma unroll
+    for (int u = 0; u < 8; u++) {
+      q[u].x |= 0x80808080u;
+      q[u].y |= 0x80808080u;
+      q[u].z |= 0x80808080u;
+      q[u].w |= 0x80808080u;
+    }
+  }
   int v = 1;
   for (; v <= p.N; v++) {
     const uint32_t v4 = (uint32_t)v * 0x01010101u;
     uint32_t cnt = 0;
+    if (narrow) {
+      uint32_t lanes4 = 0;  // four byte-wide counters
 #pragma unroll
-    for (int u = 0; u < 8; u++) {
-      const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+      for (int u = 0; u < 8; u++) {
+        lanes4 += ((q[u].x - v4) & 0x80808080u) >> 7;
+        lanes4 += ((q[u].y - v4) & 0x80808080u) >> 7;
+        lanes4 += ((q[u].z - v4) & 0x80808080u) >> 7;
+        lanes4 += ((q[u].w - v4) & 0x80808080u) >> 7;
+      }
+      cnt = (lanes4 * 0x01010101u) >> 24;
+    } else {
 #pragma unroll
-      for (int i = 0; i < 4; i++)
-        if (w[i]) cnt += __popc(__vcmpgeu4(w[i], v4));
+      for (int u = 0; u < 8; u++) {
+        const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+#pragma unroll
+        for (int i = 0; i < 4; i++)
+          if (w[i]) cnt += __popc(__vcmpgeu4(w[i], v4)) >> 3;  // (eight bits per matching byte)
+      }
     }
-    cnt = __reduce_add_sync(FULL, cnt) >> 3;  // (eight bits per matching byte)
+    cnt = __reduce_add_sync(FULL, cnt);
     if (lane == 0) {
       p.chunk_vh[(size_t)v * p.nc_pad + c] = (uint16_t)cnt;
       if (v > 1 && prev != cnt) atomicAdd(&s_tot[v - 1], prev - cnt);  // coordinates with exactly v - 1 votes
@@ -1802,7 +1827,6 @@ __device__ __forceinline__ void chunk_vote_counts(const P& p, int c, const uint4
     for (int z = v + 1 + lane; z <= p.N; z += 32) p.chunk_vh[(size_t)z * p.nc_pad + c] = 0;
   }
 }
-
 
 __global__ void __launch_bounds__(TPB) k_vote_hist(P p, const uint8_t* __restrict__ votes, uint8_t* __restrict__ copy) {
   pdl_enter();
