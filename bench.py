@@ -242,8 +242,9 @@ def run_reference(args, w: WL.Workload):
 def run_sweep(args):
     """The sweep of the configuration list: N in {4,16,64} x d in {2^20,2^24,2^27} x K/d in {1e-2,1e-3,2.5e-4},
     gradients with cross-worker correlation 0.3, residuals ~ N(0, 0.01^2).  Per cell: 3 warm-up steps, then
-    `reps` single steps, each from the same saved residual (the restore is outside the timed region), the
-    threshold sampled in every step (stateless mode); the median is reported.  One GPU."""
+    `reps` single steps, each from the same saved residual (the restore is outside the timed region); the
+    candidate threshold is carried from the step before (the default mode, --mode track: the warm-up steps
+    leave it; --mode auto samples it in every step instead); the median is reported.  One GPU."""
     from paper_2011_06495_b200 import binding as B
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
@@ -257,7 +258,8 @@ def run_sweep(args):
         err = torch.empty_like(err0)
         out_idx = torch.empty(w.K, dtype=torch.int32, device=dev)
         out_val = torch.empty(w.K, dtype=torch.float32, device=dev)
-        ctx = B.MvContext(w.N, w.d, w.K, device=dev, mode=B.MV_MODE_AUTO)
+        ctx = B.MvContext(w.N, w.d, w.K, device=dev,
+                          mode={"auto": B.MV_MODE_AUTO, "general": B.MV_MODE_GENERAL, "track": B.MV_MODE_TRACK}[args.mode])
         times = []
         for it in range(3 + reps):
             err.copy_(err0)
@@ -275,7 +277,8 @@ def run_sweep(args):
                            "l2": "inputs larger than L2" if 2 * nbytes > l2_bytes() else "inputs fit in L2"},
                 "effective_gradient_gbs": nbytes / ms / 1e6, "step_roofline_frac": 3 * nbytes / ms / 1e6 / peak,
                 "peak": peak, "peak_kind": "of " + peak_kind, "launches_per_step": ctx.last_launches(),
-                "fallback_workers": int((ctx.read_diag(w.N)[:, 2] != 0).sum()), "repeats": reps, "dtype": "f32", "data": "synthetic"}
+                "fallback_workers": int((ctx.read_diag(w.N)[:, 2] != 0).sum()), "repeats": reps, "dtype": "f32", "data": "synthetic",
+                "threshold": args.mode}
         print(json.dumps(line), flush=True)
         ctx.close()
         del grads, err0, err, out_idx, out_val, ctx
