@@ -74,8 +74,8 @@ enum {
 enum {
   MV_DBG_CAND_OVERFLOW = 1,   /* streaming pass (S_top candidate filter): a worker had more candidates than its
                                  buffer holds; the surplus was dropped and the worker takes the full-row select */
-  MV_DBG_WINDOW_OVERFLOW = 2, /* select (S_top, K-th key): the bin of the K-th key held more than 1024 keys; it was
-                                 resolved by the three-digit radix select instead */
+  MV_DBG_WINDOW_OVERFLOW = 2, /* select (S_top, K-th key): the bin of the K-th key held more than 1024 keys; it was resolved
+                                 by a second count over that bin's keys, or by the three-digit radix select */
   MV_DBG_FALLBACK = 4,        /* select: a worker's K-th key was found over its full row (candidate count outside [K, cap]) */
   MV_DBG_LIST_OVERFLOW = 8,   /* add-drop / random selection (Algorithm 2; Algorithm 1, S_rand line): a list outgrew its
                                  room and was treated as empty */
@@ -105,7 +105,7 @@ int mv_set_mode(mv_ctx* ctx, int mode);
  * Eq. 9, the shared mask, the aggregate of Eq. 8 and the residual): either as the sequence of kernels that mv_vote,
  * mv_select and mv_aggregate use, or as ONE kernel whose CTAs (one per multiprocessor, launched cooperatively) stay
  * resident and meet at grid barriers.  The single kernel can run when the device supports cooperative launches,
- * N is at most the number of multiprocessors, d <= 8192 * 4096 and the mode is not MV_MODE_GENERAL.
+ * N is at most the number of multiprocessors, d <= 32768 * 4096 = 2^27 and the mode is not MV_MODE_GENERAL.
  *   enable = 1 (default): the single kernel where it can run and K >= 65536 (many picks and outputs: there it is
  *                         faster), the sequence otherwise;  0: always the sequence;  2: the single kernel wherever
  *                         it can run.

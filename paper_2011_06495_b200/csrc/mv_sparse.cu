@@ -1955,10 +1955,23 @@ __global__ void __launch_bounds__(TPB) k_vote_write(P p, const uint8_t* __restri
 // same sequence of binary64 additions in worker order either way: with G = 8 the values are passed to it by
 // shuffles, so all 32 lanes of a warp must call together (`live` = false for lanes without an output).
 template <int G>
+__device__ __forceinline__ void gather_at(float* __restrict__ acc, int N, int64_t d, int64_t k, int64_t j, bool live, int g,
+                                          float* __restrict__ out_val, double* __restrict__ out_sum,
+                                          uint32_t* __restrict__ dbg);
+
+template <int G>
 __device__ __forceinline__ void gather_one(float* __restrict__ acc, int N, int64_t d, int64_t k, bool live, int g,
                                            const int32_t* __restrict__ idx, float* __restrict__ out_val,
                                            double* __restrict__ out_sum, uint32_t* __restrict__ dbg) {
   const int64_t j = live ? (int64_t)__ldcg(idx + k) : -1;  // (from L2: the index may have been written by this very kernel)
+  gather_at<G>(acc, N, d, k, j, live, g, out_val, out_sum, dbg);
+}
+
+// the same for output k whose coordinate j the caller already holds (j = -1 for a lane without an output)
+template <int G>
+__device__ __forceinline__ void gather_at(float* __restrict__ acc, int N, int64_t d, int64_t k, int64_t j, bool live, int g,
+                                          float* __restrict__ out_val, double* __restrict__ out_sum,
+                                          uint32_t* __restrict__ dbg) {
   const bool bad = j < 0 || j >= d;
   if (live && bad && g == 0) {
     MV_DBG(dbg, MV_DBG_GATHER_RANGE);
@@ -1990,12 +2003,14 @@ __device__ __forceinline__ void gather_one(float* __restrict__ acc, int N, int64
         v[q] = (!bad && n < N) ? __ldcg(col + (size_t)n * (size_t)d) : 0.f;
       }
 #pragma unroll
-      for (int q = 0; q < 4; q++)
+      for (int q = 0; q < 4; q++) {
+        if (n0 + q * G >= N) break;  // (uniform over the warp)
 #pragma unroll
         for (int h = 0; h < G; h++) {  // workers n0 + q G + h, in this order
           const float x = __shfl_sync(FULL, v[q], gbase + h);
           if (n0 + q * G + h < N) s += (double)x;
         }
+      }
     }
     if (bad) return;
     for (int n = g; n < N; n += G) __stcg(col + (size_t)n * (size_t)d, 0.0f);
@@ -2340,7 +2355,8 @@ struct Layout {
   size_t samp_hist, hist1, hist2, hist2b, hist3, cand_cnt, sample_done, count_done, votes_done, hot, vote_hist;
   size_t tau, tau_alt, tstate, diag_cnt, wstate, thresh, vstate, cand, chunk_base, chunk_cnt, chunk_eq, tie_base, chunk_sel;
   size_t worker_bits, worker_idx, votes, chunk_vh, out_base, tie_take;
-  size_t votes_alt;   // rows that fit one CTA (d <= SMALL_MAX_D): the second vote array of the single-kernel step
+  size_t votes_alt;   // rows that fit one CTA (d <= SMALL_MAX_D): the second vote array of the single-kernel step ...
+  size_t small_state; // ... and its two vote histograms [2][256] and two barrier words (at [512] and [528])
   // add-drop voting: the select state once more, for 2N lists of at most ad_cap entries
   uint32_t ad_cap;
   size_t ad_zero, ad_zero_bytes;  // cleared at the start of every add-drop vote
@@ -2406,6 +2422,7 @@ Layout make_layout(int N, int64_t d, int64_t K) {
   L.out_base = take(off, (nc + 1) * 4);
   L.tie_take = take(off, nc * 4);
   L.votes_alt = take(off, d <= SMALL_MAX_D ? nc * CH : 0);
+  L.small_state = take(off, d <= SMALL_MAX_D ? (512 + 32) * 4 : 0);
   {
     const size_t m = 2 * n;
     L.ad_cap = (uint32_t)((K + 7) & ~(int64_t)7);
@@ -2831,6 +2848,7 @@ int select_impl(mv_ctx* ctx, P p, const Layout& L, const uint8_t* votes, bool ha
   cudaStream_t st = ctx->stream;
   if (!have_hist) {
     ctx->clean_bytes = 0;
+    ctx->small_ready = false;  // (this call's layout may put its scratch where a small step keeps its state)
     if (cudaMemsetAsync(ctx->ws + L.votes_done, 0, L.zero_off + L.zero_bytes - L.votes_done, st) != cudaSuccess)
       return MV_ERR_CUDA;
     launch_k(k_vote_hist, dim3((p.nchunks + VH_WARPS - 1) / VH_WARPS), dim3(TPB), st, p, votes, (uint8_t*)nullptr);
@@ -2859,16 +2877,23 @@ int aggregate_impl(mv_ctx* ctx, float* acc, int N, int64_t d, int64_t K, const i
   return MV_OK;
 }
 
-// The single-kernel tail needs a cooperative launch with one CTA of FT threads and SK_KEYS keys of shared memory
-// per multiprocessor; asked once per context.
+// dynamic shared memory of the tail kernel: the candidate keys of a CTA's slice, later the output offsets
+// (nchunks + 1 words) and tie quotas (16 bits each) of all chunks
+size_t tail_smem_bytes(int nc_pad) {
+  const size_t table = ((size_t)nc_pad + 8) * 4 + (size_t)nc_pad * 2;
+  return table > (size_t)SK_KEYS * 4 ? table : (size_t)SK_KEYS * 4;
+}
+
+// The single-kernel tail needs a cooperative launch with one CTA of FT threads per multiprocessor and shared
+// memory for the largest table; asked once per context.
 bool tail_ready(mv_ctx* ctx) {
   if (ctx->tail_state == 0) {
     ctx->tail_state = -1;
     int dev = -1, coop = 0, per_sm = 0;
     if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) == cudaSuccess &&
         coop != 0 &&
-        cudaFuncSetAttribute(k_tail, cudaFuncAttributeMaxDynamicSharedMemorySize, SK_KEYS * 4) == cudaSuccess &&
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_tail, FT, SK_KEYS * 4) == cudaSuccess && per_sm >= 1)
+        cudaFuncSetAttribute(k_tail, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tail_smem_bytes(F_MAXCH)) == cudaSuccess &&
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_tail, FT, tail_smem_bytes(F_MAXCH)) == cudaSuccess && per_sm >= 1)
       ctx->tail_state = 1;
     else
       cudaGetLastError();
@@ -2905,7 +2930,7 @@ int tail_impl(mv_ctx* ctx, const P& p, const Layout& L, float* err, int32_t* out
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)ctx->sms);
   cfg.blockDim = dim3(FT);
-  cfg.dynamicSmemBytes = SK_KEYS * 4;
+  cfg.dynamicSmemBytes = tail_smem_bytes(p.nc_pad);
   cfg.stream = ctx->stream;
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeCooperative;
@@ -2964,40 +2989,64 @@ bool small_usable(mv_ctx* ctx, int N, int64_t d) {
 int small_impl(mv_ctx* ctx, const P& p, const Layout& L, const float* grads, float* err, int32_t* out_idx, float* out_val) {
   char* b = ctx->ws;
   cudaStream_t st = ctx->stream;
-  // the barrier words live in the region that is clear between steps; the two vote arrays are cleared here the
-  // first time (and after any other call that used the vote array), from then on by the kernel itself
-  if (ctx->clean_bytes < L.zero_bytes) {
-    if (cudaMemsetAsync(b + L.zero_off, 0, L.zero_bytes, st) != cudaSuccess) return MV_ERR_CUDA;
-    ctx->clean_bytes = L.zero_bytes;
-  }
+  // the kernel keeps its vote bytes, vote histogram and barrier word in two copies that alternate; both are cleared
+  // here the first time (and after any other call that used the vote array), from then on by the kernel itself
   const size_t vbytes = (size_t)L.nchunks * CH;
   if (!ctx->small_ready || ctx->small_N != p.N || ctx->small_d != p.d || ctx->small_K != p.K) {
     if (cudaMemsetAsync(b + L.votes, 0, vbytes, st) != cudaSuccess) return MV_ERR_CUDA;
     if (cudaMemsetAsync(b + L.votes_alt, 0, vbytes, st) != cudaSuccess) return MV_ERR_CUDA;
+    if (cudaMemsetAsync(b + L.small_state, 0, (512 + 32) * 4, st) != cudaSuccess) return MV_ERR_CUDA;
     ctx->small_flip = 0;
   }
+  uint32_t* const sst = (uint32_t*)(b + L.small_state);
+  const int f = ctx->small_flip;
   SmallArgs a;
   a.grads = grads;
   a.err = err;
   a.out_idx = out_idx;
   a.out_val = out_val;
-  a.votes_now = (uint32_t*)(b + (ctx->small_flip ? L.votes_alt : L.votes));
-  a.votes_next = (uint32_t*)(b + (ctx->small_flip ? L.votes : L.votes_alt));
-  a.words = (uint32_t*)(b + L.tail_words);
+  a.votes_now = (uint32_t*)(b + (f ? L.votes_alt : L.votes));
+  a.votes_next = (uint32_t*)(b + (f ? L.votes : L.votes_alt));
+  a.hist_now = sst + (f ? 256 : 0);
+  a.hist_next = sst + (f ? 0 : 256);
+  a.bar_now = sst + 512 + (f ? 16 : 0);
+  a.bar_next = sst + 512 + (f ? 0 : 16);
   a.abort_flag = (uint32_t*)(b + L.abort_flag);
   a.spin_limit = 1u << 21;
   a.dbg = p.dbg;
+  // threshold tracking as in the streaming path: a call that follows one of the same size reads the bounds that
+  // call left and leaves its own in the other array
+  const bool track = ctx->mode == MV_MODE_TRACK;
+  const bool tracked = track && ctx->track_valid && ctx->track_N == p.N && ctx->track_d == p.d && ctx->track_K == p.K;
+  if (tracked) ctx->tau_flip ^= 1;
+  a.tau_in = tracked ? (const uint32_t*)(b + (ctx->tau_flip ? L.tau_alt : L.tau)) : nullptr;
+  a.tau_out = track ? (uint32_t*)(b + (ctx->tau_flip ? L.tau : L.tau_alt)) : nullptr;
+  {
+    const double r = ceil((double)p.K * 1.35 + 6.0 * sqrt((double)p.K) + 8.0);
+    a.track_rank = (uint32_t)(r < (double)p.d ? r : (double)p.d);
+  }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)p.N);
   cfg.blockDim = dim3(FT);
   cfg.dynamicSmemBytes = SK_KEYS * 4;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeCooperative;
   attr[0].val.cooperative = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  if (cudaLaunchKernelEx(&cfg, k_small, p, a) != cudaSuccess) {
+  // launched early (the kernel waits for its predecessor on the stream at its start) if the runtime takes a
+  // cooperative launch that way; otherwise as a plain cooperative launch
+  cfg.numAttrs = ctx->tail_pdl >= 0 ? 2 : 1;
+  cudaError_t le = cudaLaunchKernelEx(&cfg, k_small, p, a);
+  if (le != cudaSuccess && cfg.numAttrs == 2) {
+    cudaGetLastError();
+    ctx->tail_pdl = -1;
+    cfg.numAttrs = 1;
+    le = cudaLaunchKernelEx(&cfg, k_small, p, a);
+  }
+  if (le != cudaSuccess) {
     cudaGetLastError();
     return MV_ERR_CUDA;
   }
@@ -3007,7 +3056,10 @@ int small_impl(mv_ctx* ctx, const P& p, const Layout& L, const float* grads, flo
   ctx->small_N = p.N;
   ctx->small_d = p.d;
   ctx->small_K = p.K;
-  ctx->track_valid = false;  // no threshold is carried out of this path
+  ctx->track_valid = track;
+  ctx->track_N = p.N;
+  ctx->track_d = p.d;
+  ctx->track_K = p.K;
   return MV_OK;
 }
 
@@ -3460,6 +3512,7 @@ int rs_select_impl(mv_ctx* ctx, const P& p, const Layout& L, const uint8_t* vote
   // region that a whole step of another size left cleared, so nothing counts as clean from here on
   // (a whole step that follows gets the zeros back from its last kernel).
   ctx->clean_bytes = 0;
+  ctx->small_ready = false;
   // one list that can hold every voted coordinate (at most min(d, N K) of them)
   const uint64_t room = (uint64_t)2 * (uint64_t)p.N * (uint64_t)L.ad_cap;
   P a = list_params(ctx, L, p, 1, p.K, (uint32_t)(room < 0xfffffff8ull ? room : 0xfffffff8ull));

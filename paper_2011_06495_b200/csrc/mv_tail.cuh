@@ -9,7 +9,8 @@
 //
 //   clear the votes | window histogram of the candidates          -- barrier 1
 //   bin of the K-th key, its keys to a short list                  -- barrier 2
-//   rank the list: T_n       [rare: three radix digits, +3 barriers, over the candidates or the full row]
+//   rank the list: T_n       [a crowded bin (very large K): its keys counted one by one, +1 barrier]
+//                            [rare: three radix digits, +3 barriers, over the candidates or the full row]
 //   picks: one vote per selected coordinate                        -- barrier 3
 //                            [rare: threshold ties kept only in part, ordered by index, +2 barriers]
 //   vote histogram per chunk and over the vector                   -- barrier 4
@@ -38,15 +39,16 @@ __device__ unsigned g_stamp_calls;
 #endif
 
 constexpr int FT = 1024;         // threads per CTA of the tail kernel (== ST: smem_pick2 and chunk_scan<ST> are shared)
-constexpr int F_MAXCH = 8192;    // most chunks (padded to eight) whose output offsets fit the shared-memory table
-constexpr int F_RADIX = 5120;    // per worker: 2048 + 2048 + 1024 counters of the three-digit route
+constexpr int F_MAXCH = 32768;   // most chunks (padded to eight) whose output offsets fit the shared-memory table
+constexpr int F_RADIX = 7168;    // per worker: 2048 + 2048 + 1024 counters of the three-digit route, 2048 of the second count
 
 struct TailArgs {
   float* err;               // [N][d] acc on entry, the residual on exit
   int32_t* out_idx;         // [K]
   float* out_val;           // [K]
   uint32_t* words;          // [16] in the cleared region: 0 barrier arrivals, 1 exit ticket, 2 "a worker needs the
-                            //      three-digit route", 3 "a worker keeps its threshold ties only in part"
+                            //      three-digit route", 3 "a worker keeps its threshold ties only in part", 4 "a worker
+                            //      counts the keys of its crowded bin a second time"
   uint32_t* abort_flag;     // workspace header: set for good when a barrier wait gave up
   uint32_t* radix;          // [N][F_RADIX] digit counts of the three-digit route
   uint4* zero_ptr;          // start of the scratch region that must be clear when the next step starts
@@ -151,7 +153,8 @@ __device__ __forceinline__ uint32_t tau_below(uint32_t tau, uint32_t key_K, uint
 }
 
 __global__ void __launch_bounds__(FT, 1) k_tail(P p, TailArgs a) {
-  extern __shared__ uint32_t dsm[];      // SK_KEYS words: the slice's keys | vote-histogram scratch | output offsets
+  extern __shared__ uint32_t dsm[];      // max(SK_KEYS, 1.5 nc_pad + 8) words: the slice's keys | vote-histogram scratch |
+                                         // output offsets and tie quotas of all chunks
   __shared__ uint32_t s_hw[H1_BINS];     // this CTA's counts (window, then one radix digit at a time)
   __shared__ uint32_t s_m[H1_BINS];      // the worker's counts: all CTAs of its group together
   __shared__ uint32_t s_ws[FT / 32];
@@ -247,9 +250,11 @@ __global__ void __launch_bounds__(FT, 1) k_tail(P p, TailArgs a) {
   if (!grid_barrier(bar)) return;  // 1
   TAIL_STAMP(2);
 
-  // ---- the bin that holds rank K; its keys go to the worker's short list ----
-  bool will_resolve = false;
+  // ---- the bin that holds rank K; its keys go to the worker's short list.  A bin too crowded for that (rows so
+  // long that many elements share every magnitude near the threshold) is counted a second time, key by key ----
+  bool will_resolve = false, lvl2 = false;
   uint32_t bw = 0, rem = 0, bt = 0, trem_w = 0;
+  uint32_t* R4 = R1 + 5120;  // the worker's second count: keys of bin bw by their low WIN_SHIFT bits
   if (has && fast) {
     uint32_t wsum = 0;
     for (int bb = tid; bb < H1_BINS; bb += FT) {
@@ -277,11 +282,22 @@ __global__ void __launch_bounds__(FT, 1) k_tail(P p, TailArgs a) {
           }
         }
       } else {
+        lvl2 = true;
         if (rank == 0 && tid == 0) MV_DBG(a.dbg, MV_DBG_WINDOW_OVERFLOW);
+        __syncthreads();
+        for (int bb = tid; bb < H1_BINS; bb += FT) s_hw[bb] = 0;
+        __syncthreads();
+        for (uint32_t li = tid; li < len; li += FT) {
+          const uint32_t kk = li < SK_KEYS ? s_keys[li] : __ldcg(&cd[s0 + li].x);
+          if (((kk - tau) >> WIN_SHIFT) == bw) atomicAdd(&s_hw[(kk - tau) & ((1u << WIN_SHIFT) - 1u)], 1u);
+        }
+        __syncthreads();
+        flush_counts(s_hw, R4, 1 << WIN_SHIFT);
+        if (tid == 0) atomicOr(a.words + 4, 1u);
       }
     }
   }
-  const bool need_slow = has && !will_resolve;  // a full-row worker, or a K-th key outside the window or in a crowded bin
+  bool need_slow = has && !will_resolve && !lvl2;  // a full-row worker, or a K-th key outside the window
   if (need_slow && tid == 0) atomicOr(a.words + 2, 1u);
   TAIL_STAMP(3);
   if (!grid_barrier(bar)) return;  // 2
@@ -326,6 +342,60 @@ __global__ void __launch_bounds__(FT, 1) k_tail(P p, TailArgs a) {
     }
     if (tracking && rank == 0 && tid == 0)
       p.tau_next[n] = trem_w != 0 ? tau + (bt << WIN_SHIFT) : tau_below(tau, T, cnt, K, p.track_rank);
+  }
+
+  // ---- the second count (the same decision in every CTA of the grid: the flag was written before barrier 2): the
+  // worker's keys of bin bw, one counter per key, give T_n, cnt_eq and need directly; ties kept only in part go to
+  // the short list with their coordinates, and the lowest coordinates among them vote ----
+  bool tie_listed = will_resolve;  // the worker's partly kept ties (if any) are settled through the short list
+  if (ld_acquire(a.words + 4) != 0u) {
+    bool list_ties = false;
+    if (lvl2) {
+      for (int bb = tid; bb < H1_BINS; bb += FT) s_m[bb] = __ldcg(&R4[bb]);
+      __syncthreads();
+      uint32_t b2, u0, u1;
+      smem_pick2<H1_BINS>(s_m, rem, 0u, b2, need, u0, u1);
+      T = tau + (bw << WIN_SHIFT) + b2;
+      cnt_eq = s_m[b2];
+      if (need < cnt_eq) {
+        if (cnt_eq <= (uint32_t)WIN_LIST) {
+          list_ties = true;
+          for (uint32_t li = tid; li < len; li += FT) {
+            const uint32_t kk = li < SK_KEYS ? s_keys[li] : __ldcg(&cd[s0 + li].x);
+            if (kk == T) {
+              const uint32_t at = atomicAdd(lcnt, 1u);
+              if (at < (uint32_t)WIN_LIST) lidx[at] = __ldcg(&cd[s0 + li].y);
+              else MV_DBG(a.dbg, MV_DBG_INTERNAL);
+            }
+          }
+        } else {  // more equal keys than the list holds: their order comes from the per-chunk route below
+          lvl2 = false;
+        }
+      }
+      if (tracking && rank == 0 && tid == 0)
+        p.tau_next[n] = trem_w != 0 ? tau + (bt << WIN_SHIFT) : tau_below(tau, T, cnt, K, p.track_rank);
+    }
+    if (!grid_barrier(bar)) return;  // +1
+    if (list_ties) {
+      tie_listed = true;
+      const uint32_t m = min(__ldcg(lcnt), (uint32_t)WIN_LIST);
+      uint32_t myidx = 0;
+      if ((uint32_t)tid < m) {
+        myidx = __ldcg(lidx + tid);
+        s_hw[tid] = myidx;
+      }
+      __syncthreads();
+      if (rank == 0 && (uint32_t)tid < m) {
+        uint32_t tie_lt = 0;
+        for (uint32_t i = 0; i < m; i++) tie_lt += s_hw[i] < myidx ? 1u : 0u;
+        if (tie_lt < need) {
+          if ((int64_t)myidx < p.d) add_vote(p.vote_words, myidx);
+          else MV_DBG(a.dbg, MV_DBG_PICK_RANGE);
+        }
+      }
+    } else if (lvl2) {
+      tie_listed = true;  // (every tie is kept, or none is left open)
+    }
   }
 
   // ---- rare: three radix digits (11 + 10 + 10 bits) for the workers that are not resolved yet, over their
@@ -416,18 +486,26 @@ __global__ void __launch_bounds__(FT, 1) k_tail(P p, TailArgs a) {
     }
   }
   const bool all_ties = need >= cnt_eq;  // alike in all CTAs of the group
-  const bool ties_open = !all_ties && !will_resolve;  // partly kept ties that still have to be put in index order
+  const bool ties_open = !all_ties && !tie_listed;  // partly kept ties that still have to be put in index order
 
   TAIL_STAMP(5);
   // ---- picks: every selected coordinate gets one more vote.  A worker that keeps only part of its threshold
   // ties (lowest index first) votes for the keys above T_n now and counts its ties per chunk; the ties follow. ----
   if (has) {
     if (fast) {
-      for (uint32_t li = tid; li < len; li += FT) {
-        const uint2 kv = __ldcg(&cd[s0 + li]);
-        if (kv.x > T || (kv.x == T && all_ties)) {
-          if ((int64_t)kv.y < p.d) add_vote(p.vote_words, kv.y);
-          else MV_DBG(a.dbg, MV_DBG_PICK_RANGE);
+      for (uint32_t l0 = 0; l0 < len; l0 += FT * 4) {  // (four candidates in flight per thread)
+        uint2 kv[4];
+#pragma unroll
+        for (int q = 0; q < 4; q++) {
+          const uint32_t li = l0 + q * FT + tid;
+          kv[q] = li < len ? __ldcg(&cd[s0 + li]) : make_uint2(0u, 0u);
+        }
+#pragma unroll
+        for (int q = 0; q < 4; q++) {
+          if (l0 + q * FT + tid < len && (kv[q].x > T || (kv[q].x == T && all_ties))) {
+            if ((int64_t)kv[q].y < p.d) add_vote(p.vote_words, kv[q].y);
+            else MV_DBG(a.dbg, MV_DBG_PICK_RANGE);
+          }
         }
       }
       if (ties_open) {
@@ -565,45 +643,51 @@ __global__ void __launch_bounds__(FT, 1) k_tail(P p, TailArgs a) {
   __syncthreads();
   const uint32_t vstar = s_vs[0], quota = s_vs[3];
 
-  // ---- output offset of every chunk and the v*-ties it keeps (lowest index first): a scan over the chunks' counts,
-  // thread t taking chunks 8t .. 8t+7; every CTA computes the whole table, in shared memory ----
-  uint32_t* s_ob = dsm;                                                  // [nchunks + 1]
-  uint16_t* s_tk = reinterpret_cast<uint16_t*>(dsm + F_MAXCH + 8);       // [nchunks]
+  // ---- output offset of every chunk and the v*-ties it keeps (lowest index first): a scan over the chunks' counts
+  // in tiles of 8 FT chunks, thread t taking chunks 8t .. 8t+7 of the tile; every CTA computes the whole table, in
+  // shared memory (ecarry / scarry: v*-ties seen and outputs placed in the tiles before) ----
+  uint32_t* s_ob = dsm;                                                  // [nc_pad + 8]: nchunks + 1 offsets
+  uint16_t* s_tk = reinterpret_cast<uint16_t*>(dsm + p.nc_pad + 8);      // [nc_pad]
   {
     const uint16_t* hge = p.chunk_vh + (size_t)vstar * p.nc_pad;                                    // votes >= v*
     const uint16_t* hgt = (int)vstar < p.N ? p.chunk_vh + (size_t)(vstar + 1) * p.nc_pad : nullptr;  // votes > v*
-    const int c = tid * 8;
-    uint4 av = make_uint4(0, 0, 0, 0), gv = make_uint4(0, 0, 0, 0);
-    if (c < p.nc_pad) {
-      av = __ldcg(reinterpret_cast<const uint4*>(hge + c));
-      if (hgt) gv = __ldcg(reinterpret_cast<const uint4*>(hgt + c));
-    }
-    const uint32_t aw[4] = {av.x, av.y, av.z, av.w}, gw[4] = {gv.x, gv.y, gv.z, gv.w};
-    uint32_t eqv[8], gtv[8], esum = 0, gsum = 0;
-#pragma unroll
-    for (int q = 0; q < 8; q++) {
-      const uint32_t ge = (aw[q >> 1] >> (16 * (q & 1))) & 0xffffu, gt = (gw[q >> 1] >> (16 * (q & 1))) & 0xffffu;
-      const bool in = c + q < p.nchunks;
-      eqv[q] = in ? ge - gt : 0u;
-      gtv[q] = in ? gt : 0u;
-      esum += eqv[q];
-      gsum += gtv[q];
-    }
-    uint32_t etot, stot;
-    const uint32_t epre = block_excl_scan<FT>(esum, s_sw, etot);
-    const uint32_t taken_before = epre < quota ? epre : quota;           // ties kept in earlier chunks
-    const uint32_t taken_here = min(epre + esum, quota) - taken_before;  // ties kept in this thread's chunks
-    const uint32_t spre = block_excl_scan<FT>(gsum + taken_here, s_sw, stot);
-    uint32_t run = epre, srun = spre;
-#pragma unroll
-    for (int q = 0; q < 8; q++) {
-      const uint32_t take = run >= quota ? 0u : min(eqv[q], quota - run);
-      if (c + q < p.nchunks) {
-        s_ob[c + q] = srun;
-        s_tk[c + q] = (uint16_t)take;
+    uint32_t ecarry = 0, scarry = 0;
+    for (int c0 = 0; c0 < p.nc_pad; c0 += FT * 8) {  // uniform over the CTA
+      const int c = c0 + tid * 8;
+      uint4 av = make_uint4(0, 0, 0, 0), gv = make_uint4(0, 0, 0, 0);
+      if (c < p.nc_pad) {
+        av = __ldcg(reinterpret_cast<const uint4*>(hge + c));
+        if (hgt) gv = __ldcg(reinterpret_cast<const uint4*>(hgt + c));
       }
-      run += eqv[q];
-      srun += gtv[q] + take;
+      const uint32_t aw[4] = {av.x, av.y, av.z, av.w}, gw[4] = {gv.x, gv.y, gv.z, gv.w};
+      uint32_t eqv[8], gtv[8], esum = 0, gsum = 0;
+#pragma unroll
+      for (int q = 0; q < 8; q++) {
+        const uint32_t ge = (aw[q >> 1] >> (16 * (q & 1))) & 0xffffu, gt = (gw[q >> 1] >> (16 * (q & 1))) & 0xffffu;
+        const bool in = c + q < p.nchunks;
+        eqv[q] = in ? ge - gt : 0u;
+        gtv[q] = in ? gt : 0u;
+        esum += eqv[q];
+        gsum += gtv[q];
+      }
+      uint32_t etot, stot;
+      const uint32_t epre = ecarry + block_excl_scan<FT>(esum, s_sw, etot);
+      const uint32_t taken_before = epre < quota ? epre : quota;           // ties kept in earlier chunks
+      const uint32_t taken_here = min(epre + esum, quota) - taken_before;  // ties kept in this thread's chunks
+      const uint32_t spre = scarry + block_excl_scan<FT>(gsum + taken_here, s_sw, stot);
+      uint32_t run = epre, srun = spre;
+#pragma unroll
+      for (int q = 0; q < 8; q++) {
+        const uint32_t take = run >= quota ? 0u : min(eqv[q], quota - run);
+        if (c + q < p.nchunks) {
+          s_ob[c + q] = srun;
+          s_tk[c + q] = (uint16_t)take;
+        }
+        run += eqv[q];
+        srun += gtv[q] + take;
+      }
+      ecarry += etot;
+      scarry += stot;
     }
     if (tid == 0) s_ob[p.nchunks] = K;
   }

@@ -171,3 +171,19 @@ def test_sweep_cell(w):
     assert torch.equal(oi2, out_idx) and torch.equal(ov2.view(torch.int32), out_val.view(torch.int32))
     assert torch.equal(err0.view(torch.int32), acc.view(torch.int32))
     assert int(ctx.read_diag(N)[:, 2].sum()) == 0
+
+
+def test_crowded_threshold_bin_in_the_single_kernel_tail():
+    """A long row on a fine grid of magnitudes: near the K-th key every level of the grid is shared by about a
+    hundred elements and the 2048-key bin of rank K holds more than a thousand, so the single-kernel tail counts
+    that bin a second time, key by key, and settles the partly kept ties of T_n through their coordinates.
+    Everything against the oracle, the kernel sequence included."""
+    N, d = 2, 1 << 26
+    K = d // 100
+    g = torch.Generator(device=DEV).manual_seed(4242)
+    grads = (torch.randn((N, d), generator=g, device=DEV) * 32768).round_() / 32768
+    err0 = torch.zeros((N, d), device=DEV)
+    ctx = B.MvContext(N, d, K, device=DEV)
+    ref = O.mv_sparse_step(PT.npy(grads), PT.npy(err0), K, threads=THREADS)
+    assert (ref["thresh"][:, 2] > ref["thresh"][:, 1] * 0 + 1).all()       # T_n is shared by several elements
+    PT.compare_all(ctx, grads, err0, K, ref=ref, label="[crowded bin] ")

@@ -649,3 +649,75 @@ def test_single_kernel_step_for_rows_that_fit_a_cta(mode):
         PT.check_out_val(PT.npy(out_val), ref, ref["acc"], ref["out_idx"].astype(np.int64), f"step {step} out_val")
         PT.first_diff(PT.bits(PT.npy(err_gpu)), PT.bits(ref["err"]), f"step {step} ({kind}) err")
         err_ref = ref["err"]
+
+
+@pytest.mark.parametrize("mode", [B.MV_MODE_AUTO, B.MV_MODE_TRACK], ids=["auto", "track"])
+def test_single_kernel_step_routes_to_the_kth_key(mode):
+    """The one-kernel step finds T_n from a lower bound (carried or sampled) and falls back to three radix digits.
+    Steps that take each route, on one context, against the oracle: a carried bound that suddenly lies far above every
+    key (residual reset, gradients 1e-4 times smaller), one far below (1e3 times larger), a row of a few distinct
+    magnitudes (the bin of rank K is too crowded to rank: radix digits), all-equal magnitudes, and a selection of
+    another size in between, whose scratch lands where the kernel keeps its alternating state."""
+    N, d, K = 5, 30_001, 300
+    g = torch.Generator().manual_seed(77)
+    ctx = B.MvContext(N, d, K, device=DEV, mode=mode)
+    err_gpu = torch.zeros(N, d, device=DEV)
+    err_ref = np.zeros((N, d), dtype=np.float32)
+    plan = [("gauss", 1.0, False), ("gauss", 1.0, False), ("gauss", 1e-4, True), ("gauss", 1.0, False), ("gauss", 1e3, False),
+            ("coarse", 1.0, True), ("gauss", 1.0, False), ("equal", 1.0, True), ("other", 1.0, False), ("gauss", 1.0, False),
+            ("gauss", 1.0, False)]
+    for step, (kind, scale, reset) in enumerate(plan):
+        grads = torch.randn(N, d, generator=g) * scale
+        if kind == "coarse":
+            grads = (grads * 2).round() / 2
+        if kind == "equal":
+            grads = torch.full((N, d), 0.75)
+            grads[:, ::3] *= -1
+        if reset:
+            err_gpu.zero_()
+            err_ref[:] = 0
+        if kind == "other":      # mv_select for another problem size on the same context
+            d2, K2 = 25_000, 100
+            votes2 = torch.randint(0, N + 1, (d2,), generator=g).to(torch.uint8).to(DEV)
+            oi2 = torch.empty(K2, dtype=torch.int32, device=DEV)
+            ctx.mv_select(votes2, N, oi2, K=K2)
+            torch.cuda.synchronize()
+            assert np.array_equal(oi2.cpu().numpy(), O.select_mask(votes2.cpu().numpy(), K2)[0])
+        ref = O.mv_sparse_step(grads.numpy(), err_ref, K)
+        out_idx = torch.full((K,), -7, dtype=torch.int32, device=DEV)
+        out_val = torch.full((K,), float("nan"), dtype=torch.float32, device=DEV)
+        ctx.mv_sparse_step(grads.to(DEV), err_gpu, out_idx, out_val, K=K)
+        torch.cuda.synchronize()
+        assert ctx.last_launches() == 1
+        PT.first_diff(PT.npy(out_idx), ref["out_idx"], f"step {step} ({kind} x{scale}) out_idx")
+        PT.check_out_val(PT.npy(out_val), ref, ref["acc"], ref["out_idx"].astype(np.int64), f"step {step} out_val")
+        PT.first_diff(PT.bits(PT.npy(err_gpu)), PT.bits(ref["err"]), f"step {step} ({kind}) err")
+        err_ref = ref["err"]
+
+
+@pytest.mark.parametrize("N,d,K", [(4, 10_000, 100), (5, 300_007, 3000)], ids=["one-kernel step", "single-kernel tail"])
+def test_a_wait_that_was_given_up_is_reported(N, d, K):
+    """The two persistent kernels bound their grid-barrier waits; a CTA that gives up sets a sticky word in the
+    workspace header, every CTA that sees it leaves at its next barrier, and the calls that wait for the stream
+    return MV_ERR_TIMEOUT.  Here the word is set by the host before the launch (no wait actually runs out): the
+    kernel leaves at its first barrier, the status comes back through the ABI, and the CUDA context stays usable
+    (a fresh context on the same stream gives the oracle's result afterwards)."""
+    grads, err = make(N, d, "gauss", seed=5)
+    ctx = B.MvContext(N, d, K, device=DEV)
+    ctx.set_tail_kernel(2)
+    out_idx = torch.empty(K, dtype=torch.int32, device=DEV)
+    out_val = torch.empty(K, dtype=torch.float32, device=DEV)
+    e = err.to(DEV)
+    ctx.mv_sparse_step(grads.to(DEV), e, out_idx, out_val)       # (the first call clears the header)
+    torch.cuda.synchronize()
+    assert ctx.fallback_count() >= 0
+    ctx.workspace[8:12] = torch.tensor([1, 0, 0, 0], dtype=torch.uint8, device=DEV)   # header word 2: "a wait gave up"
+    ctx.mv_sparse_step(grads.to(DEV), e, out_idx, out_val)
+    with pytest.raises(B.MvError) as ei:
+        ctx.read_diag(N)
+    assert ei.value.status == B.MV_ERR_TIMEOUT
+    assert "wait" in B.status_string(B.MV_ERR_TIMEOUT).lower()
+    torch.cuda.synchronize()
+    ctx.close()
+    ctx2 = B.MvContext(N, d, K, device=DEV)
+    PT.compare_all(ctx2, grads.to(DEV), err.to(DEV), K, label="[after a reported timeout] ")
