@@ -46,9 +46,9 @@ struct TailArgs {
   float* err;               // [N][d] acc on entry, the residual on exit
   int32_t* out_idx;         // [K]
   float* out_val;           // [K]
-  uint32_t* words;          // [16] in the cleared region: 0 barrier arrivals, 1 exit ticket, 2 "a worker needs the
-                            //      three-digit route", 3 "a worker keeps its threshold ties only in part", 4 "a worker
-                            //      counts the keys of its crowded bin a second time"
+  uint32_t* words;          // [16] in the cleared region: 0 barrier arrivals, 1 exit ticket, 2 bit 0 "a worker needs the
+                            //      three-digit route", bit 1 "a worker counts the keys of its crowded bin a second
+                            //      time", 3 "a worker keeps its threshold ties only in part"
   uint32_t* abort_flag;     // workspace header: set for good when a barrier wait gave up
   uint32_t* radix;          // [N][F_RADIX] digit counts of the three-digit route
   uint4* zero_ptr;          // start of the scratch region that must be clear when the next step starts
@@ -217,6 +217,7 @@ __global__ void __launch_bounds__(FT, 1) k_tail(P p, TailArgs a) {
   }
   uint32_t* R2 = R1 + 2048;
   uint32_t* R3 = R1 + 4096;
+  uint32_t* R4 = R1 + 5120;  // the worker's second count: keys of bin bw by their low WIN_SHIFT bits
   uint32_t* gh = p.hist1 + (size_t)(has ? n : 0) * H1_BINS;   // the worker's window counts
   uint32_t* lcnt = p.hist3 + (size_t)(has ? n : 0) * H3_BINS;  // length of its short list ...
   uint32_t* list = p.hist2 + (size_t)(has ? n : 0) * H2_BINS;  // ... of the keys in the bin of rank K
@@ -254,7 +255,6 @@ __global__ void __launch_bounds__(FT, 1) k_tail(P p, TailArgs a) {
   // long that many elements share every magnitude near the threshold) is counted a second time, key by key ----
   bool will_resolve = false, lvl2 = false;
   uint32_t bw = 0, rem = 0, bt = 0, trem_w = 0;
-  uint32_t* R4 = R1 + 5120;  // the worker's second count: keys of bin bw by their low WIN_SHIFT bits
   if (has && fast) {
     uint32_t wsum = 0;
     for (int bb = tid; bb < H1_BINS; bb += FT) {
@@ -293,7 +293,7 @@ __global__ void __launch_bounds__(FT, 1) k_tail(P p, TailArgs a) {
         }
         __syncthreads();
         flush_counts(s_hw, R4, 1 << WIN_SHIFT);
-        if (tid == 0) atomicOr(a.words + 4, 1u);
+        if (tid == 0) atomicOr(a.words + 2, 2u);
       }
     }
   }
@@ -304,41 +304,71 @@ __global__ void __launch_bounds__(FT, 1) k_tail(P p, TailArgs a) {
   TAIL_STAMP(4);
 
   uint32_t T = 0, need = 0, cnt_eq = 0;
+  uint32_t flags2 = 0;  // the detours that some worker of the grid needs (written before barrier 2, so alike in every CTA)
   if (will_resolve) {
     // rank the list: T_n is its rem-th largest key
     // (the list holds every candidate whose key equals T_n, with its coordinate: a thread that holds such a tie
     // also learns how many ties precede it in index order, which settles the ties without any pass of its own)
+    // (the list's length, its entries -- slot tid exists whatever the length -- and the flags are asked for together)
+    uint32_t mine = __ldcg(list + tid), myidx = __ldcg(lidx + tid), tie_lt = 0;
     const uint32_t m = __ldcg(lcnt);
-    uint32_t mine = 0, myidx = 0, tie_lt = 0;
-    if ((uint32_t)tid < m) {
-      mine = __ldcg(list + tid);
-      myidx = __ldcg(lidx + tid);
-      s_m[tid] = mine;
-      s_hw[tid] = myidx;
-    }
-    __syncthreads();
-    if ((uint32_t)tid < m) {
-      uint32_t gt = 0, eq = 0;
-      for (uint32_t i = 0; i < m; i++) {
-        const uint32_t o = s_m[i];
-        gt += o > mine;
-        eq += o == mine;
-        tie_lt += (o == mine && s_hw[i] < myidx) ? 1u : 0u;
+    flags2 = ld_acquire(a.words + 2);
+    if (m <= 96u) {  // a short list: every key against every key (alike in all threads)
+      if ((uint32_t)tid < m) {
+        s_m[tid] = mine;
+        s_hw[tid] = myidx;
       }
-      if (gt < rem && rem <= gt + eq) {  // every thread that holds T_n writes the same values
-        s_res3[0] = mine;
-        s_res3[1] = rem - gt;
-        s_res3[2] = eq;
+      __syncthreads();
+      if ((uint32_t)tid < m) {
+        uint32_t gt = 0, eq = 0;
+        for (uint32_t i = 0; i < m; i++) {
+          const uint32_t o = s_m[i];
+          gt += o > mine;
+          if (o == mine) {
+            eq++;
+            tie_lt += s_hw[i] < myidx ? 1u : 0u;
+          }
+        }
+        if (gt < rem && rem <= gt + eq) {  // every thread that holds T_n writes the same values
+          s_res3[0] = mine;
+          s_res3[1] = rem - gt;
+          s_res3[2] = eq;
+        }
       }
-    }
-    __syncthreads();
-    T = s_res3[0];
-    need = s_res3[1];
-    cnt_eq = s_res3[2];
-    // ties kept only in part: the `need` lowest coordinates among them vote here (one CTA of the group does it)
-    if (need < cnt_eq && rank == 0 && (uint32_t)tid < m && mine == T && tie_lt < need) {
-      if ((int64_t)myidx < p.d) add_vote(p.vote_words, myidx);
-      else MV_DBG(a.dbg, MV_DBG_PICK_RANGE);
+      __syncthreads();
+      T = s_res3[0];
+      need = s_res3[1];
+      cnt_eq = s_res3[2];
+      // ties kept only in part: the `need` lowest coordinates among them vote here (one CTA of the group does it)
+      if (need < cnt_eq && rank == 0 && (uint32_t)tid < m && mine == T && tie_lt < need) {
+        if ((int64_t)myidx < p.d) add_vote(p.vote_words, myidx);
+        else MV_DBG(a.dbg, MV_DBG_PICK_RANGE);
+      }
+    } else {
+      // a longer list (the pairwise count grows with its square): the list's keys all lie in bin bw, so their low
+      // WIN_SHIFT bits tell them apart; one counter per key value, and the rem-th largest is read off the counts
+      __syncthreads();
+      for (int bb = tid; bb < H1_BINS; bb += FT) s_hw[bb] = 0;
+      if (tid == 0) s_res3[0] = 0;
+      __syncthreads();
+      if ((uint32_t)tid < m) atomicAdd(&s_hw[(mine - tau) & ((1u << WIN_SHIFT) - 1u)], 1u);
+      __syncthreads();
+      uint32_t b2, u0, u1;
+      smem_pick2<H1_BINS>(s_hw, rem, 0u, b2, need, u0, u1);
+      T = tau + (bw << WIN_SHIFT) + b2;
+      cnt_eq = s_hw[b2];
+      if (need < cnt_eq && rank == 0) {  // alike in all threads: the ties, by coordinate, among themselves
+        const bool tie = (uint32_t)tid < m && mine == T;
+        if (tie) s_m[atomicAdd(&s_res3[0], 1u)] = myidx;
+        __syncthreads();
+        if (tie) {
+          for (uint32_t i = 0; i < cnt_eq; i++) tie_lt += s_m[i] < myidx ? 1u : 0u;
+          if (tie_lt < need) {
+            if ((int64_t)myidx < p.d) add_vote(p.vote_words, myidx);
+            else MV_DBG(a.dbg, MV_DBG_PICK_RANGE);
+          }
+        }
+      }
     }
     if (tracking && rank == 0 && tid == 0)
       p.tau_next[n] = trem_w != 0 ? tau + (bt << WIN_SHIFT) : tau_below(tau, T, cnt, K, p.track_rank);
@@ -348,7 +378,8 @@ __global__ void __launch_bounds__(FT, 1) k_tail(P p, TailArgs a) {
   // worker's keys of bin bw, one counter per key, give T_n, cnt_eq and need directly; ties kept only in part go to
   // the short list with their coordinates, and the lowest coordinates among them vote ----
   bool tie_listed = will_resolve;  // the worker's partly kept ties (if any) are settled through the short list
-  if (ld_acquire(a.words + 4) != 0u) {
+  if (!will_resolve) flags2 = ld_acquire(a.words + 2);
+  if ((flags2 & 2u) != 0u) {
     bool list_ties = false;
     if (lvl2) {
       for (int bb = tid; bb < H1_BINS; bb += FT) s_m[bb] = __ldcg(&R4[bb]);
@@ -401,7 +432,7 @@ __global__ void __launch_bounds__(FT, 1) k_tail(P p, TailArgs a) {
   // ---- rare: three radix digits (11 + 10 + 10 bits) for the workers that are not resolved yet, over their
   // candidates or, for a worker whose candidate count missed [K, cap], over its full row.  Whether this part
   // runs is the same for the whole grid (the flag was written before barrier 2). ----
-  if (ld_acquire(a.words + 2) != 0u) {
+  if ((flags2 & 1u) != 0u) {
     uint32_t b1 = 0, rem1 = 0, tb = 0, trem = 0, b2 = 0, rem2 = 0, tb2 = 0, trem2 = 0;
     auto slice_keys = [&](auto f) {
       if (fast) {
@@ -694,76 +725,80 @@ __global__ void __launch_bounds__(FT, 1) k_tail(P p, TailArgs a) {
   __syncthreads();
 
   TAIL_STAMP(11);
-  // ---- supp(M), ascending: a warp per chunk that holds outputs, the chunks dealt out over all warps of the grid ----
+  // ---- supp(M), ascending: a warp per chunk that holds outputs, the chunks dealt out over all warps of the grid.
+  // Lane l owns the chunk's coordinates [128 l, 128 l + 128), so lane order is index order and one scan over the
+  // lanes places the outputs (a second one, only in a chunk that keeps part of its v*-ties, places those) ----
   {
+    const uint32_t vs4 = vstar * 0x01010101u;
     for (int c = warp * G + b; c < p.nchunks; c += G * (FT / 32)) {
       const uint32_t ob = s_ob[c];
       if (s_ob[c + 1] == ob) continue;  // no coordinate of this chunk is in the mask
       const uint32_t tk = s_tk[c];
-      uint32_t orun = 0, erun = 0;  // outputs placed and v*-ties seen so far in this chunk
-      uint4 qv[8];                  // lane l owns bytes 16 (32 u + l) .. + 15 of round u: index order is (u, lane)
+      const int64_t jl = (int64_t)c * CH + (int64_t)lane * 128;  // the lane's first coordinate
+      uint4 qv[8];
 #pragma unroll
       for (int u = 0; u < 8; u++) {
-        const int64_t jb = (int64_t)c * CH + (int64_t)(u * 32 + lane) * 16;
+        const int64_t jb = jl + 16 * u;
         qv[u] = jb < p.d ? __ldcg(reinterpret_cast<const uint4*>(p.votes + jb)) : make_uint4(0, 0, 0, 0);
       }
+      // one bit per coordinate: votes > v*, votes == v* (byte compares give 0xff per hit; a multiply gathers one bit
+      // of each of the four bytes); coordinates at or beyond d are left out
+      uint32_t gm[4] = {0, 0, 0, 0}, em[4] = {0, 0, 0, 0};
 #pragma unroll
       for (int u = 0; u < 8; u++) {
-        const int64_t jb = (int64_t)c * CH + (int64_t)(u * 32 + lane) * 16;
-        const uint4 q = qv[u];
-        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-        // one bit per byte: votes > v*, votes == v* (byte compares give 0xff per hit; a multiply gathers one bit of
-        // each of the four bytes); bytes at or beyond d are left out
-        uint32_t gm = 0, em = 0;
+        const uint32_t w[4] = {qv[u].x, qv[u].y, qv[u].z, qv[u].w};
         if (vstar == 0u || (w[0] | w[1] | w[2] | w[3]) != 0u) {
-          const uint32_t vs4 = vstar * 0x01010101u;
+          uint32_t g16 = 0, e16 = 0;
 #pragma unroll
           for (int i = 0; i < 4; i++) {
-            gm |= (((__vcmpgtu4(w[i], vs4) & 0x01010101u) * 0x01020408u) >> 24) << (4 * i);
-            em |= (((__vcmpeq4(w[i], vs4) & 0x01010101u) * 0x01020408u) >> 24) << (4 * i);
+            g16 |= (((__vcmpgtu4(w[i], vs4) & 0x01010101u) * 0x01020408u) >> 24) << (4 * i);
+            e16 |= (((__vcmpeq4(w[i], vs4) & 0x01010101u) * 0x01020408u) >> 24) << (4 * i);
           }
-          const int64_t left = p.d - jb;  // bytes of this piece that are coordinates
+          const int64_t left = p.d - (jl + 16 * u);  // bytes of this piece that are coordinates
           const uint32_t inb = left >= 16 ? 0xffffu : (left <= 0 ? 0u : (1u << (int)left) - 1u);
-          gm &= inb;
-          em &= inb;
+          gm[u >> 1] |= (g16 & inb) << (16 * (u & 1));
+          em[u >> 1] |= (e16 & inb) << (16 * (u & 1));
         }
-        uint32_t sm = gm;
-        if (tk > 0 && erun < tk) {  // uniform over the warp
-          const uint32_t pe = __popc(em);
-          uint32_t x = pe;
-#pragma unroll
-          for (int off = 1; off < 32; off <<= 1) {
-            const uint32_t y = __shfl_up_sync(FULL, x, off);
-            if (lane >= off) x += y;
-          }
-          const uint32_t before = erun + x - pe;
-          if (before < tk) {
-            uint32_t room = tk - before, e2 = em;
-            while (e2 && room) {
-              const uint32_t low = e2 & (0u - e2);
-              sm |= low;
-              e2 ^= low;
-              room--;
-            }
-          }
-          erun += __shfl_sync(FULL, x, 31);
-        }
-        const uint32_t ps = __popc(sm);
-        uint32_t x = ps;
+      }
+      if (tk > 0) {  // uniform over the warp: the chunk's first tk v*-ties, in index order, are kept
+        const uint32_t pe = __popc(em[0]) + __popc(em[1]) + __popc(em[2]) + __popc(em[3]);
+        uint32_t x = pe;
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
           const uint32_t y = __shfl_up_sync(FULL, x, off);
           if (lane >= off) x += y;
         }
-        uint32_t pos = ob + orun + x - ps;
+        const uint32_t before = x - pe;
+        uint32_t room = before < tk ? tk - before : 0u;
+#pragma unroll
+        for (int i = 0; i < 4; i++) {
+          uint32_t e2 = em[i];
+          while (e2 && room) {
+            const uint32_t low = e2 & (0u - e2);
+            gm[i] |= low;
+            e2 ^= low;
+            room--;
+          }
+        }
+      }
+      const uint32_t ps = __popc(gm[0]) + __popc(gm[1]) + __popc(gm[2]) + __popc(gm[3]);
+      uint32_t x = ps;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t y = __shfl_up_sync(FULL, x, off);
+        if (lane >= off) x += y;
+      }
+      uint32_t pos = ob + x - ps;
+#pragma unroll
+      for (int i = 0; i < 4; i++) {
+        uint32_t sm = gm[i];
         while (sm) {
           const int bb = __ffs(sm) - 1;
           sm &= sm - 1;
-          if (pos < K) a.out_idx[pos] = (int32_t)(jb + bb);
+          if (pos < K) a.out_idx[pos] = (int32_t)(jl + 32 * i + bb);
           else MV_DBG(a.dbg, MV_DBG_OUT_RANGE);
           pos++;
         }
-        orun += __shfl_sync(FULL, x, 31);
       }
     }
   }
