@@ -87,6 +87,26 @@ def test_add_drop_from_given_votes():
     run_steps(N, d, K, K_ad, steps=4, kind="gauss", seed=5, prev0=prev0)
 
 
+@pytest.mark.parametrize("mode", [B.MV_MODE_AUTO, B.MV_MODE_TRACK], ids=["auto", "track"])
+def test_add_drop_from_full_votes_across_boundaries(mode):
+    """Starting masks with exactly K members (the most the contract allows), among them runs of coordinates that
+    straddle a chunk boundary, word boundaries and the end of the row: the streaming pass lists every member with
+    its key (the drop selection reads |acc| there), and that list is full to the last slot."""
+    N, d, K, K_ad = 4, 20011, 400, 40
+    rng = np.random.default_rng(2)
+    prev0 = np.zeros((N, d), dtype=bool)
+    prev0[:, 4090:4102] = True
+    prev0[:, 8191:8193] = True
+    prev0[:, 63:66] = True
+    prev0[:, d - 5:] = True
+    for n in range(N):
+        free = np.flatnonzero(~prev0[n])
+        prev0[n, rng.choice(free, size=K - int(prev0[n].sum()) - (3 * n if n else 0), replace=False)] = True
+    assert prev0[0].sum() == K
+    run_steps(N, d, K, K_ad, steps=4, kind="gauss", seed=6, prev0=prev0, mode=mode)
+    run_steps(N, d, K, K_ad, steps=3, kind="ties", seed=7, prev0=prev0, mode=mode, want_lists=False)
+
+
 def test_add_drop_without_sampling():
     run_steps(3, 50021, 500, 50, steps=3, kind="gauss", seed=9, mode=B.MV_MODE_GENERAL)
 
