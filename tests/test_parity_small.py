@@ -721,3 +721,20 @@ def test_a_wait_that_was_given_up_is_reported(N, d, K):
     ctx.close()
     ctx2 = B.MvContext(N, d, K, device=DEV)
     PT.compare_all(ctx2, grads.to(DEV), err.to(DEV), K, label="[after a reported timeout] ")
+
+
+@pytest.mark.parametrize("d,K", [(3001, 30), (50_021, 500)], ids=["one-kernel step", "single-kernel tail"])
+def test_one_cta_per_worker_at_the_device_limit(d, K):
+    """As many workers as the device has multiprocessors: the largest cooperative grid of the one-kernel step (a
+    CTA per worker) and, for the longer row, the single-kernel tail with a single CTA serving each worker; one
+    worker more and the step takes the kernel sequence.  All against the oracle."""
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    for N in (sms, min(sms + 1, 255)):
+        grads, err = make(N, d, "gauss", seed=N + d)
+        ctx = B.MvContext(N, d, K, device=DEV, mode=B.MV_MODE_TRACK)
+        ref = O.mv_sparse_step(grads.numpy(), err.numpy(), K, threads=8)
+        PT.compare_all(ctx, grads.to(DEV), err.to(DEV), K, ref=ref, label=f"[N={N} d={d}] ")
+        ctx.set_tail_kernel(2)
+        fu = PT.run_step(ctx, grads.to(DEV), err.to(DEV), K)
+        few = 1 if d <= 32768 else 2
+        assert (fu["launches"] <= few + 1) == (N <= sms), (N, fu["launches"])
