@@ -187,3 +187,35 @@ def test_crowded_threshold_bin_in_the_single_kernel_tail():
     ref = O.mv_sparse_step(PT.npy(grads), PT.npy(err0), K, threads=THREADS)
     assert (ref["thresh"][:, 2] > ref["thresh"][:, 1] * 0 + 1).all()       # T_n is shared by several elements
     PT.compare_all(ctx, grads, err0, K, ref=ref, label="[crowded bin] ")
+
+
+def test_row_one_chunk_beyond_the_single_kernel_tail():
+    """d = 2^27 + 4097: one chunk more than the persistent kernel's table of output offsets holds, so the step with
+    K = d / 100 takes the kernel sequence (ten kernels with the grid-wide select for candidate buffers this large),
+    while the same call on d = 2^27 takes two kernels.  Two workers, rows streamed through the oracle one by one."""
+    N, d = 2, (1 << 27) + 4097
+    K = d // 100
+    g = torch.Generator(device=DEV).manual_seed(99)
+    grads = torch.randn((N, d), generator=g, device=DEV)
+    err = torch.zeros((N, d), device=DEV)
+    ctx = B.MvContext(N, d, K, device=DEV)
+    out_idx = torch.empty(K, dtype=torch.int32, device=DEV)
+    out_val = torch.empty(K, dtype=torch.float32, device=DEV)
+    ctx.mv_sparse_step(grads, err, out_idx, out_val)
+    torch.cuda.synchronize()
+    assert ctx.last_launches() > 3
+    sup = []
+    for n in range(N):
+        idx, T, cnt_gt, cnt_eq = O.worker_topk(PT.npy(grads[n]), K)
+        sup.append(idx)
+    votes = np.zeros(d, dtype=np.uint8)
+    for idx in sup:
+        votes[idx.astype(np.int64)] += 1
+    ref_idx = O.select_mask(votes, K)[0]
+    PT.first_diff(PT.npy(out_idx), ref_idx, "out_idx")
+    cols = torch.from_numpy(ref_idx.astype(np.int64)).to(DEV)
+    acc_cols = np.stack([PT.npy(grads[n][cols]) for n in range(N)])
+    PT.check_out_val(PT.npy(out_val), O.aggregate(acc_cols, np.arange(K)), acc_cols, np.arange(K), "out_val")
+    for n in range(N):
+        want = O.residual(PT.npy(grads[n])[None, :], ref_idx)[0]
+        PT.first_diff(PT.bits(PT.npy(err[n])), PT.bits(want), f"err row {n}")
