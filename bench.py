@@ -16,6 +16,7 @@ spreads the workload's N workers over the ranks and all-reduces the votes and th
 from __future__ import annotations
 
 import argparse
+import contextlib
 import hashlib
 import json
 import os
@@ -456,6 +457,20 @@ def measure(w: WL.Workload, args, B, dev, dist, world, local_rank, with_e2e: boo
     return out
 
 
+@contextlib.contextmanager
+def stdout_to_stderr():
+    """File descriptor 1 points at stderr inside the block (libraries that print while they start up write there)."""
+    sys.stdout.flush()
+    saved = os.dup(1)
+    os.dup2(2, 1)
+    try:
+        yield
+    finally:
+        sys.stdout.flush()
+        os.dup2(saved, 1)
+        os.close(saved)
+
+
 def shard_rows(N: int, world: int, rank: int):
     """Rows [lo, hi) of the N workers that rank `rank` of `world` holds in the worker-sharded step."""
     return rank * N // world, (rank + 1) * N // world
@@ -481,7 +496,10 @@ def run_sharded(args, w: WL.Workload):
     torch.cuda.set_device(dev)
     os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
     os.environ.setdefault("MASTER_PORT", "29655")
-    dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
+    with stdout_to_stderr():     # (the NCCL version banner must not share stdout with the JSON line)
+        dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
+        dist.barrier()
+        torch.cuda.synchronize()
 
     def barrier():
         dist.barrier()
@@ -626,7 +644,10 @@ def main():
     if world > 1:
         import torch.distributed as dist_mod
         dist = dist_mod
-        dist.init_process_group("nccl", device_id=dev)
+        with stdout_to_stderr():     # (the NCCL version banner must not share stdout with the JSON line)
+            dist.init_process_group("nccl", device_id=dev)
+            dist.barrier()
+            torch.cuda.synchronize()
 
     res = measure(w, args, B, dev, dist, world, local_rank, with_e2e=not args.no_e2e and args.method == "mv")
     also = {}
