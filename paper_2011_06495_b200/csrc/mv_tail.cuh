@@ -224,22 +224,24 @@ __global__ void __launch_bounds__(FT, 1) k_tail(P p, TailArgs a) {
   uint32_t* lidx = p.hist2b + (size_t)(has ? n : 0) * H2_BINS; // ... and their coordinates
 
   // ---- window histogram: candidates within 2^22 of tau_n, in 2048 bins of 2^11 keys ----
+  const bool idx_kept = len <= (uint32_t)(SK_KEYS / 2);  // the slice's coordinates fit beside its keys: the picks need no second read
   if (has && fast) {
     for (int bb = tid; bb < H1_BINS; bb += FT) s_hw[bb] = 0;
     __syncthreads();
     for (uint32_t l0 = 0; l0 < len; l0 += FT * 8) {  // uniform over the CTA
-      uint32_t k[8];
+      uint2 k[8];
 #pragma unroll
       for (int q = 0; q < 8; q++) {
         const uint32_t li = l0 + q * FT + tid;
-        k[q] = li < len ? __ldcg(&cd[s0 + li].x) : 0u;
+        k[q] = li < len ? __ldcg(&cd[s0 + li]) : make_uint2(0u, 0u);
       }
 #pragma unroll
       for (int q = 0; q < 8; q++) {
         const uint32_t li = l0 + q * FT + tid;
         if (li < len) {
-          if (li < SK_KEYS) s_keys[li] = k[q];
-          const uint32_t wb = (k[q] - tau) >> WIN_SHIFT;
+          if (li < SK_KEYS) s_keys[li] = k[q].x;
+          if (idx_kept) s_keys[SK_KEYS / 2 + li] = k[q].y;  // (a slice of at most SK_KEYS / 2 keeps its coordinates too)
+          const uint32_t wb = (k[q].x - tau) >> WIN_SHIFT;
           if (wb < (uint32_t)H1_BINS) atomicAdd(&s_hw[wb], 1u);
         }
       }
@@ -275,7 +277,7 @@ __global__ void __launch_bounds__(FT, 1) k_tail(P p, TailArgs a) {
             const uint32_t at = atomicAdd(lcnt, 1u);
             if (at < (uint32_t)WIN_LIST) {
               list[at] = kk;
-              lidx[at] = __ldcg(&cd[s0 + li].y);
+              lidx[at] = idx_kept ? s_keys[SK_KEYS / 2 + li] : __ldcg(&cd[s0 + li].y);
             } else {
               MV_DBG(a.dbg, MV_DBG_INTERNAL);
             }
@@ -529,7 +531,8 @@ __global__ void __launch_bounds__(FT, 1) k_tail(P p, TailArgs a) {
 #pragma unroll
         for (int q = 0; q < 4; q++) {
           const uint32_t li = l0 + q * FT + tid;
-          kv[q] = li < len ? __ldcg(&cd[s0 + li]) : make_uint2(0u, 0u);
+          kv[q] = make_uint2(0u, 0u);
+          if (li < len) kv[q] = idx_kept ? make_uint2(s_keys[li], s_keys[SK_KEYS / 2 + li]) : __ldcg(&cd[s0 + li]);
         }
 #pragma unroll
         for (int q = 0; q < 4; q++) {
