@@ -105,6 +105,10 @@ struct P {
   uint32_t* tie_take;     // [nchunks]
   uint32_t* dbg;          // checked build (MV_DEBUG): status word that collects MV_DBG_* bits, or null
   uint32_t* fb_total;     // running count of worker selections that went over the full row (or null)
+  uint4* zero2_ptr;       // k_set_bits, optional: a region that the kernels after it (the lists of the add-drop and
+  uint32_t zero2_vecs;    //   random-selection variants) want cleared, in 16-byte units (a memset between two kernels
+                          //   would keep the second from being launched while the first still runs)
+  int all_chunks;         // k_votes: visit every chunk, whatever p.hot says
 };
 
 // Checked build: a kernel that clamps, skips or falls back says so by setting a bit of the status word
@@ -1119,6 +1123,11 @@ __device__ __forceinline__ void fullrow_picks(const P& p, int n, float* __restri
 __global__ void __launch_bounds__(TPB) k_set_bits(P p, float* __restrict__ err) {
   pdl_enter();
   __shared__ uint32_t s_we[1][9];
+  if (p.zero2_ptr != nullptr) {
+    const uint32_t nthreads = gridDim.x * gridDim.y * TPB;
+    for (uint32_t i = (blockIdx.y * gridDim.x + blockIdx.x) * TPB + threadIdx.x; i < p.zero2_vecs; i += nthreads)
+      p.zero2_ptr[i] = make_uint4(0, 0, 0, 0);
+  }
   const int n = blockIdx.y;
   const bool fast = worker_fast(p, n);
   if (p.list_mode && !fast) {  // empty list
@@ -1615,7 +1624,7 @@ __global__ void __launch_bounds__(VT) k_votes(P p) {
   __shared__ uint32_t s_sel[256];
   const int tid = threadIdx.x, lane = tid & 31;
   for (int c = blockIdx.x; c < p.nchunks; c += gridDim.x) {
-    if (__ldcg(p.hot + c) == 0) continue;  // uniform over the CTA
+    if (!p.all_chunks && __ldcg(p.hot + c) == 0) continue;  // uniform over the CTA
     __syncthreads();                       // previous chunk's readers are done
     s_vh[tid] = 0;
     s_vh[tid + VT] = 0;
@@ -2256,8 +2265,11 @@ __device__ __forceinline__ double neg_log_u(uint32_t x) {
 // (0x7fffffff - ring time bits, index): the list-mode select then keeps the K largest keys, i.e. the
 // K earliest times.
 __global__ void __launch_bounds__(TPB) k_rs_fill(P p, P a, const uint8_t* __restrict__ votes, uint32_t seed_lo,
-                                                 uint32_t seed_hi, uint32_t draw_lo, uint32_t draw_hi) {
+                                                 uint32_t seed_hi, uint32_t draw_lo, uint32_t draw_hi,
+                                                 int32_t* __restrict__ fill_idx) {
   pdl_enter();
+  // the index list starts out as all -1 (entries that no selected coordinate fills stay so)
+  for (int64_t i = (int64_t)blockIdx.x * TPB + threadIdx.x; i < p.K; i += (int64_t)gridDim.x * TPB) fill_idx[i] = -1;
   __shared__ uint32_t s_w[TPB / 32 + 1];
   __shared__ uint32_t s_base;
   __shared__ uint16_t s_off[CH];  // offset of the coordinate within the chunk
@@ -2549,6 +2561,9 @@ P make_params(const mv_ctx* ctx, const Layout& L, int N, int64_t d, int64_t K) {
   p.tie_take = (uint32_t*)(b + L.tie_take);
   p.dbg = kChecked ? (uint32_t*)(b + L.dbg) : nullptr;
   p.fb_total = (uint32_t*)(b + L.fb_total);
+  p.zero2_ptr = nullptr;
+  p.zero2_vecs = 0;
+  p.all_chunks = 0;
   return p;
 }
 
@@ -3389,11 +3404,14 @@ int mv_ad_step(mv_ctx* ctx, const float* grads, float* err, uint32_t* prev_bits,
   ctx->last_N = N;
   ctx->last_d = d;
   ctx->last_K = K;
+  char* b = ctx->ws;
+  // without add/drop outputs the picks update the vote masks in place (set for add, clear for drop);
+  // otherwise they are materialised as 2N masks first and applied by k_ad_apply
+  const bool direct = add_bits == nullptr && drop_bits == nullptr;
   // this step's top-K masks M_n (kept in the workspace); err now holds acc
   rc = vote_impl(ctx, p, L, grads, err, true);
   if (rc != MV_OK) return rc;
   // the add and drop selections: 2N lists through the select kernels in list mode
-  char* b = ctx->ws;
   P a = p;
   a.N = 2 * N;
   a.K = K_ad;
@@ -3415,10 +3433,9 @@ int mv_ad_step(mv_ctx* ctx, const float* grads, float* err, uint32_t* prev_bits,
   a.chunk_eq = (uint32_t*)(b + L.ad_chunk_eq);
   a.tie_base = (uint32_t*)(b + L.ad_tie_base);
   a.apply_rows = N;
-  // without add/drop outputs the picks update the vote masks in place (set for add, clear for drop);
-  // otherwise they are materialised as 2N masks first and applied by k_ad_apply
-  const bool direct = add_bits == nullptr && drop_bits == nullptr;
   a.apply_bits = direct ? prev_bits : nullptr;
+  // (the list state is cleared by a memset here, not by the picks kernel as in the random-selection step: measured,
+  // the step is 4 us faster this way -- the memset keeps the list fill from being launched while the picks still run)
   if (cudaMemsetAsync(b + L.ad_zero, 0, direct ? L.ad_bits - L.ad_zero : L.ad_zero_bytes, st) != cudaSuccess)
     return MV_ERR_CUDA;
   launch_k(k_ad_fill, dim3(dim3((p.nchunks + TPB / 32 - 1) / (TPB / 32), N)), dim3(TPB), st, p, a,
@@ -3499,13 +3516,19 @@ P list_params(const mv_ctx* ctx, const Layout& L, const P& p, int rows, int64_t 
   a.tie_base = (uint32_t*)(b + L.ad_tie_base);
   a.apply_rows = 0;
   a.apply_bits = nullptr;
+  a.zero2_ptr = nullptr;
+  a.zero2_vecs = 0;
   return a;
 }
 
+// bytes of list state that a random selection wants clear: the select state and one row of mask words (whole 16-byte units)
+size_t rs_zero_bytes(const Layout& L, int64_t W) { return (((L.ad_bits - L.ad_zero) + (size_t)W * 4) + 15) & ~(size_t)15; }
+
 // S_rand-weighted: voted coordinates with their ring times into one list, the K earliest through the
 // list-mode select into a bit mask, the mask into an ascending index list
+// `cleared`: the list state was cleared by the picks kernel of the step that calls (p.zero2_ptr)
 int rs_select_impl(mv_ctx* ctx, const P& p, const Layout& L, const uint8_t* votes, uint64_t seed, uint64_t draw,
-                   int32_t* out_idx, uint32_t* mask_bits) {
+                   int32_t* out_idx, uint32_t* mask_bits, bool cleared = false) {
   cudaStream_t st = ctx->stream;
   char* b = ctx->ws;
   // The list regions written here sit at offsets of this call's own (N, d, K): they may overlap the
@@ -3516,10 +3539,9 @@ int rs_select_impl(mv_ctx* ctx, const P& p, const Layout& L, const uint8_t* vote
   // one list that can hold every voted coordinate (at most min(d, N K) of them)
   const uint64_t room = (uint64_t)2 * (uint64_t)p.N * (uint64_t)L.ad_cap;
   P a = list_params(ctx, L, p, 1, p.K, (uint32_t)(room < 0xfffffff8ull ? room : 0xfffffff8ull));
-  if (cudaMemsetAsync(b + L.ad_zero, 0, (L.ad_bits - L.ad_zero) + (size_t)p.W * 4, st) != cudaSuccess) return MV_ERR_CUDA;
-  if (cudaMemsetAsync(out_idx, 0xff, (size_t)p.K * 4, st) != cudaSuccess) return MV_ERR_CUDA;
+  if (!cleared && cudaMemsetAsync(b + L.ad_zero, 0, rs_zero_bytes(L, p.W), st) != cudaSuccess) return MV_ERR_CUDA;
   launch_k(k_rs_fill, dim3(p.nchunks), dim3(TPB), st, p, a, votes, (uint32_t)seed, (uint32_t)(seed >> 32), (uint32_t)draw,
-           (uint32_t)(draw >> 32));
+           (uint32_t)(draw >> 32), out_idx);
   MV_LAUNCH_CHECK();
   uint64_t most = (uint64_t)p.N * (uint64_t)p.K;
   if (most > (uint64_t)p.d) most = (uint64_t)p.d;
@@ -3585,9 +3607,13 @@ int mv_rs_step(mv_ctx* ctx, const float* grads, float* err, int N, int64_t d, in
   ctx->last_N = N;
   ctx->last_d = d;
   ctx->last_K = K;
+  // (the picks kernel also clears the list state of the selection that follows)
+  p.zero2_ptr = (uint4*)(ctx->ws + L.ad_zero);
+  p.zero2_vecs = (uint32_t)(rs_zero_bytes(L, L.W) / 16);
   rc = vote_impl(ctx, p, L, grads, err, false, false, false, false);  // the random selection reads the votes themselves
+  p.zero2_ptr = nullptr;
   // the union of N top-K sets holds at least K coordinates, so the mask is always full
-  if (rc == MV_OK) rc = rs_select_impl(ctx, p, L, p.votes, seed, draw, out_idx, nullptr);
+  if (rc == MV_OK) rc = rs_select_impl(ctx, p, L, p.votes, seed, draw, out_idx, nullptr, true);
   if (rc == MV_OK) rc = aggregate_impl(ctx, err, N, d, K, out_idx, out_val, L.zero_bytes);
   const int rcj = join_side(ctx);
   return rc != MV_OK ? rc : rcj;
