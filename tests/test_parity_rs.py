@@ -127,3 +127,35 @@ def test_rs_step_matches_the_oracle(name, d, N, K):
         masks.append(ref["out_idx"])
         # not the K most voted: the random mask differs from the deterministic one
         assert not np.array_equal(ref["out_idx"], O.select_mask(ref["votes"], w.K)[0])
+
+
+@pytest.mark.parametrize("mode", [B.MV_MODE_AUTO, B.MV_MODE_GENERAL], ids=["auto", "general"])
+def test_rs_step_in_the_other_threshold_modes(mode):
+    """The whole random-selection step with the threshold sampled every call and with no sampling at all (the picks
+    kernel of either route clears the list state of the selection that follows), a stand-alone selection of another
+    size in between (which clears that state by itself), against the oracle."""
+    w = WL.scaled(WL.resnet_like("c2"), d=200_003, N=5, K=2000, steps=3)
+    ctx = B.MvContext(w.N, w.d, w.K, device=DEV, mode=mode)
+    err = WL.initial_err(w, device=DEV)
+    err_ref = err.cpu().numpy()
+    out_idx = torch.empty(w.K, dtype=torch.int32, device=DEV)
+    out_val = torch.empty(w.K, dtype=torch.float32, device=DEV)
+    g = torch.Generator().manual_seed(8)
+    for step in range(w.steps):
+        grads = WL.gradients(w, step, device=DEV)
+        ref = R.mv_rs_step(grads.cpu().numpy(), err_ref, w.K, seed=77, draw=step, threads=8)
+        ctx.mv_rs_step(grads, err, 77, step, out_idx, out_val)
+        torch.cuda.synchronize()
+        tag = f"[rs step {step}] "
+        PT.first_diff(PT.npy(out_idx), ref["out_idx"], tag + "out_idx")
+        PT.check_out_val(PT.npy(out_val), ref, ref["acc"], ref["out_idx"].astype(np.int64), tag + "out_val")
+        PT.first_diff(PT.bits(PT.npy(err)), PT.bits(ref["err"]), tag + "err")
+        err_ref = ref["err"]
+        if step == 0:
+            d2, K2 = 50_021, 300
+            votes2 = (torch.randint(1, w.N + 1, (d2,), generator=g) * (torch.rand(d2, generator=g) < 0.02)).to(torch.uint8).to(DEV)
+            assert K2 <= int((votes2 > 0).sum()) <= w.N * K2
+            oi2 = torch.empty(K2, dtype=torch.int32, device=DEV)
+            ctx.mv_select_rs(votes2, w.N, 5, 9, oi2, K=K2)
+            torch.cuda.synchronize()
+            assert np.array_equal(oi2.cpu().numpy(), R.select_mask_rs(votes2.cpu().numpy(), K2, seed=5, draw=9))
